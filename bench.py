@@ -1,0 +1,428 @@
+#!/usr/bin/env python
+"""Benchmark of the BCR sparse multiply on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload gru|gemv|spmm|conv] [--impl ours|reference]
+
+One "step" is one pass of the whole hot path over one batch of seeded synthetic input.  The default
+workload is the GRU configuration (2 layers, hidden 1024, 153 input features, T = 200, 8x32 blocks, 10x
+compression): two hoisted sparse projections plus two persistent recurrent kernels.  The metric is
+effective GFLOP/s = 2 * nnz * N / time (N = number of right-hand-side columns / time steps).
+
+Prints ONE JSON line (rank 0).  `--impl reference` times the CPU oracle instead (a deliberately plain
+dense fp64 program; its ratio to the GPU number says nothing about kernel quality).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "BCR SpMM/GEMV effective GFLOP/s (2*nnz*N)"
+UNIT = "GFLOP/s"
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(suffix=".csv")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu)], stdout=fd, stderr=subprocess.DEVNULL)
+            os.close(fd)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = dict(sm_mhz=None, sm_max_mhz=None, reasons=[], samples=0)
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        try:
+            rows = [l.strip().split(", ") for l in open(self.path) if l.strip()]
+            os.unlink(self.path)
+            sm = [float(r[1]) for r in rows]
+            names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+            reasons = sorted({n for r in rows for n, v in zip(names, r[5:9]) if v.strip().lower() == "active"})
+            out = dict(sm_mhz=statistics.median(sm) if sm else None, sm_max_mhz=float(rows[0][2]) if rows else None,
+                       reasons=reasons, samples=len(rows))
+        except Exception:
+            pass
+        return out
+
+
+# ------------------------------------------------------------------------------------------------ workloads
+
+
+class GruWorkload:
+    name = "gru_2x1024_in153_T200_bcr8x32_c10_fp32"
+    dtype = "f32"
+
+    def __init__(self, sample_T=200):
+        from workloads import generators as gen
+        self.m = gen.gru_model()
+        self.T, self.H = self.m["T"], self.m["hidden"]
+        self.nnz = sum(int(l["mask_ih"].sum()) + int(l["mask_hh"].sum()) for l in self.m["layers"])
+        self.flops = 2.0 * self.nnz * self.T
+        self.sample_T = sample_T
+
+    def setup(self, B, torch):
+        m = self.m
+        self.B, self.torch = B, torch
+        self.hi = [B.grim_bcr_pack(l["W_ih"], l["mask_ih"], m["bh"], m["bw"], B.GRIM_F32, B.GRIM_PACK_REORDER) for l in m["layers"]]
+        self.hh = [B.grim_bcr_pack(l["W_hh"], l["mask_hh"], m["bh"], m["bw"], B.GRIM_F32, B.GRIM_PACK_REORDER) for l in m["layers"]]
+        self.g = B.grim_gru_create(self.hi, self.hh, [l["b_ih"] for l in m["layers"]], [l["b_hh"] for l in m["layers"]], self.T)
+        self.x_host = torch.from_numpy(m["x"]).pin_memory()
+        self.y_host = torch.empty(self.T, self.H).pin_memory()
+        self.x = self.x_host.cuda()
+        self.y = torch.empty(self.T, self.H, device="cuda")
+        B.grim_gru_profile(self.g, True)
+        # algorithmic bytes of the recurrent kernel (dominant): per step the kept values and their index
+        # words of W_hh, the three pre-activation rows, h read and h written; summed over the layers
+        self.kernel_bytes = 0.0
+        for hh in self.hh:
+            i = B.grim_bcr_info(hh)
+            self.kernel_bytes += self.T * (i.value_bytes + i.index_bytes_gemv + 3 * self.H * 4 + 2 * self.H * 4)
+        self.h2d = self.x_host.numel() * 4
+        self.d2h = self.y_host.numel() * 4
+        self.kernel = "gru_recurrent_kernel"
+        self.bound = "hbm"
+
+    def step(self):
+        self.B.grim_gru_seq(self.g, self.x, self.y)
+
+    def step_e2e(self):
+        xd = self.x_host.cuda(non_blocking=True)
+        self.B.grim_gru_seq(self.g, xd, self.y)
+        self.y_host.copy_(self.y, non_blocking=True)
+
+    def kernel_ms(self):
+        return self.B.grim_gru_profile_read(self.g)[1]
+
+    def check(self):
+        assert self.B.grim_gru_status(self.g) == self.B.GRIM_OK
+
+    def oracle_sample(self):
+        from oracle import bcr_oracle as orc
+        Ts = self.sample_T
+        t0 = time.perf_counter()
+        orc.gru_seq(self.m["layers"], self.m["x"][:Ts])
+        dt = time.perf_counter() - t0
+        return 2.0 * self.nnz * Ts / dt / 1e9, f"first {Ts} of {self.T} time steps, both layers, dense fp64 NumPy mat-vec"
+
+
+class SpmmWorkload:
+    """One point of the SpMM sweep (square W).  N = 1 runs the matrix-vector kernel."""
+
+    def __init__(self, M=8192, N=1, c=8.0, bh=8, bw=32, dist="uniform", bf16=False, conv=False):
+        from workloads import generators as gen
+        self.M, self.N, self.bf16 = M, N, bf16
+        self.s = gen.sweep_case(M, N, c, bh, bw, dist, bf16=bf16)
+        self.bh, self.bw = bh, bw
+        self.name = f"spmm_M{M}_K{M}_N{N}_c{c:g}_{bh}x{bw}_{dist}_{'bf16' if bf16 else 'fp32'}"
+        self.dtype = "bf16" if bf16 else "f32"
+        self.nnz = int(self.s["mask"].sum())
+        self.flops = 2.0 * self.nnz * N
+        self.copies = 1
+
+    def setup(self, B, torch):
+        self.B, self.torch = B, torch
+        s = self.s
+        dt = B.GRIM_BF16 if self.bf16 else B.GRIM_F32
+        self.h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, B.GRIM_PACK_REORDER)
+        tdt = torch.bfloat16 if self.bf16 else torch.float32
+        self.x_host = torch.from_numpy(s["X"]).to(tdt).pin_memory()
+        self.x = self.x_host.cuda()
+        self.y = torch.empty(self.M, self.N, device="cuda")
+        self.y_host = torch.empty(self.M, self.N).pin_memory()
+        i = B.grim_bcr_info(self.h)
+        esz = 2 if self.bf16 else 4
+        idx = i.index_bytes_gemv if self.N == 1 else i.index_bytes_spmm
+        self.kernel_bytes = float(i.value_bytes + idx + i.k_used * self.N * esz + self.M * self.N * 4)
+        self.h2d = self.x_host.numel() * esz
+        self.d2h = self.y_host.numel() * 4
+        self.kernel = "bcr_gemv_kernel" if self.N == 1 else "bcr_spmm_kernel"
+        self.bound = "hbm" if self.N <= 16 else "alu"
+        self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+
+    def step(self):
+        self._ev[0].record()
+        self.B.grim_bcr_spmm(self.h, self.x, self.y)
+        self._ev[1].record()
+
+    def step_e2e(self):
+        xd = self.x_host.cuda(non_blocking=True)
+        self.B.grim_bcr_spmm(self.h, xd, self.y)
+        self.y_host.copy_(self.y, non_blocking=True)
+
+    def kernel_ms(self):
+        self._ev[1].synchronize()
+        return self._ev[0].elapsed_time(self._ev[1])
+
+    def check(self):
+        pass
+
+    def oracle_sample(self):
+        from oracle import bcr_oracle as orc
+        n = min(self.N, 64)
+        t0 = time.perf_counter()
+        orc.spmm(self.s["W"], self.s["mask"], self.s["X"][:, :n], 1 if self.bf16 else 0)
+        dt = time.perf_counter() - t0
+        return 2.0 * self.nnz * n / dt / 1e9, f"first {n} of {self.N} columns, masked dense fp64 NumPy matmul"
+
+
+class ConvWorkload:
+    def __init__(self, batch=32, bf16=False):
+        from workloads import generators as gen
+        self.L = gen.conv_layer(batch, 512, 512, 28, bf16=bf16)
+        self.batch, self.bf16 = batch, bf16
+        self.name = f"conv3x3_512to512_28x28_b{batch}_bcr16x64_c8_{'bf16' if bf16 else 'fp32'}"
+        self.dtype = "bf16" if bf16 else "f32"
+        self.nnz = int(self.L["mask"].sum())
+        self.flops = 2.0 * self.nnz * batch * 28 * 28
+
+    def setup(self, B, torch):
+        self.B, self.torch = B, torch
+        L = self.L
+        dt = B.GRIM_BF16 if self.bf16 else B.GRIM_F32
+        tdt = torch.bfloat16 if self.bf16 else torch.float32
+        self.h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, dt, B.GRIM_PACK_REORDER)
+        self.x_host = torch.from_numpy(L["x"]).to(tdt).pin_memory()
+        self.x = self.x_host.cuda()
+        self.bias = torch.from_numpy(L["bias"]).cuda()
+        self.y = torch.empty(self.batch, 512, 28, 28, device="cuda", dtype=tdt)
+        self.y_host = torch.empty(self.batch, 512, 28, 28, dtype=tdt).pin_memory()
+        i = B.grim_bcr_info(self.h)
+        esz = 2 if self.bf16 else 4
+        self.kernel_bytes = float(i.value_bytes + i.index_bytes_spmm + self.x.numel() * esz + self.y.numel() * esz)
+        self.h2d = self.x_host.numel() * esz
+        self.d2h = self.y_host.numel() * esz
+        self.kernel = "bcr_spmm_kernel<conv>"
+        self.bound = "alu"
+        self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+
+    def step(self):
+        self._ev[0].record()
+        self.B.grim_bcr_conv2d(self.h, self.x, self.y, 3, 1, 1, bias=self.bias, relu=True)
+        self._ev[1].record()
+
+    def step_e2e(self):
+        xd = self.x_host.cuda(non_blocking=True)
+        self.B.grim_bcr_conv2d(self.h, xd, self.y, 3, 1, 1, bias=self.bias, relu=True)
+        self.y_host.copy_(self.y, non_blocking=True)
+
+    def kernel_ms(self):
+        self._ev[1].synchronize()
+        return self._ev[0].elapsed_time(self._ev[1])
+
+    def check(self):
+        pass
+
+    def oracle_sample(self):
+        from oracle import bcr_oracle as orc
+        L = self.L
+        t0 = time.perf_counter()
+        orc.conv2d(L["W"], L["mask"], L["x"][:1], L["bias"], ksize=3, stride=1, pad=1, relu=True, dtype=1 if self.bf16 else 0)
+        dt = time.perf_counter() - t0
+        return 2.0 * self.nnz * 28 * 28 / dt / 1e9, f"1 of {self.batch} images, direct fp64 NumPy convolution with the masked dense weight"
+
+
+def make_workload(args):
+    w = args.workload
+    if w == "gru":
+        return GruWorkload()
+    if w == "gemv":
+        return SpmmWorkload(M=args.size, N=1, c=args.compression, bh=args.bh, bw=args.bw, dist=args.dist, bf16=args.bf16)
+    if w == "spmm":
+        return SpmmWorkload(M=args.size, N=args.ncols, c=args.compression, bh=args.bh, bw=args.bw, dist=args.dist, bf16=args.bf16)
+    if w == "conv":
+        return ConvWorkload(batch=args.batch, bf16=args.bf16)
+    raise SystemExit(f"unknown workload {w}")
+
+
+# ------------------------------------------------------------------------------------------------ arms
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    wl = make_workload(args)
+    if isinstance(wl, GruWorkload):
+        wl.sample_T = 50
+    for _ in range(args.warmup):
+        wl.oracle_sample()
+    vals, t0 = [], time.perf_counter()
+    for _ in range(args.steps):
+        v, what = wl.oracle_sample()
+        vals.append(v)
+    total = time.perf_counter() - t0
+    # harmonic mean over steps = total work / total time
+    value = len(vals) / sum(1.0 / v for v in vals)
+    cores = len(os.sched_getaffinity(0))
+    line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=args.gpus, steps=args.steps, warmup=args.warmup,
+                ms_per_step=1e3 * total / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                dtype="f64", data="synthetic", impl="reference",
+                config=dict(workload=wl.name, note="CPU oracle; each step is a bounded sample of the workload"),
+                cpu_baseline=dict(value=value, unit=UNIT, cores=cores, kind="oracle", sample=what),
+                e2e=dict(value=value, unit=UNIT, h2d_bytes_per_step=0, d2h_bytes_per_step=0), gpu_launches=0)
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    from paper_2108_11033_b200.build import build_library
+    build_library()
+    from paper_2108_11033_b200 import binding as B
+
+    wl = make_workload(args)
+    wl.setup(B, torch)
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")  # > L2 (126 MB)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        wl.step()
+    wl.check()
+    barrier()
+
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    B.grim_launch_count_reset()
+    kernel_ms = []
+    barrier()
+    for k in range(args.steps):
+        flush.zero_()  # evict the working set from L2 between timed iterations (not timed)
+        ev[k][0].record()
+        wl.step()
+        ev[k][1].record()
+        kernel_ms.append(wl.kernel_ms())
+    barrier()
+    launches = B.grim_launch_count()
+    total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    wl.check()
+
+    # end to end: host buffers, copies inside the timed region
+    for _ in range(2):
+        wl.step_e2e()
+    barrier()
+    ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    for k in range(args.steps):
+        flush.zero_()
+        ev2[k][0].record()
+        wl.step_e2e()
+        ev2[k][1].record()
+    barrier()
+    e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
+    clocks = sampler.stop() if rank == 0 else None
+
+    t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_ms = float(t[0]), float(t[1])
+
+    if rank == 0:
+        peaks = measured_peaks()
+        value = world * wl.flops * args.steps / (total_ms * 1e-3) / 1e9
+        e2e_value = world * wl.flops * args.steps / (e2e_ms * 1e-3) / 1e9
+        k_ms = statistics.mean(kernel_ms)
+        if wl.bound == "hbm":
+            achieved = wl.kernel_bytes / (k_ms * 1e-3) / 1e9
+            roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                        traffic=None, kernel=wl.kernel, kernel_ms=k_ms, algorithmic_bytes=wl.kernel_bytes,
+                        peak_source=peaks["source"])
+        else:
+            # plain fp32 FMA pipes: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
+            peak = 148 * 128 * 2 * 1.965e9 / 1e12
+            achieved = wl.flops / (k_ms * 1e-3) / 1e12
+            roof = dict(bound="alu", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
+                        kernel=wl.kernel, kernel_ms=k_ms, peak_source="derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz")
+        cpu_v, cpu_what = wl.oracle_sample()
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+                    ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
+                    dtype=wl.dtype, data="synthetic",
+                    config=dict(workload=wl.name, nnz=wl.nnz, l2="flushed between timed iterations (256 MiB write)",
+                                parallelism="replicas only" if world > 1 else "1 GPU"),
+                    clocks=clocks,
+                    e2e=dict(value=e2e_value, unit=UNIT, h2d_bytes_per_step=wl.h2d, d2h_bytes_per_step=wl.d2h,
+                             ms_per_step=e2e_ms / args.steps),
+                    gpu_launches=int(launches), roofline=roof,
+                    cpu_baseline=dict(value=cpu_v, unit=UNIT, cores=len(os.sched_getaffinity(0)), kind="oracle",
+                                      sample=cpu_what))
+        print(json.dumps(line))
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="gru", choices=["gru", "gemv", "spmm", "conv"])
+    ap.add_argument("--size", type=int, default=8192)
+    ap.add_argument("--ncols", type=int, default=128)
+    ap.add_argument("--compression", type=float, default=8.0)
+    ap.add_argument("--bh", type=int, default=8)
+    ap.add_argument("--bw", type=int, default=32)
+    ap.add_argument("--dist", default="uniform", choices=["uniform", "zipf"])
+    ap.add_argument("--bf16", action="store_true")
+    ap.add_argument("--batch", type=int, default=32)
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

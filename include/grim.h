@@ -1,0 +1,233 @@
+/*
+ * grim.h - C ABI of libgrim: multiply a Block-based Column-Row (BCR) pruned weight matrix by
+ * dense activations on one NVIDIA B200 (sm_100a).
+ *
+ * Background (paper sections are cited per entry point):
+ *   - Section 3.2 defines BCR pruning: the weight matrix W (M x K) is tiled into equal blocks of
+ *     bh rows x bw columns; inside every block whole rows and whole columns are removed
+ *     independently, and what remains of a block is a full kr x kc sub-matrix.
+ *   - Section 3.1 treats every CNN / RNN layer as W times an input matrix (GEMM) or vector (GEMV).
+ *   - Sections 4.2 - 4.5 describe the execution-side ideas this library re-derives for sm_100a:
+ *     row reorder / grouping, a compact storage that shares index lists inside a block, loading
+ *     every needed input row once and reusing it for all kept rows of a block, tiling with
+ *     tuned tile shapes, and convolution as an (implicit) im2col GEMM that skips pruned columns.
+ *
+ * Conventions
+ *   - Every function returns a grim_status_t; nothing aborts or throws across this boundary.
+ *     On failure output handles / buffers are left untouched unless stated otherwise.
+ *   - "host" pointers are ordinary CPU memory, "device" pointers are CUDA global memory of the
+ *     current device.  Handles own the device and host buffers they create; activations, outputs,
+ *     biases passed at call time stay owned by the caller.
+ *   - Compute calls are asynchronous on the given CUDA stream and do not synchronise.  A handle
+ *     must not be used by two streams at the same time (the GRU handle owns scratch buffers).
+ *   - There is no CPU fallback: compute calls need a CUDA device and fail with GRIM_ERR_CUDA
+ *     otherwise.
+ *   - Matrices are row-major.  Block shapes are rows x columns.
+ */
+#ifndef GRIM_H_
+#define GRIM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GRIM_OK = 0,
+  GRIM_ERR_INVALID_ARG = 1, /* null pointer, negative size, bad flag */
+  GRIM_ERR_SHAPE = 2,       /* operand shapes do not match the handle */
+  GRIM_ERR_DTYPE = 3,       /* operand dtype does not match the handle */
+  GRIM_ERR_NOT_BCR = 4,     /* some block's mask is not (kept rows) x (kept columns) */
+  GRIM_ERR_ALLOC = 5,       /* host or device allocation failed */
+  GRIM_ERR_CUDA = 6,        /* a CUDA runtime call failed (no device, launch error, ...) */
+  GRIM_ERR_UNSUPPORTED = 7, /* valid request outside the implemented range */
+  GRIM_ERR_TIMEOUT = 8      /* a bounded device-side wait gave up; results are invalid */
+} grim_status_t;
+
+typedef enum { GRIM_F32 = 0, GRIM_BF16 = 1 } grim_dtype_t;
+
+/* Same object as cudaStream_t (NULL = the legacy default stream). */
+typedef struct CUstream_st* grim_stream_t;
+
+typedef struct grim_bcr* grim_bcr_t; /* a packed BCR weight matrix */
+typedef struct grim_gru* grim_gru_t; /* a multi-layer GRU built from packed matrices */
+
+/* A dense row-major matrix in DEVICE memory: element (r, c) is at ptr[r * ld + c]. */
+typedef struct {
+  void* ptr;
+  int64_t rows, cols, ld;
+  grim_dtype_t dtype;
+} grim_mat_t;
+
+/* grim_bcr_pack flags */
+#define GRIM_PACK_REORDER 1u   /* schedule row bands by decreasing work; export the row permutation */
+#define GRIM_PACK_HOST_ONLY 2u /* build host-side data only (no CUDA call); compute calls then fail */
+
+typedef struct {
+  int64_t M, K;
+  int32_t bh, bw;
+  int64_t nbr, nbc;         /* block grid: ceil(M/bh) x ceil(K/bw) */
+  int64_t nnz;              /* kept weights = sum over blocks of kr*kc (mask count) */
+  int64_t nonempty_blocks;
+  int64_t k_used;           /* columns of W kept by at least one block (input rows actually read) */
+  int32_t dtype;            /* grim_dtype_t of the stored values */
+  uint32_t flags;
+  int32_t on_device;        /* 0 for GRIM_PACK_HOST_ONLY handles */
+  int32_t reserved;
+  int64_t value_bytes;      /* nnz * sizeof(value) */
+  int64_t index_bytes_spmm; /* bytes of block descriptors / tables read by the N > 1 kernels */
+  int64_t index_bytes_gemv; /* bytes of column words / chunk tables read by the N = 1 kernel */
+  int64_t export_bytes;     /* size of the canonical byte string written by grim_bcr_export */
+} grim_bcr_info_t;
+
+/* Tile-shape choice for the N > 1 kernel (Section 4.5: tile sizes are tuned per kernel).
+ * Zero in a field means "library default for this problem". */
+typedef struct {
+  int32_t tile_n;  /* output columns per thread block: 16, 32, 64 or 128 */
+  int32_t path;    /* 0 auto, 1 CUDA-core FFMA tiles, 2 tcgen05 tensor-core tiles (bf16 handles only) */
+  int32_t reserved[6];
+} grim_tune_t;
+
+/* ---------------------------------------------------------------------------------------------
+ * Packing (host).  Section 3.2 (pattern), Sections 4.2 - 4.3 (reorder + compact storage).
+ *
+ * grim_bcr_pack reads a dense fp32 weight W_host[M x K] (row stride ldw) and a keep-mask
+ * mask_host[M x K] (row stride ldm; non-zero = kept) from HOST memory and builds a handle.
+ *   - A row / column of a block counts as kept when any of its entries is kept.  Every block's
+ *     mask must equal (kept rows) x (kept columns), otherwise GRIM_ERR_NOT_BCR.
+ *   - The mask is authoritative: a kept weight whose value is 0.0 stays stored and counted.
+ *   - M or K need not be multiples of bh / bw: edge blocks are smaller (equivalent to zero padding).
+ *   - Blocks that keep nothing are legal and cost nothing.
+ *   - value_dtype GRIM_BF16 rounds the kept weights to bf16 (nearest, ties to even) once, here.
+ *   - Limits: 1 <= bh <= 16, 1 <= bw <= 64, M, K < 2^31, nnz < 2^32; else GRIM_ERR_UNSUPPORTED.
+ *   - Synchronous.  Unless GRIM_PACK_HOST_ONLY is set it allocates device memory on the current
+ *     device and uploads the packed arrays (one blocking copy per array).
+ * W_host and mask_host are only read during the call.
+ */
+grim_status_t grim_bcr_pack(const float* W_host, int64_t ldw, const uint8_t* mask_host, int64_t ldm,
+                            int64_t M, int64_t K, int bh, int bw, grim_dtype_t value_dtype,
+                            uint32_t flags, grim_bcr_t* out);
+
+/* Frees the handle's host and device buffers.  NULL is accepted. */
+grim_status_t grim_bcr_destroy(grim_bcr_t h);
+
+grim_status_t grim_bcr_info(grim_bcr_t h, grim_bcr_info_t* info);
+
+/* Canonical packed form (the compact storage idea of Section 4.3 in a fully specified layout),
+ * written to HOST memory as a little-endian byte string of info.export_bytes bytes:
+ *   8 x int64: magic "GRIMBCR1", M, K, bh, bw, nbr, nbc, dtype
+ *   per block, row-major over the block grid: u16 kr, u16 kc, u16 rows[kr], u16 cols[kc]
+ *     (block-local, ascending), values[kr*kc] row-major over (rows, cols) as fp32 or bf16 bits
+ *   int32 row_perm[M]: with GRIM_PACK_REORDER the rows sorted by kept-weight count, largest
+ *     first, ties by row index (the reorder array of Section 4.3); identity otherwise.
+ * capacity < export_bytes gives GRIM_ERR_INVALID_ARG; *written receives the size.
+ */
+grim_status_t grim_bcr_export(grim_bcr_t h, void* buf_host, int64_t capacity, int64_t* written);
+
+/* Writes the masked weight (zeros at pruned positions; bf16 handles: the rounded values) as
+ * fp32 into HOST memory W_host[M x K], row stride ldw. */
+grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);
+
+/* ---------------------------------------------------------------------------------------------
+ * Y = W * X.  Section 3.1 (unified GEMM / GEMV view), Sections 4.2, 4.4, 4.5 (execution).
+ *
+ * X: K x N, Y: M x N, both DEVICE, row-major with their own ld (>= cols).  X->dtype must equal
+ * the handle's value dtype; Y->dtype is GRIM_F32, or GRIM_BF16 for bf16 handles (rounded once,
+ * after fp32 accumulation).  Y is fully overwritten (all M rows, beta = 0): rows kept by no
+ * block are written as +0.  N = 1 selects the matrix-vector kernel.  X and Y must not overlap.
+ * Shape mismatch -> GRIM_ERR_SHAPE, dtype mismatch -> GRIM_ERR_DTYPE, both before any launch.
+ * Asynchronous on `stream`.
+ */
+grim_status_t grim_bcr_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, grim_stream_t stream);
+
+/* Same with an explicit tile choice (Section 4.5, tuning).  tune may be NULL. */
+grim_status_t grim_bcr_spmm_ex(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune,
+                               grim_stream_t stream);
+
+/* Times the candidate tile shapes for (handle, X/Y shapes and dtypes) on `stream` (synchronises)
+ * and returns the fastest in *best (Section 4.5: per-kernel tuning of tile shape; the paper's
+ * genetic search is replaced by a small fixed candidate set).  Y is overwritten. */
+grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, int reps, grim_tune_t* best,
+                            float* best_ms, grim_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Convolution as an implicit-im2col BCR GEMM.  Section 3.1 (CONV as GEMM), Section 4.5
+ * ("Computation Transformation": rows of the expanded input whose weight column is pruned are
+ * never produced).
+ *
+ * The handle holds the weight viewed as Cout x (C*KH*KW), K axis flattened as
+ * k = (c*KH + kh)*KW + kw.  in: [N, C, H, W], out: [N, Cout, OH, OW] (NCHW, contiguous, DEVICE),
+ * OH = (H + 2*pad - KH)/stride + 1, likewise OW.  out = conv(in) + bias, then max(.,0) if
+ * GRIM_CONV_RELU.  bias_dev: Cout fp32 DEVICE values or NULL.  in_dtype must equal the
+ * handle's dtype; out_dtype GRIM_F32 or (bf16 handles) GRIM_BF16.  Accumulation is fp32.
+ */
+#define GRIM_CONV_RELU 1u
+typedef struct {
+  int64_t N, C, H, W;
+  int32_t KH, KW, stride, pad;
+  const float* bias_dev;
+  uint32_t flags;
+  grim_dtype_t in_dtype, out_dtype;
+} grim_conv_desc_t;
+
+grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d, const void* in_dev, void* out_dev,
+                              grim_stream_t stream);
+
+/* 2x2 / stride-2 max-pool on NCHW DEVICE tensors (H, W even); glue between the conv layers of a
+ * VGG-style stack (Section 6.1 evaluates VGG-16), not part of the sparse multiply itself. */
+grim_status_t grim_maxpool2x2(const void* in_dev, void* out_dev, int64_t N, int64_t C, int64_t H, int64_t W,
+                              grim_dtype_t dtype, grim_stream_t stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * GRU sequence inference, batch 1.  Section 3.1 (RNN layers are matrix-vector products),
+ * Section 6.1 (a 2-layer GRU is the RNN workload).  The paper gives no equations; this is the
+ * common variant with gate order r, z, n in the 3H rows:
+ *   g = W_ih x_t + b_ih,  q = W_hh h_{t-1} + b_hh
+ *   r = sigmoid(g_r + q_r), z = sigmoid(g_z + q_z), n = tanh(g_n + r * q_n)
+ *   h_t = (1 - z) * n + z * h_{t-1};   layer l > 0 takes layer l-1's h_t as its x_t.
+ *
+ * grim_gru_create: W_ih[l] is 3H x in_l, W_hh[l] is 3H x H (fp32 handles packed with the same
+ * bh, H a multiple of bh); b_ih_host[l], b_hh_host[l]: 3H fp32 HOST values (copied).  The packed
+ * matrices are borrowed: they must outlive the GRU handle.  max_T bounds the sequence length;
+ * scratch for the hoisted input projections is allocated here.
+ *
+ * grim_gru_seq: x_dev [T x in_0], h0_dev [layers x H] or NULL (zeros), y_dev [T x H] receives the
+ * last layer's h_t, hT_dev [layers x H] or NULL receives every layer's final state; all fp32
+ * DEVICE.  Asynchronous.  The recurrent kernel keeps W_hh on-chip and exchanges h between thread
+ * blocks every step; all of its waits are bounded.  If one gives up, the outputs are invalid and
+ * grim_gru_status (which synchronises the stream used last) reports GRIM_ERR_TIMEOUT.
+ */
+grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, const grim_bcr_t* W_hh,
+                              const float* const* b_ih_host, const float* const* b_hh_host, int64_t max_T,
+                              grim_gru_t* out);
+grim_status_t grim_gru_seq(grim_gru_t g, const float* x_dev, int64_t T, const float* h0_dev, float* y_dev,
+                           float* hT_dev, grim_stream_t stream);
+grim_status_t grim_gru_status(grim_gru_t g);
+grim_status_t grim_gru_destroy(grim_gru_t g);
+
+/* Test hook for the bounded waits of the recurrent kernel (no counterpart in the paper): thread
+ * block `skip_cta` stays away from the per-step barrier (-1 = normal operation) and a waiting
+ * block gives up after `spin_limit` polls (0 = default).  With a block missing, every wait runs
+ * out, the kernel returns, and grim_gru_status reports GRIM_ERR_TIMEOUT; nothing waits forever. */
+grim_status_t grim_gru_debug_barrier(grim_gru_t g, int skip_cta, unsigned spin_limit);
+
+/* Per-kernel timing of the GRU path (measurement aid, Section 6 reports per-kernel times): when
+ * enabled, grim_gru_seq records CUDA events on its stream around the hoisted input projection and
+ * around the persistent recurrent kernel of every layer.  grim_gru_profile_read waits for the last
+ * call and returns the two sums over layers in milliseconds. */
+grim_status_t grim_gru_profile(grim_gru_t g, int enable);
+grim_status_t grim_gru_profile_read(grim_gru_t g, float* projection_ms, float* recurrent_ms);
+
+/* Counts kernel launches issued by this library since load (or since the last reset). */
+int64_t grim_launch_count(void);
+void grim_launch_count_reset(void);
+
+const char* grim_status_string(grim_status_t s);
+const char* grim_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRIM_H_ */

@@ -1,0 +1,177 @@
+// C-ABI entry points for the multiply, the convolution and small helpers: argument checks and
+// marshalling only; all arithmetic runs in the kernels.
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+#include "grim_internal.h"
+
+using namespace grim;
+
+namespace {
+
+grim_status_t check_mats(const grim_bcr* h, const grim_mat_t* X, const grim_mat_t* Y) {
+  if (!h || !X || !Y || !X->ptr || !Y->ptr) return GRIM_ERR_INVALID_ARG;
+  if (h->device < 0) return GRIM_ERR_INVALID_ARG;
+  if (X->rows != h->K || Y->rows != h->M || X->cols != Y->cols || X->cols <= 0) return GRIM_ERR_SHAPE;
+  if (X->ld < X->cols || Y->ld < Y->cols) return GRIM_ERR_SHAPE;
+  if ((int)X->dtype != h->dtype) return GRIM_ERR_DTYPE;
+  if (Y->dtype != GRIM_F32 && !(Y->dtype == GRIM_BF16 && h->dtype == GRIM_BF16)) return GRIM_ERR_DTYPE;
+  return GRIM_OK;
+}
+
+SpmmArgs mat_args(const grim_mat_t* X, const grim_mat_t* Y) {
+  SpmmArgs a;
+  a.X = X->ptr; a.Y = Y->ptr; a.ncols = X->cols;
+  a.x_sk = X->ld; a.x_sq = 1; a.y_sr = Y->ld; a.y_sq = 1;
+  a.x_dtype = X->dtype; a.y_dtype = Y->dtype;
+  return a;
+}
+
+grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune, cudaStream_t s) {
+  grim_status_t st = check_mats(h, X, Y);
+  if (st != GRIM_OK) return st;
+  const int path = tune ? tune->path : 0;
+  if (path < 0 || path > 2) return GRIM_ERR_INVALID_ARG;
+  if (X->cols == 1 && h->gemv_ok && path != 2 && !(tune && tune->tile_n))
+    return launch_gemv(h, X->ptr, X->dtype, Y->dtype == GRIM_F32 ? (float*)Y->ptr : nullptr,
+                       Y->dtype == GRIM_BF16 ? Y->ptr : nullptr, s);
+  SpmmArgs a = mat_args(X, Y);
+  a.tile_n = tune ? tune->tile_n : 0;
+  if (path == 2) {
+    if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
+    return launch_spmm_tc(h, a, s);
+  }
+  if (path == 0 && tc_path_supported(h, a) && a.ncols >= 256) return launch_spmm_tc(h, a, s);
+  return launch_spmm(h, a, s);
+}
+
+template <typename T>
+__global__ void maxpool2x2_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t planes, int H, int W) {
+  const int OH = H / 2, OW = W / 2;
+  const int64_t total = planes * OH * OW;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int ow = (int)(i % OW);
+    const int64_t t = i / OW;
+    const int oh = (int)(t % OH);
+    const int64_t pl = t / OH;
+    const T* p = in + (pl * H + 2 * oh) * W + 2 * ow;
+    const float a = (float)p[0], b = (float)p[1], c = (float)p[W], d = (float)p[W + 1];
+    out[i] = (T)fmaxf(fmaxf(a, b), fmaxf(c, d));
+  }
+}
+
+}  // namespace
+
+extern "C" grim_status_t grim_bcr_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, grim_stream_t stream) {
+  return run_spmm(h, X, Y, nullptr, (cudaStream_t)stream);
+}
+
+extern "C" grim_status_t grim_bcr_spmm_ex(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune,
+                                          grim_stream_t stream) {
+  return run_spmm(h, X, Y, tune, (cudaStream_t)stream);
+}
+
+extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, int reps, grim_tune_t* best,
+                                       float* best_ms, grim_stream_t stream) {
+  if (!best) return GRIM_ERR_INVALID_ARG;
+  grim_status_t st = check_mats(h, X, Y);
+  if (st != GRIM_OK) return st;
+  if (reps <= 0) reps = 5;
+  cudaStream_t s = (cudaStream_t)stream;
+  cudaEvent_t e0, e1;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return GRIM_ERR_CUDA;
+  float best_t = -1.f;
+  grim_tune_t cand_best{};
+  const int tiles[4] = {16, 32, 64, 128};
+  for (int path = 1; path <= 2; ++path) {
+    for (int ti = 0; ti < 4; ++ti) {
+      grim_tune_t c{};
+      c.path = path;
+      c.tile_n = tiles[ti];
+      if (path == 2) {
+        if (ti != 0) continue;
+        c.tile_n = 0;
+        SpmmArgs a = mat_args(X, Y);
+        if (!tc_path_supported(h, a)) continue;
+      } else if (c.tile_n > 16 && c.tile_n / 2 >= X->cols) {
+        continue;  // a wider tile than the matrix needs only adds idle lanes
+      }
+      st = run_spmm(h, X, Y, &c, s);  // warm-up
+      if (st != GRIM_OK) break;
+      cudaEventRecord(e0, s);
+      for (int r = 0; r < reps && st == GRIM_OK; ++r) st = run_spmm(h, X, Y, &c, s);
+      cudaEventRecord(e1, s);
+      if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
+      float ms = 0.f;
+      cudaEventElapsedTime(&ms, e0, e1);
+      ms /= reps;
+      if (best_t < 0.f || ms < best_t) { best_t = ms; cand_best = c; }
+    }
+    if (st != GRIM_OK) break;
+  }
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (st != GRIM_OK) return st;
+  *best = cand_best;
+  if (best_ms) *best_ms = best_t;
+  return GRIM_OK;
+}
+
+extern "C" grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d, const void* in, void* out,
+                                         grim_stream_t stream) {
+  if (!h || !d || !in || !out) return GRIM_ERR_INVALID_ARG;
+  if (h->device < 0) return GRIM_ERR_INVALID_ARG;
+  if (d->N <= 0 || d->C <= 0 || d->H <= 0 || d->W <= 0 || d->KH <= 0 || d->KW <= 0 || d->stride <= 0 || d->pad < 0)
+    return GRIM_ERR_INVALID_ARG;
+  if (d->flags & ~GRIM_CONV_RELU) return GRIM_ERR_INVALID_ARG;
+  if (d->C * (int64_t)d->KH * d->KW != h->K) return GRIM_ERR_SHAPE;
+  const int64_t OH = (d->H + 2 * d->pad - d->KH) / d->stride + 1;
+  const int64_t OW = (d->W + 2 * d->pad - d->KW) / d->stride + 1;
+  if (d->H + 2 * d->pad < d->KH || d->W + 2 * d->pad < d->KW || OH <= 0 || OW <= 0) return GRIM_ERR_SHAPE;
+  if ((int)d->in_dtype != h->dtype) return GRIM_ERR_DTYPE;
+  if (d->out_dtype != GRIM_F32 && !(d->out_dtype == GRIM_BF16 && h->dtype == GRIM_BF16)) return GRIM_ERR_DTYPE;
+  if (d->H > (1 << 20) || d->W > (1 << 20) || d->C > (1 << 24)) return GRIM_ERR_UNSUPPORTED;
+  SpmmArgs a;
+  a.X = in; a.Y = out; a.ncols = d->N * OH * OW;
+  a.x_dtype = d->in_dtype; a.y_dtype = d->out_dtype;
+  a.bias = d->bias_dev; a.relu = (d->flags & GRIM_CONV_RELU) ? 1 : 0;
+  a.conv = 1; a.C = (int)d->C; a.H = (int)d->H; a.W = (int)d->W; a.KH = d->KH; a.KW = d->KW;
+  a.stride = d->stride; a.pad = d->pad; a.OH = (int)OH; a.OW = (int)OW;
+  return launch_spmm(h, a, (cudaStream_t)stream);
+}
+
+extern "C" grim_status_t grim_maxpool2x2(const void* in, void* out, int64_t N, int64_t C, int64_t H, int64_t W,
+                                         grim_dtype_t dtype, grim_stream_t stream) {
+  if (!in || !out || N <= 0 || C <= 0 || H <= 0 || W <= 0) return GRIM_ERR_INVALID_ARG;
+  if ((H & 1) || (W & 1)) return GRIM_ERR_SHAPE;
+  if (dtype != GRIM_F32 && dtype != GRIM_BF16) return GRIM_ERR_DTYPE;
+  const int64_t total = N * C * (H / 2) * (W / 2);
+  const int threads = 256;
+  const int blocks = (int)std::min<int64_t>((total + threads - 1) / threads, 148 * 16);
+  cudaStream_t s = (cudaStream_t)stream;
+  if (dtype == GRIM_F32)
+    maxpool2x2_kernel<float><<<blocks, threads, 0, s>>>((const float*)in, (float*)out, N * C, (int)H, (int)W);
+  else
+    maxpool2x2_kernel<__nv_bfloat16><<<blocks, threads, 0, s>>>((const __nv_bfloat16*)in, (__nv_bfloat16*)out, N * C,
+                                                                (int)H, (int)W);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+}
+
+extern "C" const char* grim_status_string(grim_status_t s) {
+  switch (s) {
+    case GRIM_OK: return "ok";
+    case GRIM_ERR_INVALID_ARG: return "invalid argument";
+    case GRIM_ERR_SHAPE: return "shape mismatch";
+    case GRIM_ERR_DTYPE: return "dtype mismatch";
+    case GRIM_ERR_NOT_BCR: return "mask is not block-wise column-row structured";
+    case GRIM_ERR_ALLOC: return "allocation failed";
+    case GRIM_ERR_CUDA: return "CUDA error";
+    case GRIM_ERR_UNSUPPORTED: return "unsupported";
+    case GRIM_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+extern "C" const char* grim_version(void) { return "grim-b200 0.1 (sm_100a)"; }

@@ -1,0 +1,116 @@
+// Internal definitions shared by the host packer and the CUDA translation units of libgrim.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <vector>
+
+#include "grim.h"
+
+namespace grim {
+
+// ---------------------------------------------------------------------------------------------
+// Device layout for the N > 1 kernels ("stage" layout).
+//
+// Row bands (block rows) are taken in schedule order and cut into groups of G bands; one thread
+// block owns one group.  For group g and block column j the G block descriptors and the kept
+// values of those blocks are stored back to back ("blob"), so that a thread block streams one
+// contiguous piece of memory per block column (the compact, reordered storage idea of
+// Sections 4.2 - 4.3 laid out for a CTA instead of a CPU thread).
+// ---------------------------------------------------------------------------------------------
+struct __align__(16) BlockDesc {
+  unsigned long long colmask;  // bit c set: block-local column c kept (bw <= 64)
+  uint32_t val_off;            // first value of this block, in elements from the blob's value area
+  uint16_t rowmask;            // bit r set: block-local row r kept (bh <= 16)
+  uint16_t kc;                 // popcount(colmask)
+};
+
+struct __align__(16) StageEntry {
+  uint32_t blob_off16;               // blob start, in 16-byte units from the blob base
+  uint32_t blob_bytes;               // multiple of 16; 0 when no block of the group keeps anything here
+  unsigned long long union_colmask;  // columns kept by at least one of the G blocks
+};
+
+// ---------------------------------------------------------------------------------------------
+// Device layout for the N = 1 kernel ("chunk" layout).
+//
+// Per band the kept columns of all its blocks are concatenated after sorting the blocks by
+// kept-row count, and cut into chunks of at most 32 columns that all have the same kept-row count kr.
+// Lane l of a warp owns column l of a chunk.  A column word is (global column | rowmask << 16).
+// The chunk's values are stored step-major: value s of lane l is at val_off + s * ncols + l.
+// ---------------------------------------------------------------------------------------------
+struct ChunkDesc {
+  uint32_t val_off;
+  uint32_t cw_off;
+  uint32_t ncols_kr;  // ncols | kr << 16
+};
+
+struct HostBlock {
+  uint64_t colmask = 0;
+  uint32_t rowmask = 0;
+  uint16_t kr = 0, kc = 0;
+  uint64_t val_off = 0;  // into grim_bcr::vals (canonical order)
+};
+
+}  // namespace grim
+
+struct grim_bcr {
+  int64_t M = 0, K = 0;
+  int bh = 0, bw = 0;
+  int64_t nbr = 0, nbc = 0;
+  int dtype = 0;
+  uint32_t flags = 0;
+  int64_t nnz = 0, nonempty = 0, k_used = 0;
+  // host-side canonical data
+  std::vector<grim::HostBlock> blocks;  // nbr * nbc, row-major
+  std::vector<float> vals;              // kept values, canonical order (bf16 handles: already rounded)
+  std::vector<int32_t> row_perm;        // canonical row permutation
+  std::vector<uint32_t> band_order;     // schedule position -> band
+  // stage layout
+  int G = 0;  // bands per group
+  int64_t ngroups = 0;
+  uint32_t max_blob_bytes = 0;
+  int64_t index_bytes_spmm = 0, index_bytes_gemv = 0;
+  bool gemv_ok = false;
+  int64_t nchunks = 0;
+  std::vector<uint32_t> h_gemv_band_ptr;   // host copies of the chunk tables (sizing of on-chip weight residency)
+  std::vector<grim::ChunkDesc> h_chunks;
+  int64_t n_colwords = 0;
+  // device
+  int device = -1;
+  grim::StageEntry* d_stage = nullptr;
+  uint8_t* d_blob = nullptr;
+  uint32_t* d_band_order = nullptr;
+  uint32_t* d_gemv_band_ptr = nullptr;
+  grim::ChunkDesc* d_chunks = nullptr;
+  uint32_t* d_colwords = nullptr;
+  void* d_gemv_vals = nullptr;
+  // dense bf16 copy for the tensor-core path is decompressed on the fly; nothing stored here
+};
+
+namespace grim {
+
+// epilogue / addressing description handed to the N > 1 kernel
+struct SpmmArgs {
+  const void* X = nullptr;  // activations
+  void* Y = nullptr;
+  int64_t ncols = 0;        // GEMM N
+  int64_t x_sk = 0, x_sq = 1;  // X(k, q) at k * x_sk + q * x_sq (elements)
+  int64_t y_sr = 0, y_sq = 1;  // Y(r, q) at r * y_sr + q * y_sq
+  int x_dtype = 0, y_dtype = 0;
+  const float* bias = nullptr;  // per output row, or null
+  int relu = 0;
+  // implicit im2col (conv != 0): q = (img, oh, ow); k = (c, kh, kw)
+  int conv = 0;
+  int C = 0, H = 0, W = 0, KH = 0, KW = 0, stride = 1, pad = 0, OH = 0, OW = 0;
+  int tile_n = 0;  // 0 = default
+};
+
+grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
+grim_status_t launch_gemv(const grim_bcr* h, const void* x, int x_dtype, float* y_f32, void* y_bf16, cudaStream_t s);
+grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
+bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a);
+void count_launch(int n = 1);
+
+}  // namespace grim

@@ -1,0 +1,342 @@
+"""GPU parity: every CUDA entry point against the fp64 CPU oracle, element by element, through the C ABI.
+
+Tolerances (fixed by the benchmark spec): fp32 results  ||Y - Y*||_F / ||Y*||_F <= 1e-5;
+bf16 inputs with fp32 accumulation  max |err| <= 2e-2 * ||W row||_2 * ||X col||_2 (plus |bias| where
+a bias is added); packing is bit-exact (tests/test_packer_host.py).  Rows kept by no block must be
+exactly +0.
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import bcr_oracle as orc
+from workloads import generators as gen
+
+pytestmark = pytest.mark.gpu
+
+F32_TOL = 1e-5
+BF16_TOL = 2e-2
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2108_11033_b200.build import build_library
+    build_library()
+    from paper_2108_11033_b200 import binding
+    return binding
+
+
+def rel_fro(got, want):
+    want = np.asarray(want, dtype=np.float64)
+    return float(np.linalg.norm(np.asarray(got, dtype=np.float64) - want) / max(np.linalg.norm(want), 1e-300))
+
+
+def to_dev(a, bf16=False):
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
+    return t.to(torch.bfloat16) if bf16 else t
+
+
+def check_spmm(B, W, mask, X, bh, bw, *, bf16=False, flags=0, tile_n=0, y_bf16=False, path=0):
+    M, K = W.shape
+    X = gen.bf16_representable(X) if bf16 else np.asarray(X, np.float32)
+    N = X.shape[1]
+    dt = B.GRIM_BF16 if bf16 else B.GRIM_F32
+    h = B.grim_bcr_pack(W, mask, bh, bw, dt, flags)
+    try:
+        Xd = to_dev(X, bf16)
+        Yd = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16 if y_bf16 else torch.float32)
+        if tile_n or path:
+            B.grim_bcr_spmm_ex(h, Xd, Yd, tile_n=tile_n, path=path)
+        else:
+            B.grim_bcr_spmm(h, Xd, Yd)
+        torch.cuda.synchronize()
+        got = Yd.float().cpu().numpy().astype(np.float64)
+        want = orc.spmm(W, mask, X, dt)
+        dead = np.flatnonzero(mask.sum(axis=1) == 0)
+        assert np.all(got[dead] == 0.0) and not np.any(np.signbit(got[dead])), "pruned rows must be exactly +0"
+        if bf16:
+            Wm = orc.masked_weight(W, mask, dt)
+            bound = BF16_TOL * np.linalg.norm(Wm, axis=1)[:, None] * np.linalg.norm(X.astype(np.float64), axis=0)[None, :]
+            err = np.abs(got - want)
+            assert np.all(err <= bound + 1e-30), f"max excess {np.max(err - bound)}"
+            if not y_bf16:
+                assert rel_fro(got, want) < 1e-4  # fp32 accumulation of exact bf16 products
+        else:
+            assert rel_fro(got, want) <= F32_TOL, rel_fro(got, want)
+    finally:
+        B.grim_bcr_destroy(h)
+
+
+# ---------------------------------------------------------------------------------------- SpMM / GEMV
+
+
+def test_config1_spmm_fp32(B):
+    c = gen.config1_spmm()
+    check_spmm(B, c["W"], c["mask"], c["X"], c["bh"], c["bw"])
+
+
+SHAPES = [
+    # M, K, bh, bw, generator kwargs
+    (256, 256, 16, 16, dict(dist="fixed", kr_fixed=8, kc_fixed=8)),
+    (200, 333, 8, 32, dict(compression=6, dist="uniform")),
+    (96, 153, 8, 32, dict(compression=10, dist="uniform")),
+    (130, 260, 4, 16, dict(compression=8, dist="zipf")),
+    (150, 500, 16, 64, dict(compression=4, dist="zipf", empty_frac=0.25)),
+    (64, 27, 8, 32, dict(compression=3, dist="uniform")),
+    (33, 40, 3, 5, dict(compression=2, dist="uniform")),
+    (24, 48, 1, 1, dict(compression=3, dist="uniform")),
+    (16, 64, 16, 64, dict(compression=4, dist="uniform")),
+]
+
+
+@pytest.mark.parametrize("N", [1, 3, 16, 37, 64, 130, 260])
+@pytest.mark.parametrize("shape", SHAPES)
+def test_spmm_fp32_small(B, shape, N):
+    M, K, bh, bw, kw = shape
+    W = gen.dense_weight(M, K, seed=60)
+    mask = gen.bcr_mask(M, K, bh, bw, seed=61, **kw)
+    X = gen.normal_f32((K, N), 1.0, 62, 0)
+    check_spmm(B, W, mask, X, bh, bw)
+
+
+@pytest.mark.parametrize("N", [1, 5, 64, 200])
+@pytest.mark.parametrize("shape", SHAPES[1:6])
+def test_spmm_bf16_small(B, shape, N):
+    M, K, bh, bw, kw = shape
+    W = gen.dense_weight(M, K, seed=63)
+    mask = gen.bcr_mask(M, K, bh, bw, seed=64, **kw)
+    X = gen.normal_f32((K, N), 1.0, 65, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, y_bf16=True)
+
+
+@pytest.mark.parametrize("tile_n", [16, 32, 64, 128])
+@pytest.mark.parametrize("reorder", [0, 1])
+def test_spmm_tiles_and_reorder(B, tile_n, reorder):
+    M, K, bh, bw = 512, 768, 8, 32
+    W = gen.dense_weight(M, K, seed=66)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=8, dist="zipf", seed=67, empty_frac=0.1)
+    mask[40:56] = 0  # two fully pruned bands
+    X = gen.normal_f32((K, 150), 1.0, 68, 0)
+    check_spmm(B, W, mask, X, bh, bw, flags=reorder, tile_n=tile_n)
+
+
+def test_spmm_strided_operands_and_errors(B):
+    M, K, bh, bw, N = 64, 96, 8, 32, 20
+    W = gen.dense_weight(M, K, seed=69)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=4, seed=70)
+    h = B.grim_bcr_pack(W, mask, bh, bw, B.GRIM_F32, 0)
+    Xfull = torch.randn(K, N + 7, device="cuda")
+    Yfull = torch.zeros(M, N + 3, device="cuda")
+    X, Y = Xfull[:, 2:2 + N], Yfull[:, 1:1 + N]  # ld > cols, unaligned start
+    B.grim_bcr_spmm(h, X, Y)
+    torch.cuda.synchronize()
+    want = orc.spmm(W, mask, X.cpu().numpy())
+    assert rel_fro(Y.cpu().numpy(), want) <= F32_TOL
+    assert float(Yfull[:, 0].abs().max()) == 0.0 and float(Yfull[:, 1 + N:].abs().max()) == 0.0
+    with pytest.raises(B.GrimError) as e:
+        B.grim_bcr_spmm(h, torch.zeros(K + 1, N, device="cuda"), torch.zeros(M, N, device="cuda"))
+    assert e.value.status == B.GRIM_ERR_SHAPE
+    with pytest.raises(B.GrimError) as e:
+        B.grim_bcr_spmm(h, torch.zeros(K, N, device="cuda", dtype=torch.bfloat16), torch.zeros(M, N, device="cuda"))
+    assert e.value.status == B.GRIM_ERR_DTYPE
+    with pytest.raises(B.GrimError) as e:
+        B.grim_bcr_spmm(h, torch.zeros(K, N, device="cuda"), torch.zeros(M, N, device="cuda", dtype=torch.bfloat16))
+    assert e.value.status == B.GRIM_ERR_DTYPE
+    B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("case", [(4096, 1, 8.0, 8, 32, "uniform", False), (4096, 16, 16.0, 4, 16, "zipf", False),
+                                  (2048, 128, 4.0, 16, 64, "zipf", True), (4096, 1, 4.0, 16, 64, "zipf", True),
+                                  (1024, 1024, 8.0, 8, 32, "uniform", False)])
+def test_sweep_points(B, case):
+    M, N, c, bh, bw, dist, bf16 = case
+    s = gen.sweep_case(M, N, c, bh, bw, dist, bf16=bf16)
+    check_spmm(B, s["W"], s["mask"], s["X"], bh, bw, bf16=bf16, flags=1)
+
+
+def test_tune_returns_a_valid_choice(B):
+    s = gen.sweep_case(1024, 96, 8.0, 8, 32, "uniform")
+    h = B.grim_bcr_pack(s["W"], s["mask"], 8, 32, B.GRIM_F32, 0)
+    X = to_dev(s["X"])
+    Y = torch.empty(1024, 96, device="cuda")
+    best = B.grim_bcr_tune(h, X, Y, reps=3)
+    assert best["tile_n"] in (16, 32, 64, 128) and best["path"] in (1, 2) and best["ms"] > 0
+    B.grim_bcr_spmm_ex(h, X, Y, tile_n=best["tile_n"], path=best["path"])
+    torch.cuda.synchronize()
+    assert rel_fro(Y.cpu().numpy(), orc.spmm(s["W"], s["mask"], s["X"])) <= F32_TOL
+    B.grim_bcr_destroy(h)
+
+
+# ---------------------------------------------------------------------------------------- convolution
+
+
+def conv_col_norms(x, ksize, stride, pad):
+    """||im2col column||_2 per output pixel: sqrt of the box-sum of x^2 over the receptive field."""
+    xx = torch.from_numpy(np.asarray(x, np.float64) ** 2)
+    ones = torch.ones(1, xx.shape[1], ksize, ksize, dtype=torch.float64)
+    return torch.sqrt(torch.nn.functional.conv2d(xx, ones, stride=stride, padding=pad)).numpy()  # N,1,OH,OW
+
+
+def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=False):
+    W, mask, bias = L["W"], L["mask"], L["bias"]
+    dt = B.GRIM_BF16 if bf16 else B.GRIM_F32
+    x = gen.bf16_representable(batch_x) if bf16 else batch_x
+    h = B.grim_bcr_pack(W, mask, L["bh"], L["bw"], dt, 0)
+    try:
+        xd = to_dev(x, bf16)
+        Nb, C, H, Wd = x.shape
+        OH = (H + 2 * pad - ksize) // stride + 1
+        OW = (Wd + 2 * pad - ksize) // stride + 1
+        out = torch.full((Nb, W.shape[0], OH, OW), float("nan"), device="cuda",
+                         dtype=torch.bfloat16 if out_bf16 else torch.float32)
+        B.grim_bcr_conv2d(h, xd, out, ksize, stride, pad, bias=to_dev(bias), relu=relu)
+        torch.cuda.synchronize()
+        got = out.float().cpu().numpy().astype(np.float64)
+        want = orc.conv2d(W, mask, x, bias, ksize=ksize, stride=stride, pad=pad, relu=relu, dtype=dt)
+        if bf16:
+            Wm = orc.masked_weight(W, mask, dt)
+            bound = BF16_TOL * (np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x, ksize, stride, pad)
+                                + np.abs(bias.astype(np.float64))[None, :, None, None])
+            assert np.all(np.abs(got - want) <= bound + 1e-30)
+            if not out_bf16:
+                assert rel_fro(got, want) < 1e-4
+        else:
+            assert rel_fro(got, want) <= F32_TOL, rel_fro(got, want)
+    finally:
+        B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("geom", [(3, 1, 1), (3, 2, 1), (1, 1, 0), (5, 1, 2), (3, 1, 0)])
+@pytest.mark.parametrize("bf16", [False, True])
+def test_conv_small(B, geom, bf16):
+    ks, stride, pad = geom
+    L = gen.conv_layer(2, 12, 40, 13, ksize=ks, bh=8, bw=32, compression=4, seed=71)
+    x = np.maximum(gen.normal_f32((3, 12, 13, 11), 1.0, 72, 0), 0)
+    check_conv(B, L, x, ksize=ks, stride=stride, pad=pad, bf16=bf16)
+    check_conv(B, L, x, ksize=ks, stride=stride, pad=pad, bf16=bf16, relu=False, out_bf16=bf16)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+def test_config3_conv_batch1(B, bf16):
+    L = gen.conv_layer(1, 512, 512, 28, bf16=bf16)
+    check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=bf16)
+
+
+def test_config3_conv_batch32_sampled(B):
+    """Full-size launch (batch 32, the shape the benchmark times); the oracle checks 4 of the 32 images."""
+    L = gen.conv_layer(32, 512, 512, 28)
+    h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, B.GRIM_F32, 0)
+    xd = to_dev(L["x"])
+    out = torch.empty(32, 512, 28, 28, device="cuda")
+    B.grim_bcr_conv2d(h, xd, out, 3, 1, 1, bias=to_dev(L["bias"]), relu=True)
+    torch.cuda.synchronize()
+    pick = [0, 7, 19, 31]
+    want = orc.conv2d(L["W"], L["mask"], L["x"][pick], L["bias"], ksize=3, stride=1, pad=1, relu=True)
+    assert rel_fro(out[pick].cpu().numpy(), want) <= F32_TOL
+    B.grim_bcr_destroy(h)
+
+
+def test_maxpool(B):
+    x = torch.randn(2, 5, 8, 12, device="cuda")
+    out = torch.empty(2, 5, 4, 6, device="cuda")
+    B.grim_maxpool2x2(x, out)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().astype(np.float64), orc.maxpool2x2(x.cpu().numpy().astype(np.float64)))
+    xb = x.to(torch.bfloat16)
+    ob = torch.empty(2, 5, 4, 6, device="cuda", dtype=torch.bfloat16)
+    B.grim_maxpool2x2(xb, ob)
+    torch.cuda.synchronize()
+    assert np.array_equal(ob.float().cpu().numpy().astype(np.float64),
+                          orc.maxpool2x2(xb.float().cpu().numpy().astype(np.float64)))
+
+
+def test_vgg_stack_small_image_per_layer(B):
+    """Config-4 layer shapes at a 32x32 image: each layer is checked with the oracle fed the GPU's own
+    previous-layer output (bf16 in, fp32 accumulate, bf16 out)."""
+    net = gen.vgg16_stack(2, image=32)
+    cur = to_dev(net["x"], True)
+    for L in net["layers"]:
+        h = B.grim_bcr_pack(L["W"], L["mask"], net["bh"], net["bw"], B.GRIM_BF16, 0)
+        Nb, C, H, Wd = cur.shape
+        out = torch.empty(Nb, L["cout"], H, Wd, device="cuda", dtype=torch.bfloat16)
+        B.grim_bcr_conv2d(h, cur, out, 3, 1, 1, bias=to_dev(L["bias"]), relu=True)
+        torch.cuda.synchronize()
+        x_np = cur.float().cpu().numpy()
+        want = orc.conv2d(L["W"], L["mask"], x_np, L["bias"], ksize=3, stride=1, pad=1, relu=True, dtype=orc.DTYPE_BF16)
+        Wm = orc.masked_weight(L["W"], L["mask"], orc.DTYPE_BF16)
+        bound = BF16_TOL * (np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x_np, 3, 1, 1)
+                            + np.abs(L["bias"].astype(np.float64))[None, :, None, None])
+        assert np.all(np.abs(out.float().cpu().numpy() - want) <= bound + 1e-30)
+        B.grim_bcr_destroy(h)
+        if L["pool"]:
+            pooled = torch.empty(Nb, L["cout"], H // 2, Wd // 2, device="cuda", dtype=torch.bfloat16)
+            B.grim_maxpool2x2(out, pooled)
+            cur = pooled
+        else:
+            cur = out
+
+
+# ---------------------------------------------------------------------------------------- GRU
+
+
+def build_gru(B, m, max_T):
+    hi, hh = [], []
+    for lay in m["layers"]:
+        hi.append(B.grim_bcr_pack(lay["W_ih"], lay["mask_ih"], m["bh"], m["bw"], B.GRIM_F32, 0))
+        hh.append(B.grim_bcr_pack(lay["W_hh"], lay["mask_hh"], m["bh"], m["bw"], B.GRIM_F32, 0))
+    g = B.grim_gru_create(hi, hh, [l["b_ih"] for l in m["layers"]], [l["b_hh"] for l in m["layers"]], max_T)
+    return g, hi + hh
+
+
+def check_gru(B, m, h0=None):
+    T, H, L = m["T"], m["hidden"], len(m["layers"])
+    g, handles = build_gru(B, m, T)
+    try:
+        x = to_dev(m["x"])
+        y = torch.full((T, H), float("nan"), device="cuda")
+        hT = torch.full((L, H), float("nan"), device="cuda")
+        for _ in range(2):  # the handle is reusable
+            B.grim_gru_seq(g, x, y, h0=to_dev(h0) if h0 is not None else None, hT=hT)
+            assert B.grim_gru_status(g) == B.GRIM_OK
+        want_y, want_h = orc.gru_seq(m["layers"], m["x"], h0=h0)
+        assert rel_fro(y.cpu().numpy(), want_y) <= F32_TOL, rel_fro(y.cpu().numpy(), want_y)
+        assert rel_fro(hT.cpu().numpy(), want_h) <= F32_TOL
+    finally:
+        B.grim_gru_destroy(g)
+        for h in handles:
+            B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("cfg", [(20, 64, 1, 7, 8, 32), (37, 128, 2, 13, 8, 32), (16, 96, 3, 5, 4, 16),
+                                 (50, 256, 2, 9, 16, 64)])
+def test_gru_small(B, cfg):
+    in_f, H, L, T, bh, bw = cfg
+    m = gen.gru_model(in_f, H, L, T, bh=bh, bw=bw, compression=4, seed=80)
+    check_gru(B, m)
+    h0 = gen.normal_f32((L, H), 0.5, 81, 0)
+    check_gru(B, m, h0=h0)
+
+
+def test_config2_gru_full(B):
+    check_gru(B, gen.gru_model())
+
+
+def test_gru_bounded_wait_reports_timeout(B):
+    """One thread block stays away from the step barrier: every wait runs out after a small bound, the
+    kernel returns by itself and the status word says so; afterwards the handle works normally."""
+    m = gen.gru_model(20, 256, 1, 6, bh=8, bw=32, compression=4, seed=82)
+    g, handles = build_gru(B, m, 6)
+    x = to_dev(m["x"])
+    y = torch.zeros(6, 256, device="cuda")
+    B.grim_gru_debug_barrier(g, 1, 20000)
+    B.grim_gru_seq(g, x, y)
+    assert B.grim_gru_status(g) == B.GRIM_ERR_TIMEOUT
+    B.grim_gru_debug_barrier(g, -1, 0)
+    B.grim_gru_seq(g, x, y)
+    assert B.grim_gru_status(g) == B.GRIM_OK
+    want_y, _ = orc.gru_seq(m["layers"], m["x"])
+    assert rel_fro(y.cpu().numpy(), want_y) <= F32_TOL
+    B.grim_gru_destroy(g)
+    for h in handles:
+        B.grim_bcr_destroy(h)
