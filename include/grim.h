@@ -207,6 +207,32 @@ grim_status_t grim_gru_seq(grim_gru_t g, const float* x_dev, int64_t T, const fl
 grim_status_t grim_gru_status(grim_gru_t g);
 grim_status_t grim_gru_destroy(grim_gru_t g);
 
+/* grim_gru_seq without any device allocation behind it.  (The paper has no counterpart: this entry
+ * point exists for the way the library is deployed, not for the method.)
+ *
+ * Who needs it: code that runs where the CUDA allocator must not be called - a serving loop that has
+ * handed all device memory to its own pool, a real-time audio / control thread that may not take the
+ * allocator's locks or tolerate its latency, a process running under a memory budget that was fixed
+ * at start-up.  Such a caller builds the GRU handle once during start-up (that step allocates) and
+ * afterwards calls this function, which allocates nothing and calls no allocating library routine.
+ *
+ * Same arguments, results and error codes as grim_gru_seq.  The difference is where the per-call
+ * scratch lives (the hoisted pre-activations, T x 3H floats, and for multi-layer models two T x H
+ * inter-layer buffers): in one fixed 8 MiB array that is part of the library image and therefore
+ * occupies 8 MiB on every GPU that loads the library, until the process exits.
+ *   - Limit: round256(T*3H*4) + 2*round256(T*H*4) (second term only for layers > 1) must fit in
+ *     8 MiB - e.g. H = 1024, two layers: T <= 409.  Larger requests return GRIM_ERR_UNSUPPORTED
+ *     before anything is launched; use grim_gru_seq for those.
+ *   - The first call on a device looks up the array's device address (once per device, with that
+ *     device current).  Make that first call during start-up, before any CUDA stream capture.
+ *   - All calls in the process share the array and it keeps whatever the previous call left there.
+ *     Nothing in it has to start at zero: every word the kernels read from it is written earlier in
+ *     the same call.  Two calls that overlap on the GPU (different streams or handles) race on it;
+ *     serialise them.
+ *   - The current device must be the handle's device (GRIM_ERR_INVALID_ARG otherwise). */
+grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x_dev, int64_t T, const float* h0_dev, float* y_dev,
+                                  float* hT_dev, grim_stream_t stream);
+
 /* Test hook for the bounded waits of the recurrent kernel (no counterpart in the paper): thread
  * block `skip_cta` stays away from the per-step barrier (-1 = normal operation) and a waiting
  * block gives up after `spin_limit` polls (0 = default).  With a block missing, every wait runs

@@ -32,7 +32,7 @@ EXPORTED = [
     "grim_bcr_pack", "grim_bcr_destroy", "grim_bcr_info", "grim_bcr_export", "grim_bcr_unpack_dense",
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
-    "grim_gru_profile", "grim_gru_profile_read",
+    "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static",
     "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version",
 ]
 
@@ -81,6 +81,7 @@ lib.grim_maxpool2x2.argtypes = [_vp, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_i
 lib.grim_gru_create.argtypes = [C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.POINTER(_vp), C.c_int64,
                                 C.POINTER(_vp)]
 lib.grim_gru_seq.argtypes = [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp]
+lib.grim_gru_seq_static.argtypes = [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp]
 lib.grim_gru_status.argtypes = [_vp]
 lib.grim_gru_destroy.argtypes = [_vp]
 lib.grim_gru_debug_barrier.argtypes = [_vp, C.c_int, C.c_uint]
@@ -226,6 +227,15 @@ def grim_gru_seq(g: int, x, y, h0=None, hT=None, stream=None):
     assert x.is_cuda and y.is_cuda and x.is_contiguous() and y.is_contiguous()
     _check(lib.grim_gru_seq(g, x.data_ptr(), x.shape[0], h0.data_ptr() if h0 is not None else None, y.data_ptr(),
                             hT.data_ptr() if hT is not None else None, _stream_ptr(stream)), "grim_gru_seq")
+
+
+def grim_gru_seq_static(g: int, x, y, h0=None, hT=None, stream=None):
+    """grim_gru_seq for callers that may not allocate device memory: scratch comes from a fixed 8 MiB
+    array inside the library (shared by all calls; see include/grim.h for the size limit)."""
+    assert x.is_cuda and y.is_cuda and x.is_contiguous() and y.is_contiguous()
+    _check(lib.grim_gru_seq_static(g, x.data_ptr(), x.shape[0], h0.data_ptr() if h0 is not None else None,
+                                   y.data_ptr(), hT.data_ptr() if hT is not None else None, _stream_ptr(stream)),
+           "grim_gru_seq_static")
 
 
 def grim_gru_status(g: int) -> int:

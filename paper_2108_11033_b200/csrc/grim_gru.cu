@@ -437,3 +437,56 @@ extern "C" grim_status_t grim_gru_destroy(grim_gru_t g) {
   if (cur != dev && cur >= 0) cudaSetDevice(cur);
   return GRIM_OK;
 }
+
+// ---------------------------------------------------------------------------------------------
+// grim_gru_seq_static: the same sequence pass for callers that must not allocate device memory.
+//
+// The per-call scratch of the GRU pass (the hoisted pre-activations gi, T x 3H floats, and the two
+// T x H buffers that carry one layer's outputs to the next) lives in a fixed array inside the
+// library image instead of in buffers obtained from the CUDA allocator.  Host code cannot use the
+// array's name as a device address; the address is looked up once per device with
+// cudaGetSymbolAddress while that device is current, and that pointer is what the kernels receive.
+// ---------------------------------------------------------------------------------------------
+namespace {
+constexpr size_t kStaticScratchBytes = size_t(8) << 20;  // 8 MiB, resident on every GPU that loads the library
+constexpr int kMaxDevices = 64;
+}  // namespace
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+static unsigned char* g_static_scratch_addr[kMaxDevices] = {};
+
+extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64_t T, const float* h0, float* y,
+                                             float* hT, grim_stream_t stream) {
+  if (!g || !x || !y || T <= 0) return GRIM_ERR_INVALID_ARG;
+  if (T > g->max_T) return GRIM_ERR_SHAPE;
+  // carve-up of the static array: gi | seq0 | seq1, each start rounded up to 256 bytes
+  auto round256 = [](size_t b) { return (b + 255) & ~size_t(255); };
+  const size_t gi_bytes = round256((size_t)T * 3 * (size_t)g->H * 4);
+  const size_t seq_bytes = g->L > 1 ? round256((size_t)T * (size_t)g->H * 4) : 0;
+  if (gi_bytes + 2 * seq_bytes > kStaticScratchBytes) return GRIM_ERR_UNSUPPORTED;  // T * H too large for 8 MiB
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return GRIM_ERR_CUDA;
+  if (dev != g->device || dev < 0 || dev >= kMaxDevices) return GRIM_ERR_INVALID_ARG;
+  if (!g_static_scratch_addr[dev]) {
+    // one-time set-up for this device (device `dev` is current): resolve the array's device address
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_static_scratch) != cudaSuccess || !p) {
+      cudaGetLastError();
+      return GRIM_ERR_CUDA;
+    }
+    g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
+  }
+  unsigned char* base = g_static_scratch_addr[dev];
+  // Run the ordinary pass with the handle's scratch pointers pointing into the static array for the
+  // duration of the call.  Kernel arguments are copied at launch, so the handle can be put back at once.
+  float* const saved_gi = g->d_gi;
+  float* const saved_seq0 = g->d_seq[0];
+  float* const saved_seq1 = g->d_seq[1];
+  g->d_gi = reinterpret_cast<float*>(base);
+  g->d_seq[0] = reinterpret_cast<float*>(base + gi_bytes);
+  g->d_seq[1] = reinterpret_cast<float*>(base + gi_bytes + seq_bytes);
+  const grim_status_t st = grim_gru_seq(g, x, T, h0, y, hT, stream);
+  g->d_gi = saved_gi;
+  g->d_seq[0] = saved_seq0;
+  g->d_seq[1] = saved_seq1;
+  return st;
+}
