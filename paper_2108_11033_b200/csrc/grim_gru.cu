@@ -3,11 +3,17 @@
 //
 // Per layer: (1) the input-side products W_ih x_t for all T steps do not depend on the recurrence and
 // are hoisted into one sparse GEMM with N = T (bias b_ih fused); (2) one persistent kernel walks the T
-// dependent steps.  Every thread block owns a few groups of bh hidden units and the three row bands
+// dependent steps.  Every thread block owns some groups of bh hidden units and the three row bands
 // (r, z, n gates) of W_hh that produce them; it copies those bands' packed chunks into shared memory
 // once, so that W_hh is read from HBM once per sequence instead of once per step.  Per step the blocks
-// multiply their bands with h_{t-1}, apply the gate non-linearities, publish their slice of h_t and
-// meet at a grid-wide barrier whose wait is bounded.
+// multiply their bands with h_{t-1}, apply the gate non-linearities and exchange their slices of h_t.
+//
+// Two exchange schemes:
+//   gru_cluster_kernel    one thread-block cluster (up to 16 CTAs) holds all of W_hh; h_t is broadcast
+//                         with distributed-shared-memory stores and the step ends with the hardware
+//                         cluster barrier.  Used whenever the layer fits one cluster.
+//   gru_recurrent_kernel  cooperative grid of up to 128 CTAs; h_t goes through L2 and the step ends with a
+//                         grid-wide barrier in global memory whose wait is bounded (status word on expiry).
 #include <cooperative_groups.h>
 
 #include <algorithm>
@@ -16,7 +22,18 @@
 #include "grim_device.cuh"
 #include "grim_internal.h"
 
+namespace cg = cooperative_groups;
 using namespace grim;
+
+namespace {
+constexpr int kMaxLocalBands = 48;
+struct ModeCfg {
+  int tpc = 1, ks = 1, threads = 0, ctas = 0, resident = 0;
+  uint32_t max_chunks = 0, max_cw = 0, max_vals = 0;
+  size_t smem = 0;
+  bool ok = false;
+};
+}  // namespace
 
 struct grim_gru {
   int L = 0;
@@ -28,20 +45,19 @@ struct grim_gru {
   float* d_gi = nullptr;
   float* d_seq[2] = {nullptr, nullptr};
   unsigned* d_sync = nullptr;  // [0..L): barrier counters, [L]: status word
-  int tpc = 1, ks = 1, threads = 0, grid = 0, resident = 0;
-  uint32_t max_chunks = 0, max_cw = 0, max_vals = 0;
-  size_t smem = 0;
+  ModeCfg grid, cluster;       // launch shapes of the shared-memory kernels
+  ModeCfg regc;                // launch shape of the register-resident cluster kernel
+  int reg_ni = 0, reg_s = 0;   // its compiled (items per warp, slots per item) variant
   int device = -1;
   cudaStream_t last_stream = nullptr;
   int dbg_skip_cta = -1;
   unsigned spin_limit = 1u << 22;
+  bool force_grid = false;
   bool profile = false;
   std::vector<cudaEvent_t> ev;  // 3 per layer: before projection, before recurrent kernel, after it
 };
 
 namespace {
-
-constexpr int kMaxLocalBands = 24;
 
 struct GruParams {
   const uint32_t* band_ptr;
@@ -73,29 +89,32 @@ __device__ __forceinline__ void red_release_gpu_add(unsigned* p, unsigned v) {
 
 __device__ __forceinline__ float sigmoidf_(float v) { return 1.f / (1.f + expf(-v)); }
 
-template <int BH>
-__global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams p) {
-  extern __shared__ __align__(16) uint8_t smem[];
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-  const int nb = 3 * p.tpc;        // local bands: index tri * 3 + gate
-  const int nbands_gate = p.H / p.bh;
-  float* hs = reinterpret_cast<float*>(smem);
-  float* partial = hs + p.H;  // [nb][ks][BH]
-  uint32_t* s_cb = reinterpret_cast<uint32_t*>(partial + nb * p.ks * BH);  // chunk range per local band
-  uint32_t* s_ce = s_cb + kMaxLocalBands;
-  ChunkDesc* s_ch = reinterpret_cast<ChunkDesc*>(s_ce + kMaxLocalBands);
-  uint32_t* s_cw = reinterpret_cast<uint32_t*>(s_ch + p.max_chunks);
-  float* s_val = reinterpret_cast<float*>(s_cw + p.max_cw);
+// Per-CTA view of its bands' chunks: either the global arrays or copies in shared memory.
+struct BandView {
+  const ChunkDesc* ch;
+  const uint32_t* cw;
+  const float* vals;
+  const uint32_t* cb;  // chunk range per local band (local band = group * 3 + gate)
+  const uint32_t* ce;
+};
+
+// One-time set-up: locate the bands of CTA `cta` (tpc groups of bh hidden units x 3 gates) and, if they
+// fit, copy their chunk descriptors / column words / values into shared memory.  `pool` is the dynamic
+// shared memory left after the caller's own arrays.
+__device__ BandView setup_bands(const GruParams& p, int cta, uint8_t* pool) {
   __shared__ uint32_t s_src_c[kMaxLocalBands], s_src_cw[kMaxLocalBands], s_src_v[kMaxLocalBands];
   __shared__ uint32_t s_dst_cw[kMaxLocalBands], s_dst_v[kMaxLocalBands], s_n_cw[kMaxLocalBands], s_n_v[kMaxLocalBands];
-  __shared__ int s_abort;
-
-  // ---- one-time set-up: locate this block's bands and (if they fit) make them resident
+  __shared__ uint32_t s_cb[kMaxLocalBands], s_ce[kMaxLocalBands];
+  const int tid = threadIdx.x;
+  const int nb = 3 * p.tpc;
+  const int nbands_gate = p.H / p.bh;
+  ChunkDesc* s_ch = reinterpret_cast<ChunkDesc*>(pool);
+  uint32_t* s_cw = reinterpret_cast<uint32_t*>(s_ch + p.max_chunks);
+  float* s_val = reinterpret_cast<float*>(s_cw + p.max_cw);
   if (tid == 0) {
-    s_abort = 0;
     uint32_t nc = 0, ncw = 0, nv = 0;
     for (int lb = 0; lb < nb; ++lb) {
-      const int tri = blockIdx.x * p.tpc + lb / 3;
+      const int tri = cta * p.tpc + lb / 3;
       uint32_t cb = 0, ce = 0;
       if (tri < nbands_gate) {
         const uint32_t pos = p.pos_of_band[(lb % 3) * nbands_gate + tri];
@@ -118,9 +137,7 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
     }
   }
   __syncthreads();
-  const ChunkDesc* ch = p.chunks;
-  const uint32_t* cw = p.colwords;
-  const float* vals = p.vals;
+  BandView v{p.chunks, p.colwords, p.vals, s_cb, s_ce};
   if (p.resident) {
     for (int lb = 0; lb < nb; ++lb) {
       const uint32_t n = s_ce[lb] - s_cb[lb];
@@ -133,13 +150,67 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
       for (uint32_t i = tid; i < s_n_cw[lb]; i += blockDim.x) s_cw[s_dst_cw[lb] + i] = p.colwords[s_src_cw[lb] + i];
       for (uint32_t i = tid; i < s_n_v[lb]; i += blockDim.x) s_val[s_dst_v[lb] + i] = p.vals[s_src_v[lb] + i];
     }
-    ch = s_ch; cw = s_cw; vals = s_val;
+    v.ch = s_ch; v.cw = s_cw; v.vals = s_val;
   }
   __syncthreads();
+  return v;
+}
 
-  const int my_lb = warp / p.ks, my_ks = warp % p.ks;
-  const bool gemv_warp = my_lb < nb;
-  // gate threads: one per hidden unit owned by this block
+// Band x vector for work item (local band lb, k-split part ks_i): partial[(lb*ks + ks_i)*BH + row].
+template <int BH>
+__device__ __forceinline__ void band_gemv(const BandView& v, const float* hs, float* partial, int lb, int ks_i, int ks,
+                                          int lane) {
+  float acc[BH];
+#pragma unroll
+  for (int r = 0; r < BH; ++r) acc[r] = 0.f;
+  for (uint32_t c = v.cb[lb] + ks_i; c < v.ce[lb]; c += ks) {
+    const ChunkDesc cd = v.ch[c];
+    const int ncols = cd.ncols_kr & 0xFFFF;
+    if (lane < ncols) {
+      const uint32_t w = v.cw[cd.cw_off + lane];
+      const unsigned rm = w >> 16;
+      const float xv = hs[w & 0xFFFFu];
+      const float* val = v.vals + cd.val_off + lane;
+      int cnt = 0;
+#pragma unroll
+      for (int r = 0; r < BH; ++r)
+        if ((rm >> r) & 1u) { acc[r] = fmaf(val[cnt * ncols], xv, acc[r]); ++cnt; }
+    }
+  }
+  warp_reduce_rows<BH>(acc, lane);
+  partial[(lb * ks + ks_i) * BH + warp_row<BH>(lane)] = acc[0];
+}
+
+__device__ __forceinline__ float gru_gate(const float* partial, const float (&bq)[3], const float (&gi)[3], int g_tri,
+                                          int g_r, int ks, int BH, float hprev) {
+  float q[3];
+#pragma unroll
+  for (int g = 0; g < 3; ++g) {
+    float s = bq[g];
+    for (int k = 0; k < ks; ++k) s += partial[((g_tri * 3 + g) * ks + k) * BH + g_r];
+    q[g] = s;
+  }
+  const float rg = sigmoidf_(gi[0] + q[0]);
+  const float zg = sigmoidf_(gi[1] + q[1]);
+  const float ng = tanhf(gi[2] + rg * q[2]);
+  return (1.f - zg) * ng + zg * hprev;
+}
+
+// ---------------------------------------------------------------------------------------------
+// cooperative-grid version (h through L2, bounded global barrier)
+// ---------------------------------------------------------------------------------------------
+template <int BH>
+__global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams p) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int nb = 3 * p.tpc;
+  float* hs = reinterpret_cast<float*>(smem);
+  float* partial = hs + p.H;  // [nb][ks][BH]
+  __shared__ int s_abort;
+  if (tid == 0) s_abort = 0;
+  const BandView v = setup_bands(p, blockIdx.x, reinterpret_cast<uint8_t*>(partial + nb * p.ks * BH));
+
+  const int nwarps = blockDim.x >> 5;
   const bool gate_thread = tid < p.tpc * p.bh;
   const int g_tri = tid / p.bh, g_r = tid % p.bh;
   const int unit = (blockIdx.x * p.tpc + g_tri) * p.bh + g_r;
@@ -156,42 +227,10 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
     const float* hprev = t == 0 ? p.h0 : p.out + (int64_t)(t - 1) * p.H;
     for (int i = tid; i < p.H; i += blockDim.x) hs[i] = hprev ? __ldcg(hprev + i) : 0.f;
     __syncthreads();
-
-    if (gemv_warp) {
-      float acc[BH];
-#pragma unroll
-      for (int r = 0; r < BH; ++r) acc[r] = 0.f;
-      for (uint32_t c = s_cb[my_lb] + my_ks; c < s_ce[my_lb]; c += p.ks) {
-        const ChunkDesc cd = ch[c];
-        const int ncols = cd.ncols_kr & 0xFFFF;
-        if (lane < ncols) {
-          const uint32_t w = cw[cd.cw_off + lane];
-          const unsigned rm = w >> 16;
-          const float xv = hs[w & 0xFFFFu];
-          const float* v = vals + cd.val_off + lane;
-          int cnt = 0;
-#pragma unroll
-          for (int r = 0; r < BH; ++r)
-            if ((rm >> r) & 1u) { acc[r] = fmaf(v[cnt * ncols], xv, acc[r]); ++cnt; }
-        }
-      }
-      warp_reduce_rows<BH>(acc, lane);
-      partial[(my_lb * p.ks + my_ks) * BH + warp_row<BH>(lane)] = acc[0];
-    }
+    for (int item = warp; item < nb * p.ks; item += nwarps) band_gemv<BH>(v, hs, partial, item / p.ks, item % p.ks, p.ks, lane);
     __syncthreads();
-
     if (gate_live) {
-      float q[3];
-#pragma unroll
-      for (int g = 0; g < 3; ++g) {
-        float s = bq[g];
-        for (int k = 0; k < p.ks; ++k) s += partial[((g_tri * 3 + g) * p.ks + k) * BH + g_r];
-        q[g] = s;
-      }
-      const float rg = sigmoidf_(gi[0] + q[0]);
-      const float zg = sigmoidf_(gi[1] + q[1]);
-      const float ng = tanhf(gi[2] + rg * q[2]);
-      const float hn = (1.f - zg) * ng + zg * hs[unit];
+      const float hn = gru_gate(partial, bq, gi, g_tri, g_r, p.ks, BH, hs[unit]);
       p.out[(int64_t)t * p.H + unit] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
     }
@@ -215,27 +254,317 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
   }
 }
 
-size_t gru_smem_bytes(const grim_gru* g, int BH) {
-  const int nb = 3 * g->tpc;
-  size_t b = (size_t)g->H * 4 + (size_t)nb * g->ks * BH * 4 + 2 * kMaxLocalBands * 4;
-  if (g->resident) b += (size_t)g->max_chunks * sizeof(ChunkDesc) + (size_t)g->max_cw * 4 + (size_t)g->max_vals * 4;
+// ---------------------------------------------------------------------------------------------
+// cluster version (h through distributed shared memory, hardware cluster barrier - no spin waits)
+// ---------------------------------------------------------------------------------------------
+template <int BH>
+__global__ void __launch_bounds__(1024, 1) gru_cluster_kernel(const GruParams p) {
+  extern __shared__ __align__(16) uint8_t smem[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rank = (int)cluster.block_rank();
+  const int CS = (int)cluster.num_blocks();
+  const int nb = 3 * p.tpc;
+  const int U = p.tpc * p.bh;                      // hidden units owned by this CTA
+  float* hs = reinterpret_cast<float*>(smem);      // [2][H], double-buffered h
+  float* hnew = hs + 2 * p.H;                      // [U]
+  float* partial = hnew + ((U + 3) & ~3);          // [nb][ks][BH]
+  const BandView v = setup_bands(p, rank, reinterpret_cast<uint8_t*>(partial + nb * p.ks * BH));
+
+  const int nwarps = blockDim.x >> 5;
+  const bool gate_live = tid < U;
+  const int g_tri = tid / p.bh, g_r = tid % p.bh;
+  const int unit = rank * U + tid;
+  float bq[3] = {0.f, 0.f, 0.f};
+  if (gate_live)
+    for (int g = 0; g < 3; ++g) bq[g] = p.b_hh[g * p.H + unit];
+  for (int i = tid; i < p.H; i += blockDim.x) hs[i] = p.h0 ? p.h0[i] : 0.f;
+  cluster.sync();  // every CTA of the cluster is resident and has initialised its buffers
+
+  for (int t = 0; t < p.T; ++t) {
+    const float* hcur = hs + (t & 1) * p.H;
+    float* hnxt_local = hs + ((t + 1) & 1) * p.H;
+    float gi[3] = {0.f, 0.f, 0.f};
+    if (gate_live)
+      for (int g = 0; g < 3; ++g) gi[g] = __ldg(p.gi + (int64_t)t * 3 * p.H + g * p.H + unit);
+    for (int item = warp; item < nb * p.ks; item += nwarps) band_gemv<BH>(v, hcur, partial, item / p.ks, item % p.ks, p.ks, lane);
+    __syncthreads();
+    if (gate_live) {
+      const float hn = gru_gate(partial, bq, gi, g_tri, g_r, p.ks, BH, hcur[unit]);
+      hnew[tid] = hn;
+      p.out[(int64_t)t * p.H + unit] = hn;
+      if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
+    }
+    __syncthreads();
+    // broadcast this CTA's slice of h_t into the next-step buffer of every CTA of the cluster
+    if ((U & 3) == 0) {
+      const int q = U >> 2;
+      for (int i = tid; i < CS * q; i += blockDim.x) {
+        const int dst = i / q, j = i - dst * q;
+        float4* remote = cluster.map_shared_rank(reinterpret_cast<float4*>(hnxt_local + rank * U) + j, dst);
+        *remote = reinterpret_cast<const float4*>(hnew)[j];
+      }
+    } else {
+      for (int i = tid; i < CS * U; i += blockDim.x) {
+        const int dst = i / U, j = i - dst * U;
+        *cluster.map_shared_rank(hnxt_local + rank * U + j, dst) = hnew[j];
+      }
+    }
+    cluster.sync();  // release our stores, acquire everyone else's; also keeps all CTAs alive until the end
+  }
+}
+
+// ---------------------------------------------------------------------------------------------
+// cluster version with W_hh in registers.  Same exchange as gru_cluster_kernel, but every warp keeps its
+// share of the bands in registers for the whole sequence: a band is cut in two halves (work items), an
+// item's kept columns are dealt to S slots x 32 lanes, and a lane holds per slot the column index and
+// the column's BH values expanded to row positions (zeros where the row is not kept).  A time step then
+// costs one shared-memory gather of h and BH FMAs per slot - no index decoding, no predicates.
+// NI = items per warp.  Shapes that need more slots than the compiled menu use the other kernels.
+// ---------------------------------------------------------------------------------------------
+constexpr int kRegThreads = 512;
+constexpr int kRegWarps = kRegThreads / 32;
+
+template <int BH, int NI, int S>
+__global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const GruParams p) {
+  extern __shared__ __align__(16) float smem_f[];
+  cg::cluster_group cluster = cg::this_cluster();
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int rank = (int)cluster.block_rank();
+  const int CS = (int)cluster.num_blocks();
+  const int nb = 3 * p.tpc;
+  const int U = p.tpc * p.bh;
+  const int H = p.H;
+  const int nbands_gate = H / p.bh;
+  float* hs = smem_f;                         // [2][H]
+  float* hnew = hs + 2 * H;                   // [U]
+  float* partial = hnew + ((U + 3) & ~3);     // [nb][2][BH]
+
+  // ---- one-time: pull this warp's items out of the chunk layout into registers
+  float val[NI][S][BH];
+  uint32_t col[NI][S];
+#pragma unroll
+  for (int i = 0; i < NI; ++i) {
+    const int item = warp * NI + i;
+    uint32_t cb = 0, ce = 0;
+    if (item < nb * 2) {
+      const int lb = item >> 1;
+      const int tri = rank * p.tpc + lb / 3;
+      const uint32_t pos = p.pos_of_band[(lb % 3) * nbands_gate + tri];
+      cb = p.band_ptr[pos];
+      ce = p.band_ptr[pos + 1];
+    }
+    uint32_t n = 0;
+    for (uint32_t c = cb; c < ce; ++c) n += p.chunks[c].ncols_kr & 0xFFFFu;
+    const uint32_t mid = (n + 1) >> 1;
+    const uint32_t c0 = (item & 1) ? mid : 0u, c1 = (item & 1) ? n : mid;
+#pragma unroll
+    for (int s = 0; s < S; ++s) {
+      col[i][s] = 0;
+#pragma unroll
+      for (int r = 0; r < BH; ++r) val[i][s][r] = 0.f;
+      const uint32_t ci = c0 + s * 32 + lane;
+      if (ci < c1) {
+        uint32_t prefix = 0, c = cb;
+        uint32_t nk = p.chunks[c].ncols_kr;
+        while (ci >= prefix + (nk & 0xFFFFu)) {
+          prefix += nk & 0xFFFFu;
+          ++c;
+          nk = p.chunks[c].ncols_kr;
+        }
+        const uint32_t l = ci - prefix, ncols = nk & 0xFFFFu;
+        const ChunkDesc cd = p.chunks[c];
+        const uint32_t w = p.colwords[cd.cw_off + l];
+        const uint32_t rm = w >> 16;
+        col[i][s] = w & 0xFFFFu;
+#pragma unroll
+        for (int r = 0; r < BH; ++r)
+          if ((rm >> r) & 1u) val[i][s][r] = p.vals[cd.val_off + __popc(rm & ((1u << r) - 1u)) * ncols + l];
+      }
+    }
+  }
+
+  const bool gate_live = tid < U;
+  const int g_tri = tid / p.bh, g_r = tid % p.bh;
+  const int unit = rank * U + tid;
+  float bq[3] = {0.f, 0.f, 0.f};
+  float gi[3] = {0.f, 0.f, 0.f};
+  if (gate_live)
+    for (int g = 0; g < 3; ++g) {
+      bq[g] = p.b_hh[g * H + unit];
+      gi[g] = __ldg(p.gi + g * H + unit);
+    }
+  for (int i = tid; i < H; i += kRegThreads) hs[i] = p.h0 ? p.h0[i] : 0.f;
+  cluster.sync();
+
+  for (int t = 0; t < p.T; ++t) {
+    const float* hcur = hs + (t & 1) * H;
+    float* hnxt_local = hs + ((t + 1) & 1) * H;
+    // pre-activations of the next step are fetched now so that their DRAM latency hides behind this step
+    float gi_next[3] = {0.f, 0.f, 0.f};
+    if (gate_live && t + 1 < p.T)
+      for (int g = 0; g < 3; ++g) gi_next[g] = __ldg(p.gi + (int64_t)(t + 1) * 3 * H + g * H + unit);
+#pragma unroll
+    for (int i = 0; i < NI; ++i) {
+      const int item = warp * NI + i;
+      float acc[BH];
+#pragma unroll
+      for (int r = 0; r < BH; ++r) acc[r] = 0.f;
+#pragma unroll
+      for (int s = 0; s < S; ++s) {
+        const float xv = hcur[col[i][s]];
+#pragma unroll
+        for (int r = 0; r < BH; ++r) acc[r] = fmaf(val[i][s][r], xv, acc[r]);
+      }
+      warp_reduce_rows<BH>(acc, lane);
+      if (item < nb * 2) partial[item * BH + warp_row<BH>(lane)] = acc[0];
+    }
+    __syncthreads();
+    if (gate_live) {
+      const float hn = gru_gate(partial, bq, gi, g_tri, g_r, 2, BH, hcur[unit]);
+      hnew[tid] = hn;
+      p.out[(int64_t)t * H + unit] = hn;
+      if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
+    }
+    __syncthreads();
+    if ((U & 3) == 0) {
+      const int q = U >> 2;
+      for (int i = tid; i < CS * q; i += kRegThreads) {
+        const int dst = i / q, j = i - dst * q;
+        float4* remote = cluster.map_shared_rank(reinterpret_cast<float4*>(hnxt_local + rank * U) + j, dst);
+        *remote = reinterpret_cast<const float4*>(hnew)[j];
+      }
+    } else {
+      for (int i = tid; i < CS * U; i += kRegThreads) {
+        const int dst = i / U, j = i - dst * U;
+        *cluster.map_shared_rank(hnxt_local + rank * U + j, dst) = hnew[j];
+      }
+    }
+#pragma unroll
+    for (int g = 0; g < 3; ++g) gi[g] = gi_next[g];
+    cluster.sync();
+  }
+}
+
+size_t smem_bytes(const grim_gru* g, const ModeCfg& m, int BH, bool cluster) {
+  const int nb = 3 * m.tpc;
+  size_t b = (size_t)nb * m.ks * BH * 4;
+  if (cluster) b += (size_t)2 * g->H * 4 + (size_t)((m.tpc * g->bh + 3) & ~3) * 4;
+  else b += (size_t)g->H * 4;
+  if (m.resident) b += (size_t)m.max_chunks * sizeof(ChunkDesc) + (size_t)m.max_cw * 4 + (size_t)m.max_vals * 4;
   return (b + 15) & ~size_t(15);
 }
 
 template <int BH>
-cudaError_t launch_recurrent(const grim_gru* g, const GruParams& p, cudaStream_t s) {
+cudaError_t launch_grid(const grim_gru* g, const GruParams& p, cudaStream_t s) {
+  const ModeCfg& m = g->grid;
   auto kern = gru_recurrent_kernel<BH>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)g->smem);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m.smem);
   if (e != cudaSuccess) return e;
   int per_sm = 0, sms = 0;
-  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, g->threads, g->smem);
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, m.threads, m.smem);
   if (e != cudaSuccess) return e;
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, g->device);
-  if ((int64_t)per_sm * sms < g->grid) return cudaErrorCooperativeLaunchTooLarge;
+  if ((int64_t)per_sm * sms < m.ctas) return cudaErrorCooperativeLaunchTooLarge;
   void* args[] = {(void*)&p};
-  e = cudaLaunchCooperativeKernel((void*)kern, dim3(g->grid), dim3(g->threads), args, g->smem, s);
+  e = cudaLaunchCooperativeKernel((void*)kern, dim3(m.ctas), dim3(m.threads), args, m.smem, s);
   count_launch();
   return e;
+}
+
+template <typename Kern>
+cudaError_t cluster_launch_config(Kern kern, const ModeCfg& m, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr,
+                                  cudaStream_t s) {
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m.smem);
+  if (e == cudaSuccess && m.ctas > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+  if (e != cudaSuccess) return e;
+  *cfg = cudaLaunchConfig_t{};
+  cfg->gridDim = dim3(m.ctas);
+  cfg->blockDim = dim3(m.threads);
+  cfg->dynamicSmemBytes = m.smem;
+  cfg->stream = s;
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = m.ctas;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg->attrs = attr;
+  cfg->numAttrs = 1;
+  return cudaSuccess;
+}
+
+// Can one cluster of this shape be resident?  (asked once, at creation)
+template <typename Kern>
+bool cluster_fits(Kern kern, const ModeCfg& m) {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  if (cluster_launch_config(kern, m, &cfg, attr, nullptr) != cudaSuccess) { cudaGetLastError(); return false; }
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
+  return n >= 1;
+}
+
+template <typename Kern>
+cudaError_t launch_cluster(Kern kern, const ModeCfg& m, const GruParams& p, cudaStream_t s) {
+  cudaLaunchConfig_t cfg;
+  cudaLaunchAttribute attr[1];
+  cudaError_t e = cluster_launch_config(kern, m, &cfg, attr, s);
+  if (e != cudaSuccess) return e;
+  e = cudaLaunchKernelEx(&cfg, kern, p);
+  count_launch();
+  return e;
+}
+
+// The compiled variants of the register-resident kernel: (BH, items per warp, slots per item).
+using GruKernel = void (*)(const GruParams);
+GruKernel reg_kernel(int BH, int ni, int s) {
+  if (BH != 8) return nullptr;
+  if (ni == 1 && s == 2) return gru_cluster_reg_kernel<8, 1, 2>;
+  if (ni == 1 && s == 4) return gru_cluster_reg_kernel<8, 1, 4>;
+  if (ni == 3 && s == 3) return gru_cluster_reg_kernel<8, 3, 3>;
+  if (ni == 3 && s == 4) return gru_cluster_reg_kernel<8, 3, 4>;
+  return nullptr;
+}
+GruKernel smem_cluster_kernel(int BH) {
+  return BH == 4 ? gru_cluster_kernel<4> : (BH == 8 ? gru_cluster_kernel<8> : gru_cluster_kernel<16>);
+}
+
+// Largest number of kept columns in half a band, over all bands of all layers.
+int max_half_band_columns(const grim_gru* g) {
+  uint32_t mx = 0;
+  for (const grim_bcr* wh : g->Whh)
+    for (int64_t pos = 0; pos < wh->nbr; ++pos) {
+      uint32_t n = 0;
+      for (uint32_t k = wh->h_gemv_band_ptr[(size_t)pos]; k < wh->h_gemv_band_ptr[(size_t)pos + 1]; ++k)
+        n += wh->h_chunks[k].ncols_kr & 0xFFFFu;
+      mx = std::max(mx, (n + 1) / 2);
+    }
+  return (int)mx;
+}
+
+// How much of the chunk layout the busiest CTA would hold when CTA c owns groups [c*tpc, (c+1)*tpc).
+void residency_needs(const grim_gru* g, ModeCfg& m) {
+  const int ntri = (int)(g->H / g->bh);
+  const int nb = 3 * m.tpc;
+  for (size_t l = 0; l < g->Whh.size(); ++l) {
+    const grim_bcr* wh = g->Whh[l];
+    std::vector<uint32_t> pos_of_band((size_t)wh->nbr);
+    for (size_t p = 0; p < pos_of_band.size(); ++p) pos_of_band[wh->band_order[p]] = (uint32_t)p;
+    for (int c = 0; c < m.ctas; ++c) {
+      uint32_t nc = 0, ncw = 0, nv = 0;
+      for (int lb = 0; lb < nb; ++lb) {
+        const int tri = c * m.tpc + lb / 3;
+        if (tri >= ntri) continue;
+        const uint32_t pos = pos_of_band[(size_t)((lb % 3) * ntri + tri)];
+        for (uint32_t k = wh->h_gemv_band_ptr[pos]; k < wh->h_gemv_band_ptr[pos + 1]; ++k) {
+          const uint32_t nk = wh->h_chunks[k].ncols_kr;
+          ++nc; ncw += nk & 0xFFFFu; nv += (nk & 0xFFFFu) * (nk >> 16);
+        }
+      }
+      m.max_chunks = std::max(m.max_chunks, nc);
+      m.max_cw = std::max(m.max_cw, ncw);
+      m.max_vals = std::max(m.max_vals, nv);
+    }
+  }
 }
 
 void destroy(grim_gru* g) {
@@ -250,6 +579,8 @@ void destroy(grim_gru* g) {
   cudaFree(g->d_sync);
   delete g;
 }
+
+constexpr size_t kSmemLimit = 200 * 1024;
 
 }  // namespace
 
@@ -274,12 +605,7 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
   g->L = layers; g->H = H; g->max_T = max_T; g->bh = bh;
   cudaGetDevice(&g->device);
   const int ntri = (int)(H / bh);
-  g->tpc = (ntri + 127) / 128;
-  if (3 * g->tpc > kMaxLocalBands) { delete g; return GRIM_ERR_UNSUPPORTED; }
-  g->grid = (ntri + g->tpc - 1) / g->tpc;
-  const int nb = 3 * g->tpc;
-  g->ks = std::max(1, std::min(4, 32 / nb));
-  g->threads = std::max(nb * g->ks * 32, ((g->tpc * bh + 31) / 32) * 32);
+  const int BHc = bh <= 4 ? 4 : (bh <= 8 ? 8 : 16);
   grim_status_t st = GRIM_OK;
   try {
     for (int l = 0; l < layers && st == GRIM_OK; ++l) {
@@ -288,22 +614,6 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
       g->Whh.push_back(wh);
       std::vector<uint32_t> pos_of_band((size_t)wh->nbr);
       for (size_t p = 0; p < pos_of_band.size(); ++p) pos_of_band[wh->band_order[p]] = (uint32_t)p;
-      // per thread block: how much of the chunk layout it would hold on-chip
-      for (int c = 0; c < g->grid; ++c) {
-        uint32_t nc = 0, ncw = 0, nv = 0;
-        for (int lb = 0; lb < nb; ++lb) {
-          const int tri = c * g->tpc + lb / 3;
-          if (tri >= ntri) continue;
-          const uint32_t pos = pos_of_band[(size_t)((lb % 3) * ntri + tri)];
-          for (uint32_t k = wh->h_gemv_band_ptr[pos]; k < wh->h_gemv_band_ptr[pos + 1]; ++k) {
-            const uint32_t nk = wh->h_chunks[k].ncols_kr;
-            ++nc; ncw += nk & 0xFFFFu; nv += (nk & 0xFFFFu) * (nk >> 16);
-          }
-        }
-        g->max_chunks = std::max(g->max_chunks, nc);
-        g->max_cw = std::max(g->max_cw, ncw);
-        g->max_vals = std::max(g->max_vals, nv);
-      }
       float *db1 = nullptr, *db2 = nullptr;
       uint32_t* dp = nullptr;
       cudaError_t e = cudaMalloc((void**)&db1, (size_t)3 * H * 4);
@@ -325,18 +635,65 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
       if (e == cudaSuccess) e = cudaMemset(g->d_sync, 0, (size_t)(layers + 1) * 4);
       if (e != cudaSuccess) st = e == cudaErrorMemoryAllocation ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;
     }
+    if (st == GRIM_OK) {
+      // ---- cooperative-grid shape: up to 128 CTAs, weights on-chip if they fit, else streamed from L2
+      ModeCfg& m = g->grid;
+      m.tpc = (ntri + 127) / 128;
+      if (3 * m.tpc <= kMaxLocalBands) {
+        m.ctas = (ntri + m.tpc - 1) / m.tpc;
+        const int nb = 3 * m.tpc;
+        m.ks = std::max(1, std::min(4, 32 / nb));
+        m.threads = std::min(1024, std::max(nb * m.ks * 32, ((m.tpc * bh + 31) / 32) * 32));
+        residency_needs(g, m);
+        m.resident = 1;
+        m.smem = smem_bytes(g, m, BHc, false);
+        if (m.smem > kSmemLimit) { m.resident = 0; m.smem = smem_bytes(g, m, BHc, false); }
+        m.ok = m.smem <= kSmemLimit;
+      }
+      // ---- cluster shape: the largest cluster (<= 16 CTAs) that divides the unit groups evenly
+      for (int cs = 16; cs >= 1 && !g->cluster.ok; cs >>= 1) {
+        if (ntri % cs) continue;
+        ModeCfg t;
+        t.tpc = ntri / cs;
+        if (3 * t.tpc > kMaxLocalBands || t.tpc * bh > 1024) continue;
+        t.ctas = cs;
+        const int nb = 3 * t.tpc;
+        t.ks = std::max(1, std::min(4, 32 / nb));
+        t.threads = std::min(1024, std::max(std::max(nb * t.ks * 32, ((t.tpc * bh + 31) / 32) * 32), 256));
+        residency_needs(g, t);
+        t.resident = 1;
+        t.smem = smem_bytes(g, t, BHc, true);
+        if (t.smem > kSmemLimit) continue;  // the cluster scheme is only used with weights on-chip
+        g->cluster = t;
+        g->cluster.ok = cluster_fits(smem_cluster_kernel(BHc), g->cluster);
+        if (!g->cluster.ok) g->cluster = ModeCfg{};
+      }
+      // ---- register-resident cluster shape: 16 warps, two work items per band
+      const int slots_needed = (max_half_band_columns(g) + 31) / 32;
+      for (int cs = 16; cs >= 1 && !g->regc.ok; cs >>= 1) {
+        if (ntri % cs) continue;
+        ModeCfg t;
+        t.tpc = ntri / cs;
+        const int nb = 3 * t.tpc;
+        if (t.tpc * bh > kRegThreads) continue;
+        const int ni_needed = (nb * 2 + kRegWarps - 1) / kRegWarps;
+        const int menu[4][2] = {{1, 2}, {1, 4}, {3, 3}, {3, 4}};
+        for (const auto& v : menu) {
+          if (v[0] < ni_needed || v[1] < slots_needed || !reg_kernel(BHc, v[0], v[1])) continue;
+          t.ctas = cs; t.ks = 2; t.threads = kRegThreads; t.resident = 1;
+          t.smem = (((size_t)2 * H + (size_t)((t.tpc * bh + 3) & ~3) + (size_t)nb * 2 * BHc) * 4 + 15) & ~size_t(15);
+          if (t.smem > kSmemLimit || !cluster_fits(reg_kernel(BHc, v[0], v[1]), t)) continue;
+          t.ok = true;
+          g->regc = t; g->reg_ni = v[0]; g->reg_s = v[1];
+          break;
+        }
+      }
+      if (!g->grid.ok && !g->cluster.ok && !g->regc.ok) st = GRIM_ERR_UNSUPPORTED;
+    }
   } catch (const std::bad_alloc&) {
     st = GRIM_ERR_ALLOC;
   }
   if (st != GRIM_OK) { cudaGetLastError(); destroy(g); return st; }
-  const int BHc = bh <= 4 ? 4 : (bh <= 8 ? 8 : 16);
-  g->resident = 1;
-  g->smem = gru_smem_bytes(g, BHc);
-  if (g->smem > 200 * 1024) {  // does not fit on-chip: stream the chunks from L2 every step
-    g->resident = 0;
-    g->smem = gru_smem_bytes(g, BHc);
-    if (g->smem > 200 * 1024) { destroy(g); return GRIM_ERR_UNSUPPORTED; }
-  }
   *out = g;
   return GRIM_OK;
 }
@@ -348,6 +705,12 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
   cudaStream_t s = (cudaStream_t)stream;
   g->last_stream = s;
   const int64_t H = g->H;
+  // preference: weights in registers > cooperative grid > shared-memory cluster
+  const bool want_grid = g->force_grid && g->grid.ok;
+  const bool use_reg = g->regc.ok && !want_grid;
+  const bool use_cluster = !use_reg && g->cluster.ok && !g->grid.ok;
+  const ModeCfg& m = use_reg ? g->regc : (use_cluster ? g->cluster : g->grid);
+  const int BHc = g->bh <= 4 ? 4 : (g->bh <= 8 ? 8 : 16);
   if (cudaMemsetAsync(g->d_sync, 0, (size_t)(g->L + 1) * 4, s) != cudaSuccess) return GRIM_ERR_CUDA;
   const float* seq_in = x;
   for (int l = 0; l < g->L; ++l) {
@@ -369,13 +732,19 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     p.b_hh = g->d_bhh[l]; p.gi = g->d_gi; p.h0 = h0 ? h0 + (int64_t)l * H : nullptr;
     p.out = seq_out; p.hT = hT ? hT + (int64_t)l * H : nullptr;
     p.bar = g->d_sync + l; p.status = g->d_sync + g->L;
-    p.H = (int)H; p.bh = g->bh; p.T = (int)T; p.tpc = g->tpc; p.ks = g->ks; p.resident = g->resident;
-    p.max_chunks = g->max_chunks; p.max_cw = g->max_cw; p.max_vals = g->max_vals;
+    p.H = (int)H; p.bh = g->bh; p.T = (int)T; p.tpc = m.tpc; p.ks = m.ks; p.resident = m.resident;
+    p.max_chunks = m.max_chunks; p.max_cw = m.max_cw; p.max_vals = m.max_vals;
     p.skip_cta = g->dbg_skip_cta; p.spin_limit = g->spin_limit;
     cudaError_t e;
-    if (g->bh <= 4) e = launch_recurrent<4>(g, p, s);
-    else if (g->bh <= 8) e = launch_recurrent<8>(g, p, s);
-    else e = launch_recurrent<16>(g, p, s);
+    if (use_reg) {
+      e = launch_cluster(reg_kernel(BHc, g->reg_ni, g->reg_s), m, p, s);
+    } else if (use_cluster) {
+      e = launch_cluster(smem_cluster_kernel(BHc), m, p, s);
+    } else {
+      if (g->bh <= 4) e = launch_grid<4>(g, p, s);
+      else if (g->bh <= 8) e = launch_grid<8>(g, p, s);
+      else e = launch_grid<16>(g, p, s);
+    }
     if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorCooperativeLaunchTooLarge ? GRIM_ERR_UNSUPPORTED : GRIM_ERR_CUDA; }
     if (g->profile) cudaEventRecord(g->ev[3 * l + 2], s);
     seq_in = seq_out;
@@ -391,13 +760,16 @@ extern "C" grim_status_t grim_gru_status(grim_gru_t g) {
   return (grim_status_t)v;
 }
 
-// Test hook: make thread block `skip_cta` stay away from the barrier (-1: off) and set the number of
+// Test hook: selects the cooperative-grid kernel (the one with spin waits) whenever skip_cta >= 0 or a
+// poll limit is given, makes thread block `skip_cta` stay away from its barrier and sets the number of
 // polls after which a waiting block gives up.  The waits then run out and the status word reports it;
 // no thread block ever waits without a bound.
 extern "C" grim_status_t grim_gru_debug_barrier(grim_gru_t g, int skip_cta, unsigned spin_limit) {
   if (!g) return GRIM_ERR_INVALID_ARG;
+  if ((skip_cta >= 0 || spin_limit) && !g->grid.ok) return GRIM_ERR_UNSUPPORTED;
   g->dbg_skip_cta = skip_cta;
   g->spin_limit = spin_limit ? spin_limit : (1u << 22);
+  g->force_grid = skip_cta >= 0 || spin_limit != 0;
   return GRIM_OK;
 }
 

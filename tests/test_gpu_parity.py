@@ -289,10 +289,12 @@ def build_gru(B, m, max_T):
     return g, hi + hh
 
 
-def check_gru(B, m, h0=None):
+def check_gru(B, m, h0=None, grid_kernel=False):
     T, H, L = m["T"], m["hidden"], len(m["layers"])
     g, handles = build_gru(B, m, T)
     try:
+        if grid_kernel:  # a poll limit selects the cooperative-grid kernel instead of the cluster kernel
+            B.grim_gru_debug_barrier(g, -1, 1 << 22)
         x = to_dev(m["x"])
         y = torch.full((T, H), float("nan"), device="cuda")
         hT = torch.full((L, H), float("nan"), device="cuda")
@@ -316,10 +318,12 @@ def test_gru_small(B, cfg):
     check_gru(B, m)
     h0 = gen.normal_f32((L, H), 0.5, 81, 0)
     check_gru(B, m, h0=h0)
+    check_gru(B, m, h0=h0, grid_kernel=True)
 
 
-def test_config2_gru_full(B):
-    check_gru(B, gen.gru_model())
+@pytest.mark.parametrize("grid_kernel", [False, True])
+def test_config2_gru_full(B, grid_kernel):
+    check_gru(B, gen.gru_model(), grid_kernel=grid_kernel)
 
 
 def test_gru_bounded_wait_reports_timeout(B):
