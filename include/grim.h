@@ -85,8 +85,12 @@ typedef struct {
 /* Tile-shape choice for the N > 1 kernel (Section 4.5: tile sizes are tuned per kernel).
  * Zero in a field means "library default for this problem". */
 typedef struct {
-  int32_t tile_n;  /* output columns per thread block: 16, 32, 64 or 128 */
-  int32_t path;    /* 0 auto, 1 CUDA-core FFMA tiles, 2 tcgen05 tensor-core tiles (bf16 handles only) */
+  int32_t tile_n;  /* path 4: output columns per thread block (16, 32, 64 or 128);
+                      path 1: groups of 16 row bands per thread block (1, 2 or 4) */
+  int32_t path;    /* 0 auto; 1 register-tiled CUDA-core kernel (N > 16); 2 tcgen05 tensor-core tiles (bf16
+                      handles only); 3 lane-per-column kernel (N <= 16, N = 1 is the matrix-vector product);
+                      4 shared-memory slab kernel (any N; the fall-back for operands the others do not take).
+                      A path that cannot take the request returns GRIM_ERR_UNSUPPORTED. */
   int32_t reserved[6];
 } grim_tune_t;
 
@@ -141,6 +145,12 @@ grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);
  * Asynchronous on `stream`.
  */
 grim_status_t grim_bcr_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, grim_stream_t stream);
+
+/* The multiply kernels bound every device-side wait (on a shared-memory barrier that an asynchronous copy
+ * completes).  If one ever gives up, the kernel leaves, Y is invalid and an error word in the handle is set.
+ * grim_bcr_status synchronises the device, returns GRIM_ERR_TIMEOUT in that case (GRIM_OK otherwise) and
+ * clears the word.  (Robustness aid; no counterpart in the paper.) */
+grim_status_t grim_bcr_status(grim_bcr_t h);
 
 /* Same with an explicit tile choice (Section 4.5, tuning).  tune may be NULL. */
 grim_status_t grim_bcr_spmm_ex(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune,

@@ -30,7 +30,7 @@ GRIM_CONV_RELU = 1
 
 EXPORTED = [
     "grim_bcr_pack", "grim_bcr_destroy", "grim_bcr_info", "grim_bcr_export", "grim_bcr_unpack_dense",
-    "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
+    "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static",
     "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version",
@@ -69,6 +69,7 @@ _vp = C.c_void_p
 lib.grim_bcr_pack.argtypes = [_vp, C.c_int64, _vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_int,
                               C.c_uint32, C.POINTER(_vp)]
 lib.grim_bcr_destroy.argtypes = [_vp]
+lib.grim_bcr_status.argtypes = [_vp]
 lib.grim_bcr_info.argtypes = [_vp, C.POINTER(grim_bcr_info_t)]
 lib.grim_bcr_export.argtypes = [_vp, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.grim_bcr_unpack_dense.argtypes = [_vp, _vp, C.c_int64]
@@ -176,6 +177,10 @@ def grim_bcr_unpack_dense(h: int) -> np.ndarray:
 def grim_bcr_spmm(h: int, X, Y, stream=None):
     mx, my = _mat(X), _mat(Y)
     _check(lib.grim_bcr_spmm(h, C.byref(mx), C.byref(my), _stream_ptr(stream)), "grim_bcr_spmm")
+
+
+def grim_bcr_status(h: int) -> int:
+    return lib.grim_bcr_status(h)
 
 
 def grim_bcr_spmm_ex(h: int, X, Y, tile_n: int = 0, path: int = 0, stream=None):

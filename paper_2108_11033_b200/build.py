@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libgrim.so")
-SOURCES = ["grim_pack.cu", "grim_spmm.cu", "grim_tc.cu", "grim_api.cu", "grim_gru.cu"]
+SOURCES = ["grim_pack.cu", "grim_spmm.cu", "grim_ffma.cu", "grim_tc.cu", "grim_api.cu", "grim_gru.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 
@@ -56,7 +56,7 @@ def build_library(force: bool = False, verbose: bool = False) -> str:
                 sys.stderr.write(r.stderr)
     objs = [os.path.join(OBJ, s.replace(".cu", ".o")) for s in sources]
     if force or jobs or _newer(LIB, objs):
-        cmd = [nvcc] + ARCH + ["-shared", "-o", LIB] + objs + ["-lcuda"]
+        cmd = [nvcc] + ARCH + ["-shared", "-o", LIB] + objs
         r = subprocess.run(cmd, capture_output=True, text=True)
         if r.returncode != 0:
             sys.stderr.write(r.stdout + r.stderr)

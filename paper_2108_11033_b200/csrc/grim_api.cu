@@ -31,18 +31,21 @@ SpmmArgs mat_args(const grim_mat_t* X, const grim_mat_t* Y) {
 grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune, cudaStream_t s) {
   grim_status_t st = check_mats(h, X, Y);
   if (st != GRIM_OK) return st;
-  const int path = tune ? tune->path : 0;
-  if (path < 0 || path > 2) return GRIM_ERR_INVALID_ARG;
-  if (X->cols == 1 && h->gemv_ok && path != 2 && !(tune && tune->tile_n))
-    return launch_gemv(h, X->ptr, X->dtype, Y->dtype == GRIM_F32 ? (float*)Y->ptr : nullptr,
-                       Y->dtype == GRIM_BF16 ? Y->ptr : nullptr, s);
+  int path = tune ? tune->path : 0;
+  if (path < 0 || path > 4) return GRIM_ERR_INVALID_ARG;
+  if (path == 0 && tune && tune->tile_n >= 16) path = 4;  // a column-tile width only means something to the slab kernel
   SpmmArgs a = mat_args(X, Y);
   a.tile_n = tune ? tune->tile_n : 0;
   if (path == 2) {
     if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
     return launch_spmm_tc(h, a, s);
   }
+  if (path == 3 || (path == 0 && X->cols <= kSkinnyMaxN && h->gemv_ok))
+    return launch_skinny(h, X->ptr, X->dtype, X->ld, X->cols, Y->ptr, Y->dtype, Y->ld, s);
+  if (path == 4) return launch_spmm(h, a, s);
   if (path == 0 && tc_path_supported(h, a) && a.ncols >= 256) return launch_spmm_tc(h, a, s);
+  if (ffma_path_supported(h, a)) return launch_ffma(h, a, s);
+  if (path == 1) return GRIM_ERR_UNSUPPORTED;
   return launch_spmm(h, a, s);
 }
 
@@ -83,33 +86,28 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return GRIM_ERR_CUDA;
   float best_t = -1.f;
   grim_tune_t cand_best{};
-  const int tiles[4] = {16, 32, 64, 128};
-  for (int path = 1; path <= 2; ++path) {
-    for (int ti = 0; ti < 4; ++ti) {
-      grim_tune_t c{};
-      c.path = path;
-      c.tile_n = tiles[ti];
-      if (path == 2) {
-        if (ti != 0) continue;
-        c.tile_n = 0;
-        SpmmArgs a = mat_args(X, Y);
-        if (!tc_path_supported(h, a)) continue;
-      } else if (c.tile_n > 16 && c.tile_n / 2 >= X->cols) {
-        continue;  // a wider tile than the matrix needs only adds idle lanes
-      }
-      st = run_spmm(h, X, Y, &c, s);  // warm-up
-      if (st != GRIM_OK) break;
-      cudaEventRecord(e0, s);
-      for (int r = 0; r < reps && st == GRIM_OK; ++r) st = run_spmm(h, X, Y, &c, s);
-      cudaEventRecord(e1, s);
-      if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
-      float ms = 0.f;
-      cudaEventElapsedTime(&ms, e0, e1);
-      ms /= reps;
-      if (best_t < 0.f || ms < best_t) { best_t = ms; cand_best = c; }
-    }
+  // candidates: (path, tile_n); a candidate that cannot take the request is skipped
+  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {3, 0}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
+  for (const auto& cd : cand) {
+    grim_tune_t c{};
+    c.path = cd[0];
+    c.tile_n = cd[1];
+    if (c.path == 3 && X->cols > kSkinnyMaxN) continue;
+    if (c.path == 4 && c.tile_n > 16 && c.tile_n / 2 >= X->cols) continue;  // idle lanes only
+    if (c.path == 1 && c.tile_n > (h->bh <= 4 ? 4 : (h->bh <= 8 ? 2 : 1))) continue;
+    st = run_spmm(h, X, Y, &c, s);  // warm-up
+    if (st == GRIM_ERR_UNSUPPORTED) { st = GRIM_OK; continue; }
     if (st != GRIM_OK) break;
+    cudaEventRecord(e0, s);
+    for (int r = 0; r < reps && st == GRIM_OK; ++r) st = run_spmm(h, X, Y, &c, s);
+    cudaEventRecord(e1, s);
+    if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    ms /= reps;
+    if (best_t < 0.f || ms < best_t) { best_t = ms; cand_best = c; }
   }
+  if (st == GRIM_OK && best_t < 0.f) st = GRIM_ERR_UNSUPPORTED;
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
   if (st != GRIM_OK) return st;

@@ -1,0 +1,519 @@
+// Register-tiled CUDA-core kernel for Y = W * X with N > 16 (Sections 3.1, 4.2 - 4.5).
+//
+// One thread block (16 warps) owns BPW groups of 16 row bands and a tile of 128 output columns and walks
+// the block columns.  Per block column a slab of X (bw rows x 128 columns) is brought into shared memory
+// once - by TMA when X is a plain row-major matrix, otherwise by 4-byte cp.async gathers (strided X, or the
+// implicit im2col of Section 4.5 taken directly from the NCHW input) - together with the packed records of
+// the thread block's bands for that block column.  A ring of stages with full / empty mbarriers lets warps
+// run up to a stage apart, which absorbs the uneven work of bands (Section 4.2's load imbalance).
+//
+// A warp owns one band per group, a lane four output columns.  Per block the lane loads the slab rows of
+// eight kept columns into registers once (each needed input row is read once and reused by every kept row -
+// the load-redundancy idea of Section 4.4) and then, per kept row, reads the row's eight weights with two
+// broadcast 128-bit loads and issues 32 FMAs into that row's accumulators.  Which accumulator registers a
+// kept row uses is decided by one jump per (row, eight columns); everything inside is straight-line code.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+
+#include "grim_internal.h"
+
+namespace grim {
+namespace {
+
+constexpr int kFThreads = 512;
+constexpr int kFWarps = 16;
+constexpr int kTN = 128;          // output columns per thread block
+constexpr int kStages = 4;        // ring slots
+constexpr int kAhead = 2;         // stages requested ahead of the one being multiplied
+constexpr int kJlistCap = 2048;   // block columns per matrix the stage list can hold
+constexpr int kHdrBytes = (128 + kStages * 16 + kJlistCap * 2 + 127) / 128 * 128;  // barriers, flags, per-slot blob sizes, stage list
+
+enum { kModeTma = 0, kModeGather = 1 };
+
+struct FParams {
+  const RcStage* stage;
+  const uint8_t* blob;
+  const uint32_t* band_order;
+  unsigned* status;
+  int nbr, nbc, M, K, bh, bw, ngroups;
+  uint32_t blob_stride, slab_bytes;
+  unsigned spin_limit;
+  SpmmArgs a;
+};
+
+// ---- mbarrier / async-copy wrappers -----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bounded wait: false when the limit ran out (the caller then raises the abort flag and leaves).
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
+  for (unsigned i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u && *abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ void cp_async4_zfill(void* dst, const void* src, bool valid) {
+  const unsigned n = valid ? 4u : 0u;
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
+}
+__device__ __forceinline__ void cp_async16_cg(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+
+__device__ __forceinline__ float4 ld_x4(const float* slab, unsigned col, int lane) {
+  return *reinterpret_cast<const float4*>(slab + col * kTN + lane * 4);
+}
+__device__ __forceinline__ float4 ld_x4(const __nv_bfloat16* slab, unsigned col, int lane) {
+  const uint2 u = *reinterpret_cast<const uint2*>(slab + col * kTN + lane * 4);
+  return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16),
+                     __uint_as_float(u.y & 0xFFFF0000u));
+}
+
+#define GRIM_FMA4(A, W, X)          \
+  A.x = fmaf(W, X.x, A.x);          \
+  A.y = fmaf(W, X.y, A.y);          \
+  A.z = fmaf(W, X.z, A.z);          \
+  A.w = fmaf(W, X.w, A.w);
+#define GRIM_ROW_CASE(R)                                   \
+  case R: {                                                \
+    if (R < BH) {                                          \
+      float4& A = acc[b][R < BH ? R : 0];                  \
+      GRIM_FMA4(A, w0.x, x[0]) GRIM_FMA4(A, w0.y, x[1])    \
+      GRIM_FMA4(A, w0.z, x[2]) GRIM_FMA4(A, w0.w, x[3])    \
+      GRIM_FMA4(A, w1.x, x[4]) GRIM_FMA4(A, w1.y, x[5])    \
+      GRIM_FMA4(A, w1.z, x[6]) GRIM_FMA4(A, w1.w, x[7])    \
+    }                                                      \
+    break;                                                 \
+  }
+
+template <int BH, int BPW, typename XT, int MODE>
+__global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_constant__ CUtensorMap tmX, const FParams p) {
+  extern __shared__ __align__(128) uint8_t smem[];
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);
+  uint64_t* empty = full + kStages;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 64);
+  int* s_nst = reinterpret_cast<int*>(smem + 68);
+  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 128);               // [kStages][4] blob bytes per band group
+  uint16_t* jlist = reinterpret_cast<uint16_t*>(smem + 128 + kStages * 16);  // non-empty block columns, ascending
+  uint8_t* slots = smem + kHdrBytes;
+  const uint32_t slot_bytes = p.slab_bytes + BPW * p.blob_stride;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const SpmmArgs& a = p.a;
+  const int64_t q0 = (int64_t)blockIdx.x * kTN;
+  const int g0 = blockIdx.y * BPW;
+
+  if (warp == 0) {
+    int n = 0;
+    for (int j0 = 0; j0 < p.nbc; j0 += 32) {
+      const int j = j0 + lane;
+      bool f = false;
+      if (j < p.nbc)
+        for (int b = 0; b < BPW; ++b)
+          if (g0 + b < p.ngroups) f = f || p.stage[(int64_t)(g0 + b) * p.nbc + j].bytes != 0;
+      const unsigned m = __ballot_sync(0xffffffffu, f);
+      if (f) jlist[n + __popc(m & ((1u << lane) - 1u))] = (uint16_t)j;
+      n += __popc(m);
+    }
+    if (lane == 0) {
+      *s_nst = n;
+      *s_abort = 0;
+      for (int s = 0; s < kStages; ++s) {
+        mbar_init(full + s, MODE == kModeTma ? 1u : (unsigned)kFThreads);
+        mbar_init(empty + s, kFWarps);
+      }
+      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+  }
+  __syncthreads();
+  const int nst = *s_nst;
+
+  // per-thread constants of the gather loader: this thread always fills column qq of the slab
+  const int qq = tid & (kTN - 1);
+  const int kk0 = tid >> 7;  // first slab row; then every 4th
+  int ih0 = 0, iw0 = 0;
+  int64_t qoff = 0;
+  bool q_ok = false;
+  if (MODE == kModeGather) {
+    const int64_t q = q0 + qq;
+    q_ok = q < a.ncols;
+    if (a.conv) {
+      const int64_t ohw = (int64_t)a.OH * a.OW;
+      const int64_t img = q_ok ? q / ohw : 0;
+      const int pix = q_ok ? (int)(q - img * ohw) : 0;
+      const int oh = pix / a.OW, ow = pix - oh * a.OW;
+      ih0 = oh * a.stride - a.pad;
+      iw0 = ow * a.stride - a.pad;
+      qoff = img * a.C * a.H * a.W + (int64_t)ih0 * a.W + iw0;
+    } else {
+      qoff = q * a.x_sq;
+    }
+  }
+
+  // Requests stage n (the n-th non-empty block column) into its ring slot.
+  auto request = [&](int n) {
+    const int slot = n % kStages;
+    const int j = jlist[n];
+    uint8_t* base = slots + (size_t)slot * slot_bytes;
+    if (MODE == kModeTma) {
+      // one thread: sizes first (read by the consumers after the barrier completes), then the copies
+      uint32_t bytes[BPW], off[BPW], total = p.slab_bytes;
+#pragma unroll
+      for (int b = 0; b < BPW; ++b) {
+        bytes[b] = 0; off[b] = 0;
+        if (g0 + b < p.ngroups) {
+          const RcStage se = p.stage[(int64_t)(g0 + b) * p.nbc + j];
+          bytes[b] = se.bytes; off[b] = se.off16;
+        }
+        s_meta[slot * 4 + b] = bytes[b];
+        total += bytes[b];
+      }
+      mbar_arrive_expect_tx(full + slot, total);
+      tma_load_2d(base, &tmX, (int)q0, j * p.bw, full + slot);
+#pragma unroll
+      for (int b = 0; b < BPW; ++b)
+        if (bytes[b]) bulk_load(base + p.slab_bytes + b * p.blob_stride, p.blob + (size_t)off[b] * 16, bytes[b], full + slot);
+    } else {
+      float* slab = reinterpret_cast<float*>(base);
+      const float* X = static_cast<const float*>(a.X);
+      int64_t k = (int64_t)j * p.bw + kk0;
+      if (a.conv) {
+        const int khw = a.KH * a.KW;
+        int c = (int)(k / khw);
+        int rem = (int)(k - (int64_t)c * khw);
+        int kh = rem / a.KW, kw = rem - kh * a.KW;
+        for (int kk = kk0; kk < p.bw; kk += 4, k += 4) {
+          const int ih = ih0 + kh, iw = iw0 + kw;
+          const bool ok = q_ok && k < p.K && ih >= 0 && ih < a.H && iw >= 0 && iw < a.W;
+          const float* src = ok ? X + qoff + ((int64_t)c * a.H + kh) * a.W + kw : X;
+          cp_async4_zfill(slab + kk * kTN + qq, src, ok);
+          kw += 4;
+          while (kw >= a.KW) { kw -= a.KW; ++kh; }
+          while (kh >= a.KH) { kh -= a.KH; ++c; }
+        }
+      } else {
+        for (int kk = kk0; kk < p.bw; kk += 4, k += 4) {
+          const bool ok = q_ok && k < p.K;
+          cp_async4_zfill(slab + kk * kTN + qq, ok ? X + k * a.x_sk + qoff : X, ok);
+        }
+      }
+#pragma unroll
+      for (int b = 0; b < BPW; ++b) {
+        uint32_t bytes = 0, off = 0;
+        if (g0 + b < p.ngroups) {
+          const RcStage se = p.stage[(int64_t)(g0 + b) * p.nbc + j];
+          bytes = se.bytes; off = se.off16;
+        }
+        if (tid == 0) s_meta[slot * 4 + b] = bytes;
+        uint8_t* dst = base + p.slab_bytes + b * p.blob_stride;
+        const uint8_t* src = p.blob + (size_t)off * 16;
+        for (uint32_t i = tid * 16; i < bytes; i += kFThreads * 16) cp_async16_cg(dst + i, src + i);
+      }
+      cp_async_arrive_noinc(full + slot);
+    }
+  };
+
+  float4 acc[BPW][BH];
+#pragma unroll
+  for (int b = 0; b < BPW; ++b)
+#pragma unroll
+    for (int r = 0; r < BH; ++r) acc[b][r] = make_float4(0.f, 0.f, 0.f, 0.f);
+
+  // prologue: the first kAhead stages go into fresh slots
+  for (int n = 0; n < kAhead && n < nst; ++n)
+    if (MODE != kModeTma || tid == 0) request(n);
+
+  bool failed = false;
+  for (int n = 0; n < nst; ++n) {
+    // ---- producer duty: request stage n + kAhead; its slot was last used by stage n + kAhead - kStages
+    const int m = n + kAhead;
+    if (m < nst) {
+      const bool mine = MODE != kModeTma || (warp == (n % kFWarps) && lane == 0);
+      if (mine) {
+        bool ok = true;
+        if (m >= kStages) ok = mbar_wait(empty + m % kStages, (unsigned)((m / kStages - 1) & 1), p.spin_limit, s_abort);
+        if (ok) request(m);
+        else failed = true;
+      }
+    }
+    if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
+    // ---- wait for stage n
+    const int slot = n % kStages;
+    if (!mbar_wait(full + slot, (unsigned)((n / kStages) & 1), p.spin_limit, s_abort)) failed = true;
+    if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
+    const uint8_t* base = slots + (size_t)slot * slot_bytes;
+    const XT* slab = reinterpret_cast<const XT*>(base);
+#pragma unroll
+    for (int b = 0; b < BPW; ++b) {
+      if (s_meta[slot * 4 + b] == 0) continue;
+      const uint8_t* blob = base + p.slab_bytes + b * p.blob_stride;
+      const uint32_t hdr = reinterpret_cast<const uint32_t*>(blob)[warp];
+      const int kr = (hdr >> 16) & 0xFF, nch = hdr >> 24;
+      if (kr == 0) continue;
+      const uint8_t* rec = blob + (hdr & 0xFFFFu) * 16;
+      const unsigned long long rows = *reinterpret_cast<const unsigned long long*>(rec);
+      const uint8_t* cols = rec + 8;
+      const float4* wp = reinterpret_cast<const float4*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
+      for (int ch = 0; ch < nch; ++ch) {
+        const uint2 cc = *reinterpret_cast<const uint2*>(cols + ch * kRcChunk);
+        float4 x[kRcChunk];
+        x[0] = ld_x4(slab, cc.x & 0xFFu, lane);
+        x[1] = ld_x4(slab, (cc.x >> 8) & 0xFFu, lane);
+        x[2] = ld_x4(slab, (cc.x >> 16) & 0xFFu, lane);
+        x[3] = ld_x4(slab, cc.x >> 24, lane);
+        x[4] = ld_x4(slab, cc.y & 0xFFu, lane);
+        x[5] = ld_x4(slab, (cc.y >> 8) & 0xFFu, lane);
+        x[6] = ld_x4(slab, (cc.y >> 16) & 0xFFu, lane);
+        x[7] = ld_x4(slab, cc.y >> 24, lane);
+        unsigned long long rr = rows;
+        for (int ai = 0; ai < kr; ++ai) {
+          const float4 w0 = wp[0], w1 = wp[1];
+          wp += 2;
+          const unsigned r = (unsigned)rr & 15u;
+          rr >>= 4;
+          switch (r) {
+            GRIM_ROW_CASE(0) GRIM_ROW_CASE(1) GRIM_ROW_CASE(2) GRIM_ROW_CASE(3)
+            GRIM_ROW_CASE(4) GRIM_ROW_CASE(5) GRIM_ROW_CASE(6) GRIM_ROW_CASE(7)
+            GRIM_ROW_CASE(8) GRIM_ROW_CASE(9) GRIM_ROW_CASE(10) GRIM_ROW_CASE(11)
+            GRIM_ROW_CASE(12) GRIM_ROW_CASE(13) GRIM_ROW_CASE(14) GRIM_ROW_CASE(15)
+          }
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0) mbar_arrive(empty + slot);
+  }
+
+  if (failed) {
+    // a bounded wait ran out: tell every warp, record it, let copies that were requested land, leave
+    *s_abort = 1;
+    if (lane == 0) atomicExch(p.status, (unsigned)GRIM_ERR_TIMEOUT);
+  }
+  __syncthreads();
+  if (*s_abort) {
+    if (tid == 0)
+      for (int s = 0; s < kStages; ++s)
+        for (unsigned i = 0; i < 4096u && !mbar_try_wait(full + s, 0) && !mbar_try_wait(full + s, 1); ++i) {}
+    return;
+  }
+
+  // ---- epilogue: bias, activation, store every row of the band (rows kept by no block are +0)
+  const int64_t q = q0 + lane * 4;
+  if (q >= a.ncols) return;
+  const int64_t ohw = (int64_t)a.OH * a.OW;
+#pragma unroll
+  for (int b = 0; b < BPW; ++b) {
+    const int pos = (g0 + b) * kRcBands + warp;
+    if (pos >= p.nbr) continue;
+    const int band = p.band_order[pos];
+#pragma unroll
+    for (int r = 0; r < BH; ++r) {
+      const int64_t row = (int64_t)band * p.bh + r;
+      if (r >= p.bh || row >= p.M) continue;
+      float t[4] = {acc[b][r].x, acc[b][r].y, acc[b][r].z, acc[b][r].w};
+      const float bias = a.bias ? __ldg(a.bias + row) : 0.f;
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        t[e] += bias;
+        if (a.relu) t[e] = fmaxf(t[e], 0.f);
+      }
+      int64_t off0;
+      bool contiguous;
+      if (a.conv) {
+        const int64_t img = q / ohw;
+        const int64_t pix = q - img * ohw;
+        off0 = (img * p.M + row) * ohw + pix;
+        contiguous = (pix + 3 < ohw) && (q + 3 < a.ncols);
+      } else {
+        off0 = row * a.y_sr + q * a.y_sq;
+        contiguous = a.y_sq == 1 && (q + 3 < a.ncols);
+      }
+      if (a.y_dtype == GRIM_F32) {
+        float* y = static_cast<float*>(a.Y);
+        if (contiguous && ((reinterpret_cast<uintptr_t>(y + off0) & 15) == 0)) {
+          *reinterpret_cast<float4*>(y + off0) = make_float4(t[0], t[1], t[2], t[3]);
+          continue;
+        }
+      } else {
+        __nv_bfloat16* y = static_cast<__nv_bfloat16*>(a.Y);
+        if (contiguous && ((reinterpret_cast<uintptr_t>(y + off0) & 7) == 0)) {
+          __nv_bfloat162 lo = __floats2bfloat162_rn(t[0], t[1]);
+          __nv_bfloat162 hi = __floats2bfloat162_rn(t[2], t[3]);
+          uint2 u;
+          u.x = *reinterpret_cast<unsigned*>(&lo);
+          u.y = *reinterpret_cast<unsigned*>(&hi);
+          *reinterpret_cast<uint2*>(y + off0) = u;
+          continue;
+        }
+      }
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        if (q + e >= a.ncols) break;
+        int64_t off;
+        if (a.conv) {
+          const int64_t img = (q + e) / ohw;
+          const int64_t pix = (q + e) - img * ohw;
+          off = (img * p.M + row) * ohw + pix;
+        } else {
+          off = row * a.y_sr + (q + e) * a.y_sq;
+        }
+        if (a.y_dtype == GRIM_F32) static_cast<float*>(a.Y)[off] = t[e];
+        else static_cast<__nv_bfloat16*>(a.Y)[off] = __float2bfloat16_rn(t[e]);
+      }
+    }
+  }
+}
+
+// The driver's tensor-map encoder, looked up through the runtime so that the library does not link
+// against the driver (it must load on machines without one).
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      p = nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+bool tma_eligible(const SpmmArgs& a) {
+  if (a.conv || a.x_sq != 1) return false;
+  const int esz = a.x_dtype == GRIM_F32 ? 4 : 2;
+  return (reinterpret_cast<uintptr_t>(a.X) % 16 == 0) && ((a.x_sk * esz) % 16 == 0) && a.ncols < (int64_t(1) << 31);
+}
+
+template <int BH, int BPW, typename XT, int MODE>
+cudaError_t launch_variant(const CUtensorMap& tm, const FParams& p, size_t smem, dim3 grid, cudaStream_t s) {
+  auto kern = bcr_ffma_kernel<BH, BPW, XT, MODE>;
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return e;
+  kern<<<grid, kFThreads, smem, s>>>(tm, p);
+  return cudaGetLastError();
+}
+
+template <int BH, typename XT, int MODE>
+cudaError_t launch_bpw(int bpw, const CUtensorMap& tm, const FParams& p, size_t smem, dim3 grid, cudaStream_t s) {
+  if (BH <= 8 && bpw == 2) return launch_variant<BH, (BH <= 8 ? 2 : 1), XT, MODE>(tm, p, smem, grid, s);
+  if (BH <= 4 && bpw == 4) return launch_variant<BH, (BH <= 4 ? 4 : 1), XT, MODE>(tm, p, smem, grid, s);
+  return launch_variant<BH, 1, XT, MODE>(tm, p, smem, grid, s);
+}
+
+template <typename XT, int MODE>
+cudaError_t launch_bh(int BHc, int bpw, const CUtensorMap& tm, const FParams& p, size_t smem, dim3 grid, cudaStream_t s) {
+  if (BHc == 4) return launch_bpw<4, XT, MODE>(bpw, tm, p, smem, grid, s);
+  if (BHc == 8) return launch_bpw<8, XT, MODE>(bpw, tm, p, smem, grid, s);
+  return launch_bpw<16, XT, MODE>(bpw, tm, p, smem, grid, s);
+}
+
+constexpr size_t kSmemBudget = 220 * 1024;
+
+size_t smem_need(const grim_bcr* h, int bpw, int esz) {
+  const size_t blob_stride = ((size_t)h->rc_max_blob + 127) & ~size_t(127);
+  return kHdrBytes + (size_t)kStages * ((size_t)h->bw * kTN * esz + bpw * blob_stride);
+}
+
+}  // namespace
+
+bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a) {
+  if (h->device < 0 || !h->d_rc_stage || !h->d_status) return false;
+  if (h->nbc > kJlistCap || h->rc_max_blob == 0 || h->rc_max_blob > 0xFFFF * 16u) return false;
+  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTN) return false;
+  const bool tma = tma_eligible(a);
+  if (!tma && a.x_dtype != GRIM_F32) return false;  // the gather loader moves 4-byte elements
+  if ((h->bw * kTN * (a.x_dtype == GRIM_F32 ? 4 : 2)) % 128 != 0) return false;
+  return smem_need(h, 1, a.x_dtype == GRIM_F32 ? 4 : 2) <= kSmemBudget;
+}
+
+grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
+  if (!ffma_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
+  const bool tma = tma_eligible(a);
+  const int esz = a.x_dtype == GRIM_F32 ? 4 : 2;
+  const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);
+  const int64_t qtiles = (a.ncols + kTN - 1) / kTN;
+  // band groups per thread block: as many as the accumulators allow, fewer when the grid would not fill the GPU
+  int bpw = BHc == 4 ? 4 : (BHc == 8 ? 2 : 1);
+  while (bpw > 1 && (smem_need(h, bpw, esz) > kSmemBudget || qtiles * ((h->rc_groups + bpw - 1) / bpw) < 148)) bpw >>= 1;
+  if (a.tile_n == 1 || a.tile_n == 2 || a.tile_n == 4) bpw = std::min(a.tile_n, BHc == 4 ? 4 : (BHc == 8 ? 2 : 1));
+  if (smem_need(h, bpw, esz) > kSmemBudget) return GRIM_ERR_UNSUPPORTED;
+  const int64_t gy = (h->rc_groups + bpw - 1) / bpw;
+  if (gy > 65535) return GRIM_ERR_UNSUPPORTED;
+
+  FParams p;
+  p.stage = h->d_rc_stage; p.blob = h->d_rc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
+  p.nbr = (int)h->nbr; p.nbc = (int)h->nbc; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.bw = h->bw;
+  p.ngroups = (int)h->rc_groups;
+  p.blob_stride = (h->rc_max_blob + 127u) & ~127u;
+  p.slab_bytes = (uint32_t)(h->bw * kTN * esz);
+  p.spin_limit = 1u << 20;
+  p.a = a;
+
+  CUtensorMap tm;
+  memset(&tm, 0, sizeof(tm));
+  if (tma) {
+    const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
+    const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * esz)};
+    const cuuint32_t box[2] = {(cuuint32_t)kTN, (cuuint32_t)h->bw};
+    const cuuint32_t estr[2] = {1, 1};
+    EncodeTiledFn encode = encode_tiled_fn();
+    if (!encode) return GRIM_ERR_CUDA;
+    const CUresult r = encode(&tm, esz == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16,
+                                              2, const_cast<void*>(a.X), dims, strides, box, estr,
+                                              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+                                              CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return GRIM_ERR_CUDA;
+  }
+  const size_t smem = smem_need(h, bpw, esz);
+  dim3 grid((unsigned)qtiles, (unsigned)gy);
+  cudaError_t e;
+  if (tma) {
+    e = esz == 4 ? launch_bh<float, kModeTma>(BHc, bpw, tm, p, smem, grid, s)
+                 : launch_bh<__nv_bfloat16, kModeTma>(BHc, bpw, tm, p, smem, grid, s);
+  } else {
+    e = launch_bh<float, kModeGather>(BHc, bpw, tm, p, smem, grid, s);
+  }
+  count_launch();
+  return e == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+}
+
+}  // namespace grim

@@ -124,7 +124,7 @@ __device__ BandView setup_bands(const GruParams& p, int cta, uint8_t* pool) {
       uint32_t n_cw = 0, n_v = 0;
       for (uint32_t c = cb; c < ce; ++c) {
         const uint32_t nk = p.chunks[c].ncols_kr;
-        n_cw += nk & 0xFFFFu;
+        n_cw += 32;  // every chunk owns 32 column words
         n_v += (nk & 0xFFFFu) * (nk >> 16);
       }
       s_src_c[lb] = cb;
@@ -557,7 +557,7 @@ void residency_needs(const grim_gru* g, ModeCfg& m) {
         const uint32_t pos = pos_of_band[(size_t)((lb % 3) * ntri + tri)];
         for (uint32_t k = wh->h_gemv_band_ptr[pos]; k < wh->h_gemv_band_ptr[pos + 1]; ++k) {
           const uint32_t nk = wh->h_chunks[k].ncols_kr;
-          ++nc; ncw += nk & 0xFFFFu; nv += (nk & 0xFFFFu) * (nk >> 16);
+          ++nc; ncw += 32; nv += (nk & 0xFFFFu) * (nk >> 16);
         }
       }
       m.max_chunks = std::max(m.max_chunks, nc);

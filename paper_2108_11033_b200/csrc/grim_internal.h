@@ -38,12 +38,33 @@ struct __align__(16) StageEntry {
 // Per band the kept columns of all its blocks are concatenated after sorting the blocks by
 // kept-row count, and cut into chunks of at most 32 columns that all have the same kept-row count kr.
 // Lane l of a warp owns column l of a chunk.  A column word is (global column | rowmask << 16).
+// Every chunk owns 32 column words (chunk c starts at word 32 * c; unused slots are 0, i.e. "no
+// row kept"), so that a warp can fetch the words without reading the descriptor first.
 // The chunk's values are stored step-major: value s of lane l is at val_off + s * ncols + l.
 // ---------------------------------------------------------------------------------------------
 struct ChunkDesc {
   uint32_t val_off;
   uint32_t cw_off;
   uint32_t ncols_kr;  // ncols | kr << 16
+};
+
+// ---------------------------------------------------------------------------------------------
+// Device layout for the register-tiled N > 16 kernel and the tensor-core kernel ("row-chunk"
+// layout).  Bands in schedule order are cut into groups of kRcBands; for group g and block column
+// j one contiguous blob:
+//   u32 hdr[kRcBands]     per band slot: record offset in 16-byte units | kr << 16 | nch << 24
+//   per band with kr > 0, 16-byte aligned:
+//     u64 rows            nibble a = block-local index of the a-th kept row
+//     u8  cols[nch * 8]   block-local kept columns, padded to a multiple of 8 by repeating the
+//                         first kept column (its padded weights are 0); then padding to 16 bytes
+//     f32 w[nch][kr][8]   w[c][a][e] = weight of kept row a and column cols[c * 8 + e]
+// Values are always fp32 here (bf16 handles store the rounded values widened to fp32).
+// ---------------------------------------------------------------------------------------------
+constexpr int kRcBands = 16;
+constexpr int kRcChunk = 8;
+struct RcStage {
+  uint32_t off16;  // blob start in 16-byte units from the blob base
+  uint32_t bytes;  // multiple of 16; 0 when no band of the group keeps anything in this block column
 };
 
 struct HostBlock {
@@ -77,8 +98,15 @@ struct grim_bcr {
   std::vector<uint32_t> h_gemv_band_ptr;   // host copies of the chunk tables (sizing of on-chip weight residency)
   std::vector<grim::ChunkDesc> h_chunks;
   int64_t n_colwords = 0;
+  // row-chunk layout
+  int64_t rc_groups = 0;
+  uint32_t rc_max_blob = 0;
+  int64_t index_bytes_rc = 0;
   // device
   int device = -1;
+  grim::RcStage* d_rc_stage = nullptr;
+  uint8_t* d_rc_blob = nullptr;
+  unsigned* d_status = nullptr;  // error word written by kernels whose bounded waits ran out
   grim::StageEntry* d_stage = nullptr;
   uint8_t* d_blob = nullptr;
   uint32_t* d_band_order = nullptr;
@@ -108,7 +136,11 @@ struct SpmmArgs {
 };
 
 grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
-grim_status_t launch_gemv(const grim_bcr* h, const void* x, int x_dtype, float* y_f32, void* y_bf16, cudaStream_t s);
+constexpr int kSkinnyMaxN = 16;  // widest right-hand side taken by the lane-per-column kernel
+grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
+                            int64_t ldy, cudaStream_t s);
+grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
+bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a);
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a);
 void count_launch(int n = 1);

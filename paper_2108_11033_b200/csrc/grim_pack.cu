@@ -46,6 +46,9 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_chunks);
   cudaFree(h->d_colwords);
   cudaFree(h->d_gemv_vals);
+  cudaFree(h->d_rc_stage);
+  cudaFree(h->d_rc_blob);
+  cudaFree(h->d_status);
 }
 
 int bands_per_group(int bh) { return bh <= 4 ? 32 : (bh <= 8 ? 16 : 8); }
@@ -247,6 +250,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
                 if ((m >> c) & 1ull) { if (b-- == 0) break; }
               colwords.push_back((uint32_t)(j * bw + c) | (hb.rowmask << 16));
             }
+            colwords.resize(chunks.size() * 32, 0u);  // every chunk owns 32 words; unused slots: no row kept
             for (int s = 0; s < kr; ++s)
               for (int l = 0; l < nc; ++l) {
                 const HostBlock& hb = h->blocks[(size_t)(i * nbc + cols[c0 + l].first)];
@@ -271,12 +275,77 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
                             (nbr + 1) * 4 + nbr * 4;
     }
 
+    // ---- row-chunk layout for the register-tiled and tensor-core kernels
+    std::vector<RcStage> rc_stage;
+    std::vector<uint8_t> rc_blob;
+    {
+      h->rc_groups = (nbr + kRcBands - 1) / kRcBands;
+      rc_stage.resize((size_t)(h->rc_groups * nbc));
+      rc_blob.reserve((size_t)nnz * 5 + (size_t)h->nonempty * 32 + 1024);
+      uint32_t rc_max = 0;
+      for (int64_t g = 0; g < h->rc_groups && st == GRIM_OK; ++g) {
+        for (int64_t j = 0; j < nbc; ++j) {
+          RcStage& se = rc_stage[(size_t)(g * nbc + j)];
+          se.off16 = (uint32_t)(rc_blob.size() / 16);
+          se.bytes = 0;
+          bool any = false;
+          for (int b = 0; b < kRcBands && !any; ++b) {
+            const int64_t pos = g * kRcBands + b;
+            if (pos >= nbr) break;
+            const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
+            any = hb.kr && hb.kc;
+          }
+          if (!any) continue;
+          if (rc_blob.size() / 16 >= (uint64_t(1) << 32)) { st = GRIM_ERR_UNSUPPORTED; break; }
+          const size_t start = rc_blob.size();
+          rc_blob.resize(start + kRcBands * 4, 0);
+          for (int b = 0; b < kRcBands; ++b) {
+            const int64_t pos = g * kRcBands + b;
+            if (pos >= nbr) break;
+            const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
+            if (!(hb.kr && hb.kc)) continue;
+            const int kr = hb.kr, kc = hb.kc, nch = (kc + kRcChunk - 1) / kRcChunk;
+            const size_t rec = rc_blob.size();
+            const uint32_t hdr = (uint32_t)((rec - start) / 16) | ((uint32_t)kr << 16) | ((uint32_t)nch << 24);
+            std::memcpy(&rc_blob[start + (size_t)b * 4], &hdr, 4);
+            const size_t idx_bytes = ((size_t)8 + (size_t)nch * kRcChunk + 15) / 16 * 16;
+            rc_blob.resize(rec + idx_bytes + (size_t)nch * kr * kRcChunk * 4, 0);
+            uint64_t rows = 0;
+            int a = 0;
+            for (int r = 0; r < 16; ++r)
+              if ((hb.rowmask >> r) & 1u) rows |= (uint64_t)r << (4 * a++);
+            std::memcpy(&rc_blob[rec], &rows, 8);
+            uint8_t cols[64];
+            int n = 0;
+            for (int c = 0; c < 64; ++c)
+              if ((hb.colmask >> c) & 1ull) cols[n++] = (uint8_t)c;
+            for (int c = 0; c < nch * kRcChunk; ++c) rc_blob[rec + 8 + (size_t)c] = cols[c < kc ? c : 0];
+            float* w = reinterpret_cast<float*>(&rc_blob[rec + idx_bytes]);
+            const float* src = &h->vals[(size_t)hb.val_off];
+            for (int c = 0; c < kc; ++c)
+              for (int aa = 0; aa < kr; ++aa)
+                w[((size_t)(c / kRcChunk) * kr + aa) * kRcChunk + (c % kRcChunk)] = src[(size_t)aa * kc + c];
+          }
+          se.bytes = (uint32_t)(rc_blob.size() - start);
+          rc_max = std::max(rc_max, se.bytes);
+        }
+      }
+      if (st != GRIM_OK) { delete h; return st; }
+      h->rc_max_blob = rc_max;
+      h->index_bytes_rc = (int64_t)rc_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)rc_blob.size() - (int64_t)nnz * 4 +
+                          nbr * 4;
+    }
+
     // ---- upload
     if (!(flags & GRIM_PACK_HOST_ONLY)) {
       cudaError_t e = cudaGetDevice(&h->device);
       if (e == cudaSuccess) e = upload(&h->d_stage, stage.data(), stage.size() * sizeof(StageEntry));
       if (e == cudaSuccess) e = upload(&h->d_blob, blob.data(), blob.size());
       if (e == cudaSuccess) e = upload(&h->d_band_order, h->band_order.data(), h->band_order.size() * 4);
+      if (e == cudaSuccess) e = upload(&h->d_rc_stage, rc_stage.data(), rc_stage.size() * sizeof(RcStage));
+      if (e == cudaSuccess) e = upload(&h->d_rc_blob, rc_blob.data(), rc_blob.size());
+      const unsigned zero = 0;
+      if (e == cudaSuccess) e = upload(&h->d_status, &zero, 4);
       if (e == cudaSuccess && h->gemv_ok) {
         e = upload(&h->d_gemv_band_ptr, band_ptr.data(), band_ptr.size() * 4);
         if (e == cudaSuccess) e = upload(&h->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkDesc));
@@ -326,7 +395,7 @@ extern "C" grim_status_t grim_bcr_info(grim_bcr_t h, grim_bcr_info_t* info) {
   info->nnz = h->nnz; info->nonempty_blocks = h->nonempty; info->k_used = h->k_used; info->dtype = h->dtype;
   info->flags = h->flags; info->on_device = h->device >= 0;
   info->value_bytes = h->nnz * (h->dtype == GRIM_BF16 ? 2 : 4);
-  info->index_bytes_spmm = h->index_bytes_spmm;
+  info->index_bytes_spmm = h->index_bytes_rc;
   info->index_bytes_gemv = h->index_bytes_gemv;
   info->export_bytes = export_size(h);
   return GRIM_OK;
@@ -383,4 +452,13 @@ extern "C" grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W, int64_t l
       }
     }
   return GRIM_OK;
+}
+
+extern "C" grim_status_t grim_bcr_status(grim_bcr_t h) {
+  if (!h || h->device < 0 || !h->d_status) return GRIM_ERR_INVALID_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return GRIM_ERR_CUDA;
+  unsigned v = 0;
+  if (cudaMemcpy(&v, h->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GRIM_ERR_CUDA;
+  if (v != 0) cudaMemset(h->d_status, 0, 4);
+  return (grim_status_t)v;
 }

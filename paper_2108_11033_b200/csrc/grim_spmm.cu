@@ -8,9 +8,10 @@
 //                   arrive as one contiguous piece ("blob") through cp.async.  With CONV the slab is
 //                   produced on the fly from the NCHW input (implicit im2col, Section 4.5); rows whose
 //                   column is kept by no block of the group are not read.
-//  bcr_gemv_kernel  N = 1.  A warp owns (part of) a band; a lane owns one kept column of one block, reads
-//                   x[col] once and multiplies it with that column's kr kept values (coalesced across
-//                   lanes), accumulating into per-row registers selected by the block's row mask.
+//  bcr_skinny_kernel  N <= 16 (N = 1: matrix-vector).  A warp owns (part of) a band; a lane owns one kept
+//                   column of one block, reads its activations once and multiplies them with that column's
+//                   kr kept values (coalesced across lanes), accumulating into per-row registers selected
+//                   by the block's row mask.
 #include <cuda_bf16.h>
 
 #include <atomic>
@@ -316,56 +317,119 @@ __global__ void __launch_bounds__(kThreads) bcr_spmm_kernel(const KParams p) {
 }
 
 // ---------------------------------------------------------------------------------------------
-// N = 1
+// N <= 16 ("skinny" right-hand side, N = 1 is the matrix-vector product)
+//
+// A warp owns a contiguous run of a band's chunks, a lane one kept column of a chunk.  The lane reads
+// the NQ activations of its column once and multiplies them with the column's kr kept values, which are
+// read straight from global memory (coalesced across lanes, each value used NQ times) and accumulated
+// into per-row registers selected by the block's row mask.  U chunks are processed per pass so that
+// their loads are in flight together; column words have a fixed place (32 per chunk), so a pass starts
+// with two independent loads (words and value offsets) instead of a dependent chain.
 // ---------------------------------------------------------------------------------------------
-template <int BH, typename VT, typename XT>
-__global__ void __launch_bounds__(kThreads) bcr_gemv_kernel(const uint32_t* __restrict__ band_ptr,
-                                                            const ChunkDesc* __restrict__ chunks,
-                                                            const uint32_t* __restrict__ colwords,
-                                                            const VT* __restrict__ vals,
-                                                            const uint32_t* __restrict__ band_order,
-                                                            const XT* __restrict__ x, float* __restrict__ y32,
-                                                            __nv_bfloat16* __restrict__ y16, int nbr, int M, int bh,
-                                                            int wpb /* warps per band: 1, 2, 4 or 8 */) {
-  __shared__ float part[kWarps][BH];
+struct SkinnyParams {
+  const uint32_t* band_ptr;
+  const ChunkDesc* chunks;
+  const uint32_t* colwords;
+  const void* vals;
+  const uint32_t* band_order;
+  const void* X;
+  void* Y;
+  int64_t ldx, ldy;
+  int N, nbr, M, bh, wpb, y_dtype, vec_ok;
+};
+
+template <int NQ, typename XT>
+__device__ __forceinline__ void load_x_row(const SkinnyParams& p, uint32_t col, int q0, float (&x)[NQ]) {
+  const XT* row = static_cast<const XT*>(p.X) + (int64_t)col * p.ldx + q0;
+  if (NQ >= 4 && p.vec_ok) {
+    if (sizeof(XT) == 4) {
+#pragma unroll
+      for (int i = 0; i < NQ / 4; ++i) {
+        const float4 v = __ldg(reinterpret_cast<const float4*>(row) + i);
+        x[4 * i] = v.x; x[4 * i + 1] = v.y; x[4 * i + 2] = v.z; x[4 * i + 3] = v.w;
+      }
+    } else {
+#pragma unroll
+      for (int i = 0; i < NQ / 4; ++i) {
+        const uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + i);
+        x[4 * i] = __uint_as_float(u.x << 16); x[4 * i + 1] = __uint_as_float(u.x & 0xFFFF0000u);
+        x[4 * i + 2] = __uint_as_float(u.y << 16); x[4 * i + 3] = __uint_as_float(u.y & 0xFFFF0000u);
+      }
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < NQ; ++i) x[i] = (q0 + i < p.N) ? to_f32(row[i]) : 0.f;
+  }
+}
+
+template <int BH, int NQ, int U, typename VT, typename XT>
+__global__ void __launch_bounds__(kThreads) bcr_skinny_kernel(const SkinnyParams p) {
+  __shared__ float part[kWarps][BH][NQ];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int bpc = kWarps / wpb;
+  const int wpb = p.wpb, bpc = kWarps / wpb;
   const int bi = warp / wpb, ks = warp % wpb;
   const int pos = blockIdx.x * bpc + bi;
-  float acc[BH];
+  const int q0 = blockIdx.y * NQ;
+  const VT* __restrict__ vals = static_cast<const VT*>(p.vals);
+  float acc[BH][NQ];
 #pragma unroll
-  for (int r = 0; r < BH; ++r) acc[r] = 0.f;
-  if (pos < nbr) {
-    const uint32_t cbeg = band_ptr[pos], cend = band_ptr[pos + 1];
-    for (uint32_t c = cbeg + ks; c < cend; c += wpb) {
-      const ChunkDesc cd = chunks[c];
-      const int ncols = cd.ncols_kr & 0xFFFF;
-      if (lane < ncols) {
-        const uint32_t cw = __ldg(colwords + cd.cw_off + lane);
-        const unsigned rm = cw >> 16;
-        const float xv = to_f32(x[cw & 0xFFFFu]);
-        const VT* v = vals + cd.val_off + lane;
-        int cnt = 0;
+  for (int r = 0; r < BH; ++r)
 #pragma unroll
-        for (int r = 0; r < BH; ++r) {
-          if ((rm >> r) & 1u) {
-            acc[r] = fmaf(to_f32(v[cnt * ncols]), xv, acc[r]);
-            ++cnt;
+    for (int q = 0; q < NQ; ++q) acc[r][q] = 0.f;
+  if (pos < p.nbr) {
+    const uint32_t cbeg = p.band_ptr[pos], cend = p.band_ptr[pos + 1];
+    const uint32_t per = (cend - cbeg + wpb - 1) / wpb;
+    const uint32_t my_beg = min(cbeg + ks * per, cend), my_end = min(my_beg + per, cend);
+    for (uint32_t base = my_beg; base < my_end; base += U) {
+      uint32_t cw[U], voff[U];
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const uint32_t c = base + u;
+        const bool live = c < my_end;
+        cw[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
+        voff[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+        const unsigned rm = cw[u] >> 16;
+        const int ncols = __popc(__ballot_sync(0xffffffffu, rm != 0));
+        if (rm) {
+          float x[NQ];
+          load_x_row<NQ, XT>(p, cw[u] & 0xFFFFu, q0, x);
+          const VT* v = vals + voff[u] + lane;
+          int cnt = 0;
+#pragma unroll
+          for (int r = 0; r < BH; ++r) {
+            if ((rm >> r) & 1u) {
+              const float w = to_f32(v[cnt * ncols]);
+              ++cnt;
+#pragma unroll
+              for (int q = 0; q < NQ; ++q) acc[r][q] = fmaf(w, x[q], acc[r][q]);
+            }
           }
         }
       }
     }
   }
-  warp_reduce_rows<BH>(acc, lane);
-  part[warp][warp_row<BH>(lane)] = acc[0];  // lanes that share a row hold the same total
+  const int myrow = warp_row<BH>(lane);
+#pragma unroll
+  for (int q = 0; q < NQ; ++q) {
+    float t[BH];
+#pragma unroll
+    for (int r = 0; r < BH; ++r) t[r] = acc[r][q];
+    warp_reduce_rows<BH>(t, lane);
+    part[warp][myrow][q] = t[0];  // lanes that share a row hold the same total
+  }
   __syncthreads();
-  if (pos < nbr && ks == 0 && lane < BH && lane < bh) {
-    float s = 0.f;
-    for (int w = 0; w < wpb; ++w) s += part[bi * wpb + w][lane];
-    const int64_t row = (int64_t)band_order[pos] * bh + lane;
-    if (row < M) {
-      if (y32) y32[row] = s;
-      else y16[row] = __float2bfloat16_rn(s);
+  if (pos < p.nbr && ks == 0) {
+    for (int idx = lane; idx < BH * NQ; idx += 32) {
+      const int r = idx / NQ, q = idx % NQ;
+      const int64_t row = (int64_t)p.band_order[pos] * p.bh + r;
+      if (r >= p.bh || row >= p.M || q0 + q >= p.N) continue;
+      float s = 0.f;
+      for (int w = 0; w < wpb; ++w) s += part[bi * wpb + w][r][q];
+      if (p.y_dtype == GRIM_F32) static_cast<float*>(p.Y)[row * p.ldy + q0 + q] = s;
+      else static_cast<__nv_bfloat16*>(p.Y)[row * p.ldy + q0 + q] = __float2bfloat16_rn(s);
     }
   }
 }
@@ -431,36 +495,55 @@ grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   return e == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
 }
 
-grim_status_t launch_gemv(const grim_bcr* h, const void* x, int x_dtype, float* y32, void* y16, cudaStream_t s) {
-  if (h->device < 0 || !h->gemv_ok) return GRIM_ERR_UNSUPPORTED;
+namespace {
+
+template <int BH, typename VT, typename XT>
+cudaError_t launch_skinny_nq(const SkinnyParams& p, int nq, dim3 grid, cudaStream_t s) {
+  switch (nq) {
+    case 1: bcr_skinny_kernel<BH, 1, 8, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    case 4: bcr_skinny_kernel<BH, 4, 8, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    case 8: bcr_skinny_kernel<BH, 8, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    default:
+      if (BH > 8) return cudaErrorInvalidValue;
+      bcr_skinny_kernel<(BH <= 8 ? BH : 8), 16, 4, VT, XT><<<grid, kThreads, 0, s>>>(p);
+  }
+  return cudaGetLastError();
+}
+
+template <typename VT, typename XT>
+cudaError_t launch_skinny_bh(const SkinnyParams& p, int BHc, int nq, dim3 grid, cudaStream_t s) {
+  if (BHc == 4) return launch_skinny_nq<4, VT, XT>(p, nq, grid, s);
+  if (BHc == 8) return launch_skinny_nq<8, VT, XT>(p, nq, grid, s);
+  return launch_skinny_nq<16, VT, XT>(p, nq, grid, s);
+}
+
+}  // namespace
+
+grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
+                            int64_t ldy, cudaStream_t s) {
+  if (h->device < 0 || !h->gemv_ok || N < 1 || N > kSkinnyMaxN) return GRIM_ERR_UNSUPPORTED;
+  if (x_dtype != h->dtype) return GRIM_ERR_DTYPE;
   const int nbr = (int)h->nbr;
+  const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);
+  int nq = N == 1 ? 1 : (N <= 4 ? 4 : (N <= 8 ? 8 : 16));
+  if (BHc == 16 && nq == 16) nq = 8;  // 16 x 16 accumulators do not fit the register file: two passes of 8
+  const int passes = (int)((N + nq - 1) / nq);
   // enough warps to keep every SM's memory pipeline busy: split a band over several warps when bands are few
   int wpb = 1;
-  const int64_t want_warps = 148 * 24;
-  while (wpb < 8 && (int64_t)nbr * wpb < want_warps && (int64_t)nbr * wpb * 2 <= h->nchunks) wpb *= 2;
+  const int64_t want_warps = 148 * 16;
+  while (wpb < 8 && (int64_t)nbr * passes * wpb < want_warps && (int64_t)nbr * wpb * 4 <= h->nchunks) wpb *= 2;
   const int bpc = kWarps / wpb;
-  const int grid = (nbr + bpc - 1) / bpc;
-  const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);
-  auto* y16p = static_cast<__nv_bfloat16*>(y16);
-#define GEMV_LAUNCH(BHV, VT, XT)                                                                               \
-  bcr_gemv_kernel<BHV, VT, XT><<<grid, kThreads, 0, s>>>(h->d_gemv_band_ptr, h->d_chunks, h->d_colwords,       \
-                                                         static_cast<const VT*>(h->d_gemv_vals), h->d_band_order, \
-                                                         static_cast<const XT*>(x), y32, y16p, nbr, (int)h->M,  \
-                                                         h->bh, wpb)
-  if (h->dtype == GRIM_F32) {
-    if (x_dtype != GRIM_F32) return GRIM_ERR_DTYPE;
-    if (BHc == 4) GEMV_LAUNCH(4, float, float);
-    else if (BHc == 8) GEMV_LAUNCH(8, float, float);
-    else GEMV_LAUNCH(16, float, float);
-  } else {
-    if (x_dtype != GRIM_BF16) return GRIM_ERR_DTYPE;
-    if (BHc == 4) GEMV_LAUNCH(4, __nv_bfloat16, __nv_bfloat16);
-    else if (BHc == 8) GEMV_LAUNCH(8, __nv_bfloat16, __nv_bfloat16);
-    else GEMV_LAUNCH(16, __nv_bfloat16, __nv_bfloat16);
-  }
-#undef GEMV_LAUNCH
+  SkinnyParams p;
+  p.band_ptr = h->d_gemv_band_ptr; p.chunks = h->d_chunks; p.colwords = h->d_colwords; p.vals = h->d_gemv_vals;
+  p.band_order = h->d_band_order; p.X = X; p.Y = Y; p.ldx = ldx; p.ldy = ldy;
+  p.N = (int)N; p.nbr = nbr; p.M = (int)h->M; p.bh = h->bh; p.wpb = wpb; p.y_dtype = y_dtype;
+  const int esz = x_dtype == GRIM_F32 ? 4 : 2;
+  p.vec_ok = (N % nq == 0) && ldx % 4 == 0 && (reinterpret_cast<uintptr_t>(X) % (4 * esz)) == 0;
+  dim3 grid((unsigned)((nbr + bpc - 1) / bpc), (unsigned)passes);
+  cudaError_t e = h->dtype == GRIM_F32 ? launch_skinny_bh<float, float>(p, BHc, nq, grid, s)
+                                       : launch_skinny_bh<__nv_bfloat16, __nv_bfloat16>(p, BHc, nq, grid, s);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+  return e == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
 }
 
 }  // namespace grim
