@@ -108,17 +108,11 @@ __device__ __forceinline__ float4 ld_x4(const __nv_bfloat16* slab, unsigned col,
   A.y = fmaf(W, X.y, A.y);          \
   A.z = fmaf(W, X.z, A.z);          \
   A.w = fmaf(W, X.w, A.w);
-#define GRIM_ROW_CASE(R)                                   \
-  case R: {                                                \
-    if (R < BH) {                                          \
-      float4& A = acc[b][R < BH ? R : 0];                  \
-      GRIM_FMA4(A, w0.x, x[0]) GRIM_FMA4(A, w0.y, x[1])    \
-      GRIM_FMA4(A, w0.z, x[2]) GRIM_FMA4(A, w0.w, x[3])    \
-      GRIM_FMA4(A, w1.x, x[4]) GRIM_FMA4(A, w1.y, x[5])    \
-      GRIM_FMA4(A, w1.z, x[6]) GRIM_FMA4(A, w1.w, x[7])    \
-    }                                                      \
-    break;                                                 \
-  }
+#define GRIM_ROW_FMA(A)                                \
+  GRIM_FMA4(A, w0.x, x[0]) GRIM_FMA4(A, w0.y, x[1])    \
+  GRIM_FMA4(A, w0.z, x[2]) GRIM_FMA4(A, w0.w, x[3])    \
+  GRIM_FMA4(A, w1.x, x[4]) GRIM_FMA4(A, w1.y, x[5])    \
+  GRIM_FMA4(A, w1.z, x[6]) GRIM_FMA4(A, w1.w, x[7])
 
 template <int BH, int BPW, typename XT, int MODE>
 __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_constant__ CUtensorMap tmX, const FParams p) {
@@ -285,7 +279,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
       const int kr = (hdr >> 16) & 0xFF, nch = hdr >> 24;
       if (kr == 0) continue;
       const uint8_t* rec = blob + (hdr & 0xFFFFu) * 16;
-      const unsigned long long rows = *reinterpret_cast<const unsigned long long*>(rec);
+      const unsigned rm = *reinterpret_cast<const unsigned*>(rec);  // kept rows of this block (same for the whole warp)
       const uint8_t* cols = rec + 8;
       const float4* wp = reinterpret_cast<const float4*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
       for (int ch = 0; ch < nch; ++ch) {
@@ -299,17 +293,13 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
         x[5] = ld_x4(slab, (cc.y >> 8) & 0xFFu, lane);
         x[6] = ld_x4(slab, (cc.y >> 16) & 0xFFu, lane);
         x[7] = ld_x4(slab, cc.y >> 24, lane);
-        unsigned long long rr = rows;
-        for (int ai = 0; ai < kr; ++ai) {
-          const float4 w0 = wp[0], w1 = wp[1];
-          wp += 2;
-          const unsigned r = (unsigned)rr & 15u;
-          rr >>= 4;
-          switch (r) {
-            GRIM_ROW_CASE(0) GRIM_ROW_CASE(1) GRIM_ROW_CASE(2) GRIM_ROW_CASE(3)
-            GRIM_ROW_CASE(4) GRIM_ROW_CASE(5) GRIM_ROW_CASE(6) GRIM_ROW_CASE(7)
-            GRIM_ROW_CASE(8) GRIM_ROW_CASE(9) GRIM_ROW_CASE(10) GRIM_ROW_CASE(11)
-            GRIM_ROW_CASE(12) GRIM_ROW_CASE(13) GRIM_ROW_CASE(14) GRIM_ROW_CASE(15)
+        // one test per row of the band; a kept row consumes the next eight weights
+#pragma unroll
+        for (int r = 0; r < BH; ++r) {
+          if ((rm >> r) & 1u) {
+            const float4 w0 = wp[0], w1 = wp[1];
+            wp += 2;
+            GRIM_ROW_FMA(acc[b][r])
           }
         }
       }

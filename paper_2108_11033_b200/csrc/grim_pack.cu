@@ -310,10 +310,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
             std::memcpy(&rc_blob[start + (size_t)b * 4], &hdr, 4);
             const size_t idx_bytes = ((size_t)8 + (size_t)nch * kRcChunk + 15) / 16 * 16;
             rc_blob.resize(rec + idx_bytes + (size_t)nch * kr * kRcChunk * 4, 0);
-            uint64_t rows = 0;
-            int a = 0;
-            for (int r = 0; r < 16; ++r)
-              if ((hb.rowmask >> r) & 1u) rows |= (uint64_t)r << (4 * a++);
+            const uint64_t rows = hb.rowmask;  // bit r: block-local row r kept
             std::memcpy(&rc_blob[rec], &rows, 8);
             uint8_t cols[64];
             int n = 0;

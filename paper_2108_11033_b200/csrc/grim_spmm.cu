@@ -380,14 +380,25 @@ __global__ void __launch_bounds__(kThreads) bcr_skinny_kernel(const SkinnyParams
     const uint32_t cbeg = p.band_ptr[pos], cend = p.band_ptr[pos + 1];
     const uint32_t per = (cend - cbeg + wpb - 1) / wpb;
     const uint32_t my_beg = min(cbeg + ks * per, cend), my_end = min(my_beg + per, cend);
+    // column words and value offsets of a pass are requested one pass ahead of their use
+    uint32_t cw_n[U], voff_n[U];
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+      const uint32_t c = my_beg + u;
+      const bool live = c < my_end;
+      cw_n[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
+      voff_n[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
+    }
     for (uint32_t base = my_beg; base < my_end; base += U) {
       uint32_t cw[U], voff[U];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
-        const uint32_t c = base + u;
+        cw[u] = cw_n[u];
+        voff[u] = voff_n[u];
+        const uint32_t c = base + U + u;
         const bool live = c < my_end;
-        cw[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
-        voff[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
+        cw_n[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
+        voff_n[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
       }
 #pragma unroll
       for (int u = 0; u < U; ++u) {
@@ -500,8 +511,8 @@ namespace {
 template <int BH, typename VT, typename XT>
 cudaError_t launch_skinny_nq(const SkinnyParams& p, int nq, dim3 grid, cudaStream_t s) {
   switch (nq) {
-    case 1: bcr_skinny_kernel<BH, 1, 8, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
-    case 4: bcr_skinny_kernel<BH, 4, 8, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    case 1: bcr_skinny_kernel<BH, 1, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    case 4: bcr_skinny_kernel<BH, 4, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
     case 8: bcr_skinny_kernel<BH, 8, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
     default:
       if (BH > 8) return cudaErrorInvalidValue;
@@ -530,8 +541,8 @@ grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64
   const int passes = (int)((N + nq - 1) / nq);
   // enough warps to keep every SM's memory pipeline busy: split a band over several warps when bands are few
   int wpb = 1;
-  const int64_t want_warps = 148 * 16;
-  while (wpb < 8 && (int64_t)nbr * passes * wpb < want_warps && (int64_t)nbr * wpb * 4 <= h->nchunks) wpb *= 2;
+  const int64_t want_warps = 148 * 20;
+  while (wpb < 8 && (int64_t)nbr * passes * wpb < want_warps && (int64_t)nbr * wpb * 8 <= h->nchunks) wpb *= 2;
   const int bpc = kWarps / wpb;
   SkinnyParams p;
   p.band_ptr = h->d_gemv_band_ptr; p.chunks = h->d_chunks; p.colwords = h->d_colwords; p.vals = h->d_gemv_vals;
