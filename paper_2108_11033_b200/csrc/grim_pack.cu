@@ -266,6 +266,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
           }
         }
       }
+      gvals.resize(gvals.size() + 64 * vsz, 0);  // the kernels may read (and discard) up to a warp's width past a chunk
       band_ptr[(size_t)nbr] = (uint32_t)chunks.size();
       h->nchunks = (int64_t)chunks.size();
       h->h_gemv_band_ptr = band_ptr;

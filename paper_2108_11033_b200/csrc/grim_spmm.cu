@@ -378,45 +378,62 @@ __global__ void __launch_bounds__(kThreads) bcr_skinny_kernel(const SkinnyParams
     for (int q = 0; q < NQ; ++q) acc[r][q] = 0.f;
   if (pos < p.nbr) {
     const uint32_t cbeg = p.band_ptr[pos], cend = p.band_ptr[pos + 1];
-    const uint32_t per = (cend - cbeg + wpb - 1) / wpb;
-    const uint32_t my_beg = min(cbeg + ks * per, cend), my_end = min(my_beg + per, cend);
+    // warp ks takes chunks cbeg + ks, cbeg + ks + wpb, ...: chunks are sorted by kept-row count, so a strided
+    // share gives every warp of the band the same mix of heavy and light chunks
+    const uint32_t my_beg = cbeg + ks, my_end = cend;
     // column words and value offsets of a pass are requested one pass ahead of their use
     uint32_t cw_n[U], voff_n[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const uint32_t c = my_beg + u;
+      const uint32_t c = my_beg + u * wpb;
       const bool live = c < my_end;
       cw_n[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
       voff_n[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
     }
-    for (uint32_t base = my_beg; base < my_end; base += U) {
+    for (uint32_t base = my_beg; base < my_end; base += U * wpb) {
       uint32_t cw[U], voff[U];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         cw[u] = cw_n[u];
         voff[u] = voff_n[u];
-        const uint32_t c = base + U + u;
+        const uint32_t c = base + (U + u) * wpb;
         const bool live = c < my_end;
         cw_n[u] = live ? __ldg(p.colwords + (size_t)c * 32 + lane) : 0u;
         voff_n[u] = live ? __ldg(&p.chunks[c].val_off) : 0u;
       }
+      // all loads of the pass first (values land in their row's slot, 0 for rows the block does not keep),
+      // so that they are in flight together; the multiplies follow
+      float w[U][BH], x[U][NQ];
 #pragma unroll
       for (int u = 0; u < U; ++u) {
         const unsigned rm = cw[u] >> 16;
         const int ncols = __popc(__ballot_sync(0xffffffffu, rm != 0));
-        if (rm) {
-          float x[NQ];
-          load_x_row<NQ, XT>(p, cw[u] & 0xFFFFu, q0, x);
-          const VT* v = vals + voff[u] + lane;
-          int cnt = 0;
+        if (rm) load_x_row<NQ, XT>(p, cw[u] & 0xFFFFu, q0, x[u]);
+        else {
 #pragma unroll
-          for (int r = 0; r < BH; ++r) {
-            if ((rm >> r) & 1u) {
-              const float w = to_f32(v[cnt * ncols]);
-              ++cnt;
+          for (int q = 0; q < NQ; ++q) x[u][q] = 0.f;
+        }
+        const VT* v = vals + voff[u] + lane;
+        int cnt = 0;
 #pragma unroll
-              for (int q = 0; q < NQ; ++q) acc[r][q] = fmaf(w, x[q], acc[r][q]);
-            }
+        for (int r = 0; r < BH; ++r) {
+          // unconditional load (a pruned row re-reads the chunk's first line) + select: no branch, so every
+          // load of the pass is issued before the first use
+          const bool kept = (rm >> r) & 1u;
+          const float val = to_f32(v[kept ? cnt * ncols : 0]);
+          w[u][r] = kept ? val : 0.f;
+          cnt += kept ? 1 : 0;
+        }
+      }
+#pragma unroll
+      for (int u = 0; u < U; ++u) {
+#pragma unroll
+        for (int r = 0; r < BH; ++r) {
+          if (NQ == 1) {
+            acc[r][0] = fmaf(w[u][r], x[u][0], acc[r][0]);
+          } else if ((cw[u] >> (16 + r)) & 1u) {
+#pragma unroll
+            for (int q = 0; q < NQ; ++q) acc[r][q] = fmaf(w[u][r], x[u][q], acc[r][q]);
           }
         }
       }
@@ -513,10 +530,10 @@ cudaError_t launch_skinny_nq(const SkinnyParams& p, int nq, dim3 grid, cudaStrea
   switch (nq) {
     case 1: bcr_skinny_kernel<BH, 1, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
     case 4: bcr_skinny_kernel<BH, 4, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
-    case 8: bcr_skinny_kernel<BH, 8, 4, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
+    case 8: bcr_skinny_kernel<BH, 8, 2, VT, XT><<<grid, kThreads, 0, s>>>(p); break;
     default:
       if (BH > 8) return cudaErrorInvalidValue;
-      bcr_skinny_kernel<(BH <= 8 ? BH : 8), 16, 4, VT, XT><<<grid, kThreads, 0, s>>>(p);
+      bcr_skinny_kernel<(BH <= 8 ? BH : 8), 16, 2, VT, XT><<<grid, kThreads, 0, s>>>(p);
   }
   return cudaGetLastError();
 }
