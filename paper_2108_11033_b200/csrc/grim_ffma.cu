@@ -41,6 +41,8 @@ struct FParams {
   int nbr, nbc, M, K, bh, bw, ngroups;
   uint32_t blob_stride, slab_bytes;
   unsigned spin_limit;
+  int slab_ld;  // floats between slab rows: kTN, or kTN + 4 when the gather writes down the columns (X stored q-major)
+  int ksplit;  // > 1: blockIdx.z takes a share of the block columns and adds its partial sums into a zeroed Y
   SpmmArgs a;
 };
 
@@ -94,11 +96,11 @@ __device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
   asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
-__device__ __forceinline__ float4 ld_x4(const float* slab, unsigned col, int lane) {
-  return *reinterpret_cast<const float4*>(slab + col * kTN + lane * 4);
+__device__ __forceinline__ float4 ld_x4(const float* slab, unsigned col, int lane, int sld) {
+  return *reinterpret_cast<const float4*>(slab + col * sld + lane * 4);
 }
-__device__ __forceinline__ float4 ld_x4(const __nv_bfloat16* slab, unsigned col, int lane) {
-  const uint2 u = *reinterpret_cast<const uint2*>(slab + col * kTN + lane * 4);
+__device__ __forceinline__ float4 ld_x4(const __nv_bfloat16* slab, unsigned col, int lane, int sld) {
+  const uint2 u = *reinterpret_cast<const uint2*>(slab + col * sld + lane * 4);
   return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16),
                      __uint_as_float(u.y & 0xFFFF0000u));
 }
@@ -122,11 +124,15 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 64);
   int* s_nst = reinterpret_cast<int*>(smem + 68);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 128);               // [kStages][4] blob bytes per band group
-  uint16_t* jlist = reinterpret_cast<uint16_t*>(smem + 128 + kStages * 16);  // non-empty block columns, ascending
+  const uint16_t* jlist = reinterpret_cast<const uint16_t*>(smem + 128 + kStages * 16);  // non-empty block columns, ascending
   uint8_t* slots = smem + kHdrBytes;
   const uint32_t slot_bytes = p.slab_bytes + BPW * p.blob_stride;
+  const int sld = MODE == kModeTma ? kTN : p.slab_ld;
 
-  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int tid = threadIdx.x, lane = tid & 31;
+  // broadcast from lane 0 so that the compiler knows the warp index (and all that derives from it) is the same
+  // in every lane: branches on the band's header and row mask then need no divergence handling
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   const SpmmArgs& a = p.a;
   const int64_t q0 = (int64_t)blockIdx.x * kTN;
   const int g0 = blockIdx.y * BPW;
@@ -140,7 +146,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
         for (int b = 0; b < BPW; ++b)
           if (g0 + b < p.ngroups) f = f || p.stage[(int64_t)(g0 + b) * p.nbc + j].bytes != 0;
       const unsigned m = __ballot_sync(0xffffffffu, f);
-      if (f) jlist[n + __popc(m & ((1u << lane) - 1u))] = (uint16_t)j;
+      if (f) const_cast<uint16_t*>(jlist)[n + __popc(m & ((1u << lane) - 1u))] = (uint16_t)j;
       n += __popc(m);
     }
     if (lane == 0) {
@@ -154,7 +160,11 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
     }
   }
   __syncthreads();
-  const int nst = *s_nst;
+  // with a split over block columns this thread block multiplies only its share of the stage list
+  const int nst_all = *s_nst;
+  const int n_lo = (int)((int64_t)blockIdx.z * nst_all / p.ksplit), n_hi = (int)((int64_t)(blockIdx.z + 1) * nst_all / p.ksplit);
+  const int nst = n_hi - n_lo;
+  jlist += n_lo;
 
   // per-thread constants of the gather loader: this thread always fills column qq of the slab
   const int qq = tid & (kTN - 1);
@@ -214,15 +224,24 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
           const int ih = ih0 + kh, iw = iw0 + kw;
           const bool ok = q_ok && k < p.K && ih >= 0 && ih < a.H && iw >= 0 && iw < a.W;
           const float* src = ok ? X + qoff + ((int64_t)c * a.H + kh) * a.W + kw : X;
-          cp_async4_zfill(slab + kk * kTN + qq, src, ok);
+          cp_async4_zfill(slab + kk * sld + qq, src, ok);
           kw += 4;
           while (kw >= a.KW) { kw -= a.KW; ++kh; }
           while (kh >= a.KH) { kh -= a.KH; ++c; }
         }
-      } else {
+      } else if (a.x_sq == 1) {
         for (int kk = kk0; kk < p.bw; kk += 4, k += 4) {
           const bool ok = q_ok && k < p.K;
-          cp_async4_zfill(slab + kk * kTN + qq, ok ? X + k * a.x_sk + qoff : X, ok);
+          cp_async4_zfill(slab + kk * sld + qq, ok ? X + k * a.x_sk + qoff : X, ok);
+        }
+      } else {
+        // X stored q-major: consecutive threads take consecutive k so that the reads coalesce; the padded row
+        // stride keeps the column-wise shared-memory writes to a few bank conflicts
+        for (int e = tid; e < p.bw * kTN; e += kFThreads) {
+          const int kk = e % p.bw, qe = e / p.bw;
+          const int64_t ke = (int64_t)j * p.bw + kk, q = q0 + qe;
+          const bool ok = q < a.ncols && ke < p.K;
+          cp_async4_zfill(slab + kk * sld + qe, ok ? X + ke * a.x_sk + q * a.x_sq : X, ok);
         }
       }
 #pragma unroll
@@ -275,24 +294,24 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
     for (int b = 0; b < BPW; ++b) {
       if (s_meta[slot * 4 + b] == 0) continue;
       const uint8_t* blob = base + p.slab_bytes + b * p.blob_stride;
-      const uint32_t hdr = reinterpret_cast<const uint32_t*>(blob)[warp];
+      const uint32_t hdr = __shfl_sync(0xffffffffu, reinterpret_cast<const uint32_t*>(blob)[warp], 0);
       const int kr = (hdr >> 16) & 0xFF, nch = hdr >> 24;
       if (kr == 0) continue;
       const uint8_t* rec = blob + (hdr & 0xFFFFu) * 16;
-      const unsigned rm = *reinterpret_cast<const unsigned*>(rec);  // kept rows of this block (same for the whole warp)
+      const unsigned rm = __shfl_sync(0xffffffffu, *reinterpret_cast<const unsigned*>(rec), 0);  // kept rows of this block
       const uint8_t* cols = rec + 8;
       const float4* wp = reinterpret_cast<const float4*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
       for (int ch = 0; ch < nch; ++ch) {
         const uint2 cc = *reinterpret_cast<const uint2*>(cols + ch * kRcChunk);
         float4 x[kRcChunk];
-        x[0] = ld_x4(slab, cc.x & 0xFFu, lane);
-        x[1] = ld_x4(slab, (cc.x >> 8) & 0xFFu, lane);
-        x[2] = ld_x4(slab, (cc.x >> 16) & 0xFFu, lane);
-        x[3] = ld_x4(slab, cc.x >> 24, lane);
-        x[4] = ld_x4(slab, cc.y & 0xFFu, lane);
-        x[5] = ld_x4(slab, (cc.y >> 8) & 0xFFu, lane);
-        x[6] = ld_x4(slab, (cc.y >> 16) & 0xFFu, lane);
-        x[7] = ld_x4(slab, cc.y >> 24, lane);
+        x[0] = ld_x4(slab, cc.x & 0xFFu, lane, sld);
+        x[1] = ld_x4(slab, (cc.x >> 8) & 0xFFu, lane, sld);
+        x[2] = ld_x4(slab, (cc.x >> 16) & 0xFFu, lane, sld);
+        x[3] = ld_x4(slab, cc.x >> 24, lane, sld);
+        x[4] = ld_x4(slab, cc.y & 0xFFu, lane, sld);
+        x[5] = ld_x4(slab, (cc.y >> 8) & 0xFFu, lane, sld);
+        x[6] = ld_x4(slab, (cc.y >> 16) & 0xFFu, lane, sld);
+        x[7] = ld_x4(slab, cc.y >> 24, lane, sld);
         // one test per row of the band; a kept row consumes the next eight weights
 #pragma unroll
         for (int r = 0; r < BH; ++r) {
@@ -335,6 +354,24 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
       const int64_t row = (int64_t)band * p.bh + r;
       if (r >= p.bh || row >= p.M) continue;
       float t[4] = {acc[b][r].x, acc[b][r].y, acc[b][r].z, acc[b][r].w};
+      if (p.ksplit > 1) {
+        // partial sums of one share of the block columns: added into Y (fp32, zeroed before the launch);
+        // bias and activation follow in a separate pass
+        float* y = static_cast<float*>(a.Y);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          if (q + e >= a.ncols) break;
+          int64_t off;
+          if (a.conv) {
+            const int64_t img = (q + e) / ohw;
+            off = (img * p.M + row) * ohw + ((q + e) - img * ohw);
+          } else {
+            off = row * a.y_sr + (q + e) * a.y_sq;
+          }
+          if (t[e] != 0.f) atomicAdd(y + off, t[e]);
+        }
+        continue;
+      }
       const float bias = a.bias ? __ldg(a.bias + row) : 0.f;
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
@@ -407,10 +444,43 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
+// Second pass of a split multiply: Y = act(Y + bias) in place.
+__global__ void bcr_finalize_kernel(const SpmmArgs a, int M) {
+  const int64_t total = (int64_t)M * a.ncols;
+  const int64_t ohw = (int64_t)a.OH * a.OW;
+  float* y = static_cast<float*>(a.Y);
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    int64_t off, row;
+    if (a.conv) {  // i runs over the NCHW output
+      off = i;
+      row = (i / ohw) % M;
+    } else if (a.y_sq == 1) {
+      row = i / a.ncols;
+      off = row * a.y_sr + (i - row * a.ncols);
+    } else {
+      const int64_t q = i / M;
+      row = i - q * M;
+      off = row * a.y_sr + q * a.y_sq;
+    }
+    float v = y[off] + (a.bias ? __ldg(a.bias + row) : 0.f);
+    if (a.relu) v = fmaxf(v, 0.f);
+    y[off] = v;
+  }
+}
+
 bool tma_eligible(const SpmmArgs& a) {
   if (a.conv || a.x_sq != 1) return false;
   const int esz = a.x_dtype == GRIM_F32 ? 4 : 2;
   return (reinterpret_cast<uintptr_t>(a.X) % 16 == 0) && ((a.x_sk * esz) % 16 == 0) && a.ncols < (int64_t(1) << 31);
+}
+
+// Zeroes the M x ncols region of Y that a split multiply accumulates into.
+cudaError_t zero_output(const SpmmArgs& a, int64_t M, cudaStream_t s) {
+  float* y = static_cast<float*>(a.Y);
+  if (a.conv) return cudaMemsetAsync(y, 0, (size_t)M * a.ncols * 4, s);
+  if (a.y_sq == 1) return cudaMemset2DAsync(y, (size_t)a.y_sr * 4, 0, (size_t)a.ncols * 4, (size_t)M, s);
+  if (a.y_sr == 1) return cudaMemset2DAsync(y, (size_t)a.y_sq * 4, 0, (size_t)M * 4, (size_t)a.ncols, s);
+  return cudaErrorInvalidValue;
 }
 
 template <int BH, int BPW, typename XT, int MODE>
@@ -438,9 +508,11 @@ cudaError_t launch_bh(int BHc, int bpw, const CUtensorMap& tm, const FParams& p,
 
 constexpr size_t kSmemBudget = 220 * 1024;
 
-size_t smem_need(const grim_bcr* h, int bpw, int esz) {
+int slab_ld_for(const SpmmArgs& a, bool tma) { return (!tma && !a.conv && a.x_sq != 1) ? kTN + 4 : kTN; }
+size_t slab_bytes_for(const grim_bcr* h, int sld, int esz) { return ((size_t)h->bw * sld * esz + 127) & ~size_t(127); }
+size_t smem_need(const grim_bcr* h, int bpw, int esz, int sld = kTN + 4) {
   const size_t blob_stride = ((size_t)h->rc_max_blob + 127) & ~size_t(127);
-  return kHdrBytes + (size_t)kStages * ((size_t)h->bw * kTN * esz + bpw * blob_stride);
+  return kHdrBytes + (size_t)kStages * (slab_bytes_for(h, sld, esz) + bpw * blob_stride);
 }
 
 }  // namespace
@@ -451,7 +523,6 @@ bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTN) return false;
   const bool tma = tma_eligible(a);
   if (!tma && a.x_dtype != GRIM_F32) return false;  // the gather loader moves 4-byte elements
-  if ((h->bw * kTN * (a.x_dtype == GRIM_F32 ? 4 : 2)) % 128 != 0) return false;
   return smem_need(h, 1, a.x_dtype == GRIM_F32 ? 4 : 2) <= kSmemBudget;
 }
 
@@ -464,18 +535,29 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   // band groups per thread block: as many as the accumulators allow, fewer when the grid would not fill the GPU
   int bpw = BHc == 4 ? 4 : (BHc == 8 ? 2 : 1);
   while (bpw > 1 && (smem_need(h, bpw, esz) > kSmemBudget || qtiles * ((h->rc_groups + bpw - 1) / bpw) < 148)) bpw >>= 1;
-  if (a.tile_n == 1 || a.tile_n == 2 || a.tile_n == 4) bpw = std::min(a.tile_n, BHc == 4 ? 4 : (BHc == 8 ? 2 : 1));
+  const int tn = a.tile_n % 256;
+  if (tn == 1 || tn == 2 || tn == 4) bpw = std::min(tn, BHc == 4 ? 4 : (BHc == 8 ? 2 : 1));
   if (smem_need(h, bpw, esz) > kSmemBudget) return GRIM_ERR_UNSUPPORTED;
   const int64_t gy = (h->rc_groups + bpw - 1) / bpw;
   if (gy > 65535) return GRIM_ERR_UNSUPPORTED;
+  // too few tiles for the GPU: split the block columns over several thread blocks (fp32 output only)
+  int ksplit = 1;
+  const bool split_ok = a.y_dtype == GRIM_F32 && (a.conv || a.y_sq == 1 || a.y_sr == 1);
+  if (split_ok && qtiles * gy * 2 <= 148) {
+    ksplit = (int)std::min<int64_t>(std::min<int64_t>(8, 148 / (qtiles * gy)), std::max<int64_t>(1, h->nbc / 4));
+    if (ksplit < 1) ksplit = 1;
+  }
+  if (a.tile_n >= 256) ksplit = split_ok ? std::max(1, std::min(8, a.tile_n / 256)) : 1;  // test / tuning override
 
   FParams p;
   p.stage = h->d_rc_stage; p.blob = h->d_rc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
   p.nbr = (int)h->nbr; p.nbc = (int)h->nbc; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.bw = h->bw;
   p.ngroups = (int)h->rc_groups;
   p.blob_stride = (h->rc_max_blob + 127u) & ~127u;
-  p.slab_bytes = (uint32_t)(h->bw * kTN * esz);
+  p.slab_ld = slab_ld_for(a, tma);
+  p.slab_bytes = (uint32_t)slab_bytes_for(h, p.slab_ld, esz);
   p.spin_limit = 1u << 20;
+  p.ksplit = ksplit;
   p.a = a;
 
   CUtensorMap tm;
@@ -493,9 +575,13 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
                                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return GRIM_ERR_CUDA;
   }
-  const size_t smem = smem_need(h, bpw, esz);
-  dim3 grid((unsigned)qtiles, (unsigned)gy);
-  cudaError_t e;
+  const size_t smem = smem_need(h, bpw, esz, p.slab_ld);
+  dim3 grid((unsigned)qtiles, (unsigned)gy, (unsigned)ksplit);
+  cudaError_t e = cudaSuccess;
+  if (ksplit > 1) {
+    e = zero_output(a, h->M, s);
+    if (e != cudaSuccess) return GRIM_ERR_CUDA;
+  }
   if (tma) {
     e = esz == 4 ? launch_bh<float, kModeTma>(BHc, bpw, tm, p, smem, grid, s)
                  : launch_bh<__nv_bfloat16, kModeTma>(BHc, bpw, tm, p, smem, grid, s);
@@ -503,6 +589,12 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
     e = launch_bh<float, kModeGather>(BHc, bpw, tm, p, smem, grid, s);
   }
   count_launch();
+  if (e == cudaSuccess && ksplit > 1 && (a.bias || a.relu)) {
+    const int64_t total = h->M * a.ncols;
+    bcr_finalize_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8), 256, 0, s>>>(a, (int)h->M);
+    count_launch();
+    e = cudaGetLastError();
+  }
   return e == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
 }
 

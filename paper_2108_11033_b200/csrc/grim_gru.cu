@@ -721,7 +721,7 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     a.x_sk = 1; a.x_sq = wi->K; a.y_sr = 1; a.y_sq = 3 * H;
     a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32; a.bias = g->d_bih[l];
     if (g->profile) cudaEventRecord(g->ev[3 * l], s);
-    grim_status_t st = launch_spmm(wi, a, s);
+    grim_status_t st = ffma_path_supported(wi, a) ? launch_ffma(wi, a, s) : launch_spmm(wi, a, s);
     if (st != GRIM_OK) return st;
     if (g->profile) cudaEventRecord(g->ev[3 * l + 1], s);
     float* seq_out = (l == g->L - 1) ? y : g->d_seq[l & 1];

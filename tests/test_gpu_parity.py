@@ -136,6 +136,25 @@ def test_register_tiled_kernel_explicit(B, case, bf16):
     check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=groups, path=1, flags=1)
 
 
+@pytest.mark.parametrize("split", [2, 5, 8])
+def test_split_multiply(B, split):
+    """Few output tiles: several thread blocks share a tile's block columns and add their partial sums into a
+    zeroed Y (pruned rows must stay exactly +0)."""
+    M, K, bh, bw = 160, 2100, 8, 32
+    W = gen.dense_weight(M, K, seed=83)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=8, dist="uniform", seed=84, empty_frac=0.2)
+    mask[16:24] = 0
+    X = gen.normal_f32((K, 200), 1.0, 85, 0)
+    check_spmm(B, W, mask, X, bh, bw, path=1, tile_n=1 + 256 * split)
+
+
+def test_conv_split_with_bias_and_relu(B):
+    """A layer with few output pixels and many input channels takes the split path (separate bias / ReLU pass)."""
+    L = gen.conv_layer(1, 96, 48, 9, ksize=3, bh=8, bw=32, compression=4, seed=86)
+    check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=False)
+    check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=False, relu=False)
+
+
 @pytest.mark.parametrize("N", [2, 7, 12, 16])
 def test_lane_per_column_kernel_explicit(B, N):
     M, K, bh, bw = 200, 333, 16, 64

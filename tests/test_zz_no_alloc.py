@@ -46,10 +46,16 @@ def test_static_scratch_gru_matches_allocating_entry_point(B):
             assert B.grim_gru_status(g) == B.GRIM_OK
             y = torch.full((T, H), float("nan"), device="cuda")
             hT = torch.full((L, H), float("nan"), device="cuda")
-            before = torch.cuda.memory_allocated()
+            # nothing may be allocated during the call: neither through torch's allocator (its running count of
+            # allocations must not move; frees by Python's garbage collector do not matter) nor from the driver
+            # (the device's free memory must not shrink)
+            torch.cuda.synchronize()
+            allocs_before = torch.cuda.memory_stats().get("allocation.all.allocated", 0)
+            free_before = torch.cuda.mem_get_info()[0]
             B.grim_gru_seq_static(g, x, y, h0=h, hT=hT)
             assert B.grim_gru_status(g) == B.GRIM_OK
-            assert torch.cuda.memory_allocated() == before
+            assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
+            assert torch.cuda.mem_get_info()[0] >= free_before
             assert _rel(y, y_ref) <= 1e-5 and _rel(hT, hT_ref) <= 1e-5
         # a request that does not fit the 8 MiB array is refused on the host, before any launch
         big_T = 5000
