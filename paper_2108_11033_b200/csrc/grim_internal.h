@@ -54,7 +54,7 @@ struct ChunkDesc {
 // j one contiguous blob:
 //   u32 hdr[kRcBands]     per band slot: record offset in 16-byte units | kr << 16 | nch << 24
 //   per band with kr > 0, 16-byte aligned:
-//     u64 rows            bit r set: block-local row r kept (kept rows are numbered a = 0.. in ascending order)
+//     u32 rowmask, u32 kc bit r of rowmask set: block-local row r kept (kept rows are numbered a = 0.. ascending)
 //     u8  cols[nch * 8]   block-local kept columns, padded to a multiple of 8 by repeating the
 //                         first kept column (its padded weights are 0); then padding to 16 bytes
 //     f32 w[nch][kr][8]   w[c][a][e] = weight of kept row a and column cols[c * 8 + e]

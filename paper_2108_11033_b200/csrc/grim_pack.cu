@@ -311,7 +311,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
             std::memcpy(&rc_blob[start + (size_t)b * 4], &hdr, 4);
             const size_t idx_bytes = ((size_t)8 + (size_t)nch * kRcChunk + 15) / 16 * 16;
             rc_blob.resize(rec + idx_bytes + (size_t)nch * kr * kRcChunk * 4, 0);
-            const uint64_t rows = hb.rowmask;  // bit r: block-local row r kept
+            const uint64_t rows = (uint64_t)hb.rowmask | ((uint64_t)kc << 32);  // low word: bit r = row r kept; high word: kc
             std::memcpy(&rc_blob[rec], &rows, 8);
             uint8_t cols[64];
             int n = 0;

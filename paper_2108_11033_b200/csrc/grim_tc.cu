@@ -1,8 +1,405 @@
-// Tensor-core (tcgen05) path for bf16 handles at large N.  Placeholder until the kernel lands:
-// reports the path as unavailable so that callers stay on the CUDA-core kernels.
+// Tensor-core (tcgen05) kernel for Y = W * X with bf16 operands and fp32 accumulation, large N
+// (Section 3.1: every layer is a GEMM; Sections 4.3 - 4.4: compact storage, expanded only on chip).
+//
+// The packed weights never exist in dense form in HBM.  A thread block owns 128 rows of W (in schedule
+// order) and 256 output columns and walks K in tiles of 64.  Per K tile
+//   - one thread asks TMA for the 64 x 256 tile of X (128-byte swizzle, the layout the tensor core reads
+//     directly as the N-major operand) and for the packed records of the thread block's bands,
+//   - four warps expand those records into a zero-filled 128 x 64 bf16 tile in shared memory, written in
+//     the K-major 128-byte-swizzled layout of the other operand,
+//   - one thread issues four tcgen05.mma (128 x 256 x 16) that accumulate in tensor memory.
+// A ring of stages with full / ready / empty mbarriers overlaps the three.  After the last K tile the four
+// warps read the accumulators back (tcgen05.ld), add bias, apply the activation and store Y.
+//
+// The multiply therefore runs at the tensor core's dense rate on a tile whose density is that of the
+// pruned matrix; it is chosen for bf16 handles when N is large, where even so it is several times faster
+// than the CUDA-core kernels.  Every wait is bounded; tensor memory is released on every exit path.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+#include <cstring>
+
 #include "grim_internal.h"
 
 namespace grim {
-bool tc_path_supported(const grim_bcr*, const SpmmArgs&) { return false; }
-grim_status_t launch_spmm_tc(const grim_bcr*, const SpmmArgs&, cudaStream_t) { return GRIM_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int kTcThreads = 192;   // warp 0: copies, warp 1: tensor core, warps 2-5: expansion + epilogue
+constexpr int kTM = 128;          // rows of W per thread block
+constexpr int kTQ = 256;          // output columns per thread block
+constexpr int kTK = 64;           // K per stage
+constexpr int kTcStages = 3;
+constexpr int kATileBytes = kTM * kTK * 2;   // 16 KiB
+constexpr int kBTileBytes = kTQ * kTK * 2;   // 32 KiB
+constexpr int kMaxBlobs = 8;                 // packed-record pieces per stage (band groups x block columns)
+constexpr int kTcHdrBytes = 1024;
+constexpr unsigned kTmemCols = 256;
+
+struct TcParams {
+  const RcStage* stage;
+  const uint8_t* blob;
+  const uint32_t* band_order;
+  unsigned* status;
+  int nbr, nbc, M, K, bh, bw, ngroups;
+  int bh_shift, slots_per_tile, groups_per_tile, j_per_tile;
+  uint32_t blob_stride, stage_bytes;
+  unsigned spin_limit;
+  SpmmArgs a;
+};
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
+  for (unsigned i = 0; i < limit; ++i) {
+    if (mbar_try_wait(bar, parity)) return true;
+    if ((i & 63u) == 63u && *abort_flag) return false;
+  }
+  return false;
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
+// Shared-memory matrix descriptor of the tensor core: start address, leading / stride byte offsets
+// (all without their 4 low bits), descriptor version 1, 128-byte swizzle.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4) | ((uint64_t)(lbo_bytes >> 4) << 16) | ((uint64_t)(sbo_bytes >> 4) << 32) |
+         (1ull << 46) | (2ull << 61);
+}
+// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = 256.
+constexpr uint32_t kIdesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) | ((kTQ >> 3) << 17) | ((kTM >> 4) << 24);
+
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}"
+      ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(kIdesc), "r"(accumulate)
+      : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+        "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+        "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+        "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+  asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
+  extern __shared__ uint8_t smem_raw[];
+  // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // copies of a stage have landed
+  uint64_t* ready = full + kTcStages;                          // the expanded weight tile of a stage is written
+  uint64_t* empty = ready + kTcStages;                         // the tensor core is done with a stage
+  uint64_t* acc_done = empty + kTcStages;                      // all multiplies of the tile are complete
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 128);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 132);
+  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 256);  // [stage][kMaxBlobs] bytes of each packed piece
+  uint8_t* stages = smem + kTcHdrBytes;
+  const uint32_t stage_bytes = p.stage_bytes;
+
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
+  const SpmmArgs& a = p.a;
+  const int64_t q0 = (int64_t)blockIdx.x * kTQ;
+  const int pos0 = blockIdx.y * p.slots_per_tile;  // first band (schedule position) of this tile
+  const int nkt = (p.K + kTK - 1) / kTK;
+
+  if (tid == 0) {
+    for (int s = 0; s < kTcStages; ++s) {
+      mbar_init(full + s, 1);
+      mbar_init(ready + s, 4);
+      mbar_init(empty + s, 1);
+    }
+    mbar_init(acc_done, 1);
+    *s_abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+  const uint32_t tmem_base = *s_tmem;
+
+  bool failed = false;
+  if (warp == 0) {
+    // ------------------------------------------------------------------ copies
+    if (lane == 0) {
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int slot = kt % kTcStages;
+        if (kt >= kTcStages && !mbar_wait(empty + slot, (unsigned)((kt / kTcStages - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
+        uint8_t* st = stages + (size_t)slot * stage_bytes;
+        uint32_t bytes[kMaxBlobs], off[kMaxBlobs], total = kBTileBytes;
+        const int g_first = pos0 / kRcBands;
+#pragma unroll
+        for (int i = 0; i < kMaxBlobs; ++i) {
+          bytes[i] = 0; off[i] = 0;
+          const int gi = i / p.j_per_tile, jj = i - gi * p.j_per_tile;
+          const int g = g_first + gi, j = kt * p.j_per_tile + jj;
+          if (gi < p.groups_per_tile && g < p.ngroups && j < p.nbc) {
+            const RcStage se = p.stage[(int64_t)g * p.nbc + j];
+            bytes[i] = se.bytes; off[i] = se.off16;
+          }
+          s_meta[slot * kMaxBlobs + i] = bytes[i];
+          total += bytes[i];
+        }
+        mbar_arrive_expect_tx(full + slot, total);
+#pragma unroll
+        for (int i = 0; i < kTQ / 64; ++i)
+          tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+#pragma unroll
+        for (int i = 0; i < kMaxBlobs; ++i)
+          if (bytes[i]) bulk_load(st + kATileBytes + kBTileBytes + i * p.blob_stride, p.blob + (size_t)off[i] * 16, bytes[i], full + slot);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ tensor core
+    if (lane == 0) {
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int slot = kt % kTcStages;
+        const unsigned par = (unsigned)((kt / kTcStages) & 1);
+        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort)) { failed = true; break; }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a_addr = smem_u32(stages + (size_t)slot * stage_bytes);
+        const uint32_t b_addr = a_addr + kATileBytes;
+#pragma unroll
+        for (int s = 0; s < kTK / 16; ++s) {
+          // A: K-major, rows 128 bytes apart, 8-row groups 1 KiB apart; 16 K-elements = 32 bytes further on
+          const uint64_t ad = smem_desc(a_addr + s * 32, 16, 1024);
+          // B: N-major, 64-column groups 8 KiB apart, 8-row K groups 1 KiB apart; 16 K-rows = 2 KiB further on
+          const uint64_t bd = smem_desc(b_addr + s * 2048, 64 * kTK * 2, 1024);
+          umma_bf16(tmem_base, ad, bd, (kt > 0 || s > 0) ? 1u : 0u);
+        }
+        umma_commit(empty + slot);  // arrives when the multiplies above have read their operands
+      }
+      if (!failed) umma_commit(acc_done);
+    }
+  } else {
+    // ------------------------------------------------------------------ expansion of the packed weights
+    const int ww = warp - 2;   // 0..3
+    for (int kt = 0; kt < nkt; ++kt) {
+      const int slot = kt % kTcStages;
+      if (!mbar_wait(full + slot, (unsigned)((kt / kTcStages) & 1), p.spin_limit, s_abort)) { failed = true; break; }
+      uint8_t* st = stages + (size_t)slot * stage_bytes;
+      // warp ww owns the bands of the tile whose index is ww mod 4: it clears their rows, then fills them, so no
+      // barrier between warps is needed
+      const int band_bytes = p.bh * 128;  // bh rows of 64 bf16
+      for (int ts = ww; ts < p.slots_per_tile; ts += 4) {
+        uint4* rows16 = reinterpret_cast<uint4*>(st + ts * band_bytes);
+        for (int i = lane; i < band_bytes / 16; i += 32) rows16[i] = make_uint4(0u, 0u, 0u, 0u);
+      }
+      __syncwarp();
+      for (int bi = 0; bi < p.groups_per_tile * p.j_per_tile; ++bi) {
+        if (s_meta[slot * kMaxBlobs + bi] == 0) continue;
+        const int gi = bi / p.j_per_tile, jj = bi - gi * p.j_per_tile;
+        const uint8_t* blob = st + kATileBytes + kBTileBytes + bi * p.blob_stride;
+        // band slots of group (g_first + gi) that belong to this tile
+        const int gpos0 = (pos0 / kRcBands + gi) * kRcBands;
+        for (int sl = ww; sl < kRcBands; sl += 4) {
+          const int tslot = gpos0 + sl - pos0;  // band index inside the tile
+          if (tslot < 0 || tslot >= p.slots_per_tile) continue;
+          const uint32_t hdr = reinterpret_cast<const uint32_t*>(blob)[sl];
+          const int kr = (hdr >> 16) & 0xFF, nch = hdr >> 24;
+          if (kr == 0) continue;
+          const uint8_t* rec = blob + (hdr & 0xFFFFu) * 16;
+          const uint32_t rowmask = reinterpret_cast<const uint32_t*>(rec)[0];
+          const int kc = (int)reinterpret_cast<const uint32_t*>(rec)[1];
+          const uint8_t* cols = rec + 8;
+          const float* w = reinterpret_cast<const float*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
+          const int n = nch * kr * kRcChunk;
+          for (int i = lane; i < n; i += 32) {
+            const int e = i & 7, ar = i >> 3;
+            const int ch = ar / kr, ai = ar - ch * kr;
+            const int c = ch * kRcChunk + e;
+            if (c >= kc) continue;  // padding of the last chunk
+            const int r = __fns(rowmask, 0, ai + 1);
+            const int row = (tslot << p.bh_shift) + r;
+            const int k = jj * p.bw + cols[c];
+            const uint32_t byte = row * 128 + ((((unsigned)k >> 3) ^ ((unsigned)row & 7u)) << 4) + ((k & 7) << 1);
+            *reinterpret_cast<__nv_bfloat16*>(st + byte) = __float2bfloat16_rn(w[i]);  // exact: the value is bf16 already
+          }
+        }
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
+      __syncwarp();
+      if (lane == 0) mbar_arrive(ready + slot);
+    }
+    // ------------------------------------------------------------------ epilogue
+    if (!__any_sync(0xffffffffu, failed)) {
+      if (!mbar_wait(acc_done, 0, p.spin_limit, s_abort)) failed = true;
+    }
+    if (!__any_sync(0xffffffffu, failed)) {
+      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+      const int quarter = warp & 3;                 // the tensor-memory lanes this warp may read
+      const int trow = quarter * 32 + lane;         // row of the tile held by this thread's lane
+      const int pos = pos0 + (trow >> p.bh_shift);
+      const int r = trow & (p.bh - 1);
+      int64_t row = -1;
+      if (pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + r;
+      const bool row_ok = row >= 0 && row < p.M;
+      const float bias = (row_ok && a.bias) ? __ldg(a.bias + row) : 0.f;
+      for (int cb = 0; cb < kTQ / 32; ++cb) {
+        uint32_t v[32];
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 32), v);
+        const int64_t q = q0 + cb * 32;
+        if (!row_ok || q >= a.ncols) continue;
+        float t[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+          t[i] = __uint_as_float(v[i]) + bias;
+          if (a.relu) t[i] = fmaxf(t[i], 0.f);
+        }
+        const int64_t off0 = row * a.y_sr + q;
+        const bool full_chunk = q + 31 < a.ncols;
+        if (a.y_dtype == GRIM_F32) {
+          float* y = static_cast<float*>(a.Y) + off0;
+          if (full_chunk && ((reinterpret_cast<uintptr_t>(y) & 15) == 0)) {
+#pragma unroll
+            for (int i = 0; i < 8; ++i) reinterpret_cast<float4*>(y)[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
+          } else {
+            for (int i = 0; i < 32 && q + i < a.ncols; ++i) y[i] = t[i];
+          }
+        } else {
+          __nv_bfloat16* y = static_cast<__nv_bfloat16*>(a.Y) + off0;
+          if (full_chunk && ((reinterpret_cast<uintptr_t>(y) & 15) == 0)) {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              uint4 u;
+              __nv_bfloat162 b0 = __floats2bfloat162_rn(t[8 * i], t[8 * i + 1]), b1 = __floats2bfloat162_rn(t[8 * i + 2], t[8 * i + 3]);
+              __nv_bfloat162 b2 = __floats2bfloat162_rn(t[8 * i + 4], t[8 * i + 5]), b3 = __floats2bfloat162_rn(t[8 * i + 6], t[8 * i + 7]);
+              u.x = *reinterpret_cast<unsigned*>(&b0); u.y = *reinterpret_cast<unsigned*>(&b1);
+              u.z = *reinterpret_cast<unsigned*>(&b2); u.w = *reinterpret_cast<unsigned*>(&b3);
+              reinterpret_cast<uint4*>(y)[i] = u;
+            }
+          } else {
+            for (int i = 0; i < 32 && q + i < a.ncols; ++i) y[i] = __float2bfloat16_rn(t[i]);
+          }
+        }
+      }
+    }
+  }
+
+  if (__any_sync(0xffffffffu, failed)) {
+    *s_abort = 1;
+    if (lane == 0) atomicExch(p.status, (unsigned)GRIM_ERR_TIMEOUT);
+  }
+  asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+  __syncthreads();
+  if (warp == 1) {
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+  }
+}
+
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn encode_tiled_fn() {
+  static EncodeTiledFn fn = [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) != cudaSuccess ||
+        q != cudaDriverEntryPointSuccess) {
+      cudaGetLastError();
+      p = nullptr;
+    }
+    return reinterpret_cast<EncodeTiledFn>(p);
+  }();
+  return fn;
+}
+
+int tc_blobs_per_stage(const grim_bcr* h) { return std::max(1, (kTM / h->bh) / kRcBands) * (kTK / h->bw); }
+size_t tc_stage_bytes(const grim_bcr* h) {
+  const size_t blob_stride = ((size_t)h->rc_max_blob + 127) & ~size_t(127);
+  return (kATileBytes + kBTileBytes + tc_blobs_per_stage(h) * blob_stride + 1023) & ~size_t(1023);
+}
+size_t tc_smem_need(const grim_bcr* h) { return 1024 + kTcHdrBytes + (size_t)kTcStages * tc_stage_bytes(h); }
+
+}  // namespace
+
+bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
+  if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_rc_stage || !h->d_status) return false;
+  if (h->bh != 4 && h->bh != 8 && h->bh != 16) return false;
+  if (h->bw != 16 && h->bw != 32 && h->bw != 64) return false;
+  if (a.conv || a.x_dtype != GRIM_BF16 || a.x_sq != 1 || a.y_sq != 1) return false;
+  if (reinterpret_cast<uintptr_t>(a.X) % 16 != 0 || (a.x_sk * 2) % 16 != 0) return false;
+  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->rc_max_blob == 0) return false;
+  if (tc_blobs_per_stage(h) > kMaxBlobs) return false;
+  if (tc_smem_need(h) > 225 * 1024) return false;
+  if ((h->nbr + (kTM / h->bh) - 1) / (kTM / h->bh) > 65535) return false;
+  return encode_tiled_fn() != nullptr;
+}
+
+grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
+  if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
+  TcParams p;
+  p.stage = h->d_rc_stage; p.blob = h->d_rc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
+  p.nbr = (int)h->nbr; p.nbc = (int)h->nbc; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.bw = h->bw;
+  p.ngroups = (int)h->rc_groups;
+  p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
+  p.slots_per_tile = kTM / h->bh;
+  p.groups_per_tile = std::max(1, p.slots_per_tile / kRcBands);
+  p.j_per_tile = kTK / h->bw;
+  p.blob_stride = (h->rc_max_blob + 127u) & ~127u;
+  p.stage_bytes = (uint32_t)tc_stage_bytes(h);
+  p.spin_limit = 1u << 20;
+  p.a = a;
+
+  CUtensorMap tm;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
+  const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * 2)};
+  const cuuint32_t box[2] = {64, (cuuint32_t)kTK};
+  const cuuint32_t estr[2] = {1, 1};
+  if (encode_tiled_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.X), dims, strides, box, estr,
+                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return GRIM_ERR_CUDA;
+  const size_t smem = tc_smem_need(h);
+  cudaError_t e = cudaFuncSetAttribute(bcr_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  if (e != cudaSuccess) return GRIM_ERR_CUDA;
+  const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
+  const int64_t mtiles = (h->nbr + p.slots_per_tile - 1) / p.slots_per_tile;
+  dim3 grid((unsigned)qtiles, (unsigned)mtiles);
+  bcr_tc_kernel<<<grid, kTcThreads, smem, s>>>(tm, p);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+}
+
 }  // namespace grim

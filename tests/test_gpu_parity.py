@@ -136,6 +136,20 @@ def test_register_tiled_kernel_explicit(B, case, bf16):
     check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=groups, path=1, flags=1)
 
 
+@pytest.mark.parametrize("y_bf16", [False, True])
+@pytest.mark.parametrize("case", [(256, 512, 8, 32, 256), (200, 333, 8, 32, 328), (300, 520, 4, 16, 520), (260, 700, 16, 64, 264),
+                                  (96, 153, 8, 32, 1024), (512, 2048, 16, 64, 776)])
+def test_tensor_core_kernel_explicit(B, case, y_bf16):
+    """The tcgen05 path asked for by name (path 2): bf16 operands, fp32 accumulation in tensor memory; ragged M, K
+    and N, empty blocks, pruned bands, every supported block shape."""
+    M, K, bh, bw, N = case
+    W = gen.dense_weight(M, K, seed=87)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=88, empty_frac=0.1)
+    mask[: 2 * bh] = 0
+    X = gen.normal_f32((K, N), 1.0, 89, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=2, flags=1, y_bf16=y_bf16)
+
+
 @pytest.mark.parametrize("split", [2, 5, 8])
 def test_split_multiply(B, split):
     """Few output tiles: several thread blocks share a tile's block columns and add their partial sums into a
