@@ -67,6 +67,18 @@ struct RcStage {
   uint32_t bytes;  // multiple of 16; 0 when no band of the group keeps anything in this block column
 };
 
+// ---------------------------------------------------------------------------------------------
+// Device layout for the tensor-core kernel (bf16 handles with bh in {4, 8, 16}, bw in {16, 32, 64}).
+// The matrix is cut into tiles of kTcRows rows (consecutive bands in schedule order) x kTcK columns;
+// per tile one contiguous record that lists its kept columns, sorted by kept-row count (largest first):
+//   u32 ncols, u32 nvals, u32 0, u32 0
+//   u32 colword[ncols]   k inside the tile (6 bits) | band inside the tile << 6 | row mask << 16; padded to x4
+//   u16 voff[ncols]      first value of the column; padded to x8
+//   bf16 val[nvals]      the column's kept values, top row first; padded to x8
+// ---------------------------------------------------------------------------------------------
+constexpr int kTcRows = 128;
+constexpr int kTcK = 64;
+
 struct HostBlock {
   uint64_t colmask = 0;
   uint32_t rowmask = 0;
@@ -106,6 +118,12 @@ struct grim_bcr {
   int device = -1;
   grim::RcStage* d_rc_stage = nullptr;
   uint8_t* d_rc_blob = nullptr;
+  // tensor-core layout
+  int64_t tc_mtiles = 0, tc_ktiles = 0;
+  uint32_t tc_max_rec = 0;
+  int64_t index_bytes_tc = 0;
+  grim::RcStage* d_tc_stage = nullptr;
+  uint8_t* d_tc_blob = nullptr;
   unsigned* d_status = nullptr;  // error word written by kernels whose bounded waits ran out
   grim::StageEntry* d_stage = nullptr;
   uint8_t* d_blob = nullptr;

@@ -48,6 +48,8 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_gemv_vals);
   cudaFree(h->d_rc_stage);
   cudaFree(h->d_rc_blob);
+  cudaFree(h->d_tc_stage);
+  cudaFree(h->d_tc_blob);
   cudaFree(h->d_status);
 }
 
@@ -334,6 +336,68 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
                           nbr * 4;
     }
 
+    // ---- tensor-core layout (bf16 handles whose block shape tiles 128 x 64 evenly)
+    std::vector<RcStage> tc_stage;
+    std::vector<uint8_t> tc_blob;
+    const bool tc_shape = vdt == GRIM_BF16 && (bh == 4 || bh == 8 || bh == 16) && (bw == 16 || bw == 32 || bw == 64);
+    if (tc_shape) {
+      const int S = kTcRows / bh, J = kTcK / bw;
+      h->tc_mtiles = (nbr + S - 1) / S;
+      h->tc_ktiles = (nbc + J - 1) / J;
+      tc_stage.resize((size_t)(h->tc_mtiles * h->tc_ktiles));
+      struct Col { uint32_t word; uint16_t kr, kc; const float* src; };
+      std::vector<Col> cols;
+      uint32_t tc_max = 0;
+      for (int64_t t = 0; t < h->tc_mtiles && st == GRIM_OK; ++t)
+        for (int64_t kt = 0; kt < h->tc_ktiles; ++kt) {
+          cols.clear();
+          uint32_t nvals = 0;
+          for (int ts = 0; ts < S; ++ts) {
+            const int64_t pos = t * S + ts;
+            if (pos >= nbr) break;
+            for (int jj = 0; jj < J; ++jj) {
+              const int64_t j = kt * J + jj;
+              if (j >= nbc) break;
+              const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
+              if (!(hb.kr && hb.kc)) continue;
+              int b = 0;
+              for (int c = 0; c < bw; ++c)
+                if ((hb.colmask >> c) & 1ull) {
+                  cols.push_back(Col{(uint32_t)(jj * bw + c) | ((uint32_t)ts << 6) | (hb.rowmask << 16), hb.kr, hb.kc,
+                                     &h->vals[(size_t)hb.val_off + (size_t)b]});
+                  ++b;
+                  nvals += hb.kr;
+                }
+            }
+          }
+          RcStage& se = tc_stage[(size_t)(t * h->tc_ktiles + kt)];
+          se.off16 = (uint32_t)(tc_blob.size() / 16);
+          se.bytes = 0;
+          if (cols.empty()) continue;
+          if (tc_blob.size() / 16 >= (uint64_t(1) << 32) || nvals > 0xFFFFu) { st = GRIM_ERR_UNSUPPORTED; break; }
+          std::stable_sort(cols.begin(), cols.end(), [](const Col& x, const Col& y) { return x.kr > y.kr; });
+          const size_t n = cols.size(), n4 = (n + 3) / 4 * 4, n8 = (n + 7) / 8 * 8, v8 = ((size_t)nvals + 7) / 8 * 8;
+          const size_t start = tc_blob.size();
+          tc_blob.resize(start + 16 + n4 * 4 + n8 * 2 + v8 * 2, 0);
+          uint32_t* hdr = reinterpret_cast<uint32_t*>(&tc_blob[start]);
+          hdr[0] = (uint32_t)n; hdr[1] = nvals;
+          uint32_t* cw = hdr + 4;
+          uint16_t* vo = reinterpret_cast<uint16_t*>(cw + n4);
+          uint16_t* vv = vo + n8;
+          uint32_t o = 0;
+          for (size_t i = 0; i < n; ++i) {
+            cw[i] = cols[i].word;
+            vo[i] = (uint16_t)o;
+            for (int a = 0; a < cols[i].kr; ++a) vv[o++] = bf16_bits(cols[i].src[(size_t)a * cols[i].kc]);
+          }
+          se.bytes = (uint32_t)(tc_blob.size() - start);
+          tc_max = std::max(tc_max, se.bytes);
+        }
+      if (st != GRIM_OK) { delete h; return st; }
+      h->tc_max_rec = tc_max;
+      h->index_bytes_tc = (int64_t)tc_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)tc_blob.size() - (int64_t)nnz * 2 + nbr * 4;
+    }
+
     // ---- upload
     if (!(flags & GRIM_PACK_HOST_ONLY)) {
       cudaError_t e = cudaGetDevice(&h->device);
@@ -342,6 +406,10 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       if (e == cudaSuccess) e = upload(&h->d_band_order, h->band_order.data(), h->band_order.size() * 4);
       if (e == cudaSuccess) e = upload(&h->d_rc_stage, rc_stage.data(), rc_stage.size() * sizeof(RcStage));
       if (e == cudaSuccess) e = upload(&h->d_rc_blob, rc_blob.data(), rc_blob.size());
+      if (e == cudaSuccess && tc_shape) {
+        e = upload(&h->d_tc_stage, tc_stage.data(), tc_stage.size() * sizeof(RcStage));
+        if (e == cudaSuccess) e = upload(&h->d_tc_blob, tc_blob.data(), tc_blob.size());
+      }
       const unsigned zero = 0;
       if (e == cudaSuccess) e = upload(&h->d_status, &zero, 4);
       if (e == cudaSuccess && h->gemv_ok) {

@@ -5,10 +5,10 @@
 // order) and 256 output columns and walks K in tiles of 64.  Per K tile
 //   - one thread asks TMA for the 64 x 256 tile of X (128-byte swizzle, the layout the tensor core reads
 //     directly as the N-major operand) and for the packed records of the thread block's bands,
-//   - four warps expand those records into a zero-filled 128 x 64 bf16 tile in shared memory, written in
+//   - eight warps expand those records into a zero-filled 128 x 64 bf16 tile in shared memory, written in
 //     the K-major 128-byte-swizzled layout of the other operand,
 //   - one thread issues four tcgen05.mma (128 x 256 x 16) that accumulate in tensor memory.
-// A ring of stages with full / ready / empty mbarriers overlaps the three.  After the last K tile the four
+// A ring of stages with full / ready / empty mbarriers overlaps the three.  After the last K tile the eight
 // warps read the accumulators back (tcgen05.ld), add bias, apply the activation and store Y.
 //
 // The multiply therefore runs at the tensor core's dense rate on a tile whose density is that of the
@@ -25,14 +25,14 @@
 namespace grim {
 namespace {
 
-constexpr int kTcThreads = 192;   // warp 0: copies, warp 1: tensor core, warps 2-5: expansion + epilogue
+constexpr int kTcWorkers = 8;      // warps that expand the packed weights and later run the epilogue
+constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
 constexpr int kTM = 128;          // rows of W per thread block
 constexpr int kTQ = 256;          // output columns per thread block
 constexpr int kTK = 64;           // K per stage
-constexpr int kTcStages = 3;
+constexpr int kTcStages = 4;
 constexpr int kATileBytes = kTM * kTK * 2;   // 16 KiB
 constexpr int kBTileBytes = kTQ * kTK * 2;   // 32 KiB
-constexpr int kMaxBlobs = 8;                 // packed-record pieces per stage (band groups x block columns)
 constexpr int kTcHdrBytes = 1024;
 constexpr unsigned kTmemCols = 256;
 
@@ -41,9 +41,9 @@ struct TcParams {
   const uint8_t* blob;
   const uint32_t* band_order;
   unsigned* status;
-  int nbr, nbc, M, K, bh, bw, ngroups;
-  int bh_shift, slots_per_tile, groups_per_tile, j_per_tile;
-  uint32_t blob_stride, stage_bytes;
+  int nbr, M, K, bh, nkt;
+  int bh_shift, slots_per_tile;
+  uint32_t stage_bytes;
   unsigned spin_limit;
   SpmmArgs a;
 };
@@ -123,12 +123,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // copies of a stage have landed
-  uint64_t* ready = full + kTcStages;                          // the expanded weight tile of a stage is written
+  uint64_t* zeroed = full + kTcStages;                         // every worker has cleared its part of the weight tile
+  uint64_t* ready = zeroed + kTcStages;                        // the expanded weight tile of a stage is written
   uint64_t* empty = ready + kTcStages;                         // the tensor core is done with a stage
   uint64_t* acc_done = empty + kTcStages;                      // all multiplies of the tile are complete
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 128);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 132);
-  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 256);  // [stage][kMaxBlobs] bytes of each packed piece
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 192);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 196);
+  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 256);  // [stage] bytes of the stage's packed record (0: none)
   uint8_t* stages = smem + kTcHdrBytes;
   const uint32_t stage_bytes = p.stage_bytes;
 
@@ -137,12 +138,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
   const SpmmArgs& a = p.a;
   const int64_t q0 = (int64_t)blockIdx.x * kTQ;
   const int pos0 = blockIdx.y * p.slots_per_tile;  // first band (schedule position) of this tile
-  const int nkt = (p.K + kTK - 1) / kTK;
+  const int nkt = p.nkt;
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full + s, 1);
-      mbar_init(ready + s, 4);
+      mbar_init(zeroed + s, kTcWorkers);
+      mbar_init(ready + s, kTcWorkers);
       mbar_init(empty + s, 1);
     }
     mbar_init(acc_done, 1);
@@ -166,27 +168,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
         const int slot = kt % kTcStages;
         if (kt >= kTcStages && !mbar_wait(empty + slot, (unsigned)((kt / kTcStages - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
         uint8_t* st = stages + (size_t)slot * stage_bytes;
-        uint32_t bytes[kMaxBlobs], off[kMaxBlobs], total = kBTileBytes;
-        const int g_first = pos0 / kRcBands;
-#pragma unroll
-        for (int i = 0; i < kMaxBlobs; ++i) {
-          bytes[i] = 0; off[i] = 0;
-          const int gi = i / p.j_per_tile, jj = i - gi * p.j_per_tile;
-          const int g = g_first + gi, j = kt * p.j_per_tile + jj;
-          if (gi < p.groups_per_tile && g < p.ngroups && j < p.nbc) {
-            const RcStage se = p.stage[(int64_t)g * p.nbc + j];
-            bytes[i] = se.bytes; off[i] = se.off16;
-          }
-          s_meta[slot * kMaxBlobs + i] = bytes[i];
-          total += bytes[i];
-        }
-        mbar_arrive_expect_tx(full + slot, total);
+        const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt];
+        s_meta[slot] = se.bytes;
+        mbar_arrive_expect_tx(full + slot, kBTileBytes + se.bytes);
 #pragma unroll
         for (int i = 0; i < kTQ / 64; ++i)
           tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
-#pragma unroll
-        for (int i = 0; i < kMaxBlobs; ++i)
-          if (bytes[i]) bulk_load(st + kATileBytes + kBTileBytes + i * p.blob_stride, p.blob + (size_t)off[i] * 16, bytes[i], full + slot);
+        if (se.bytes) bulk_load(st + kATileBytes + kBTileBytes, p.blob + (size_t)se.off16 * 16, se.bytes, full + slot);
       }
     }
   } else if (warp == 1) {
@@ -213,47 +201,37 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
-    const int ww = warp - 2;   // 0..3
+    const int wt = tid - 64;   // 0 .. 32 * kTcWorkers - 1
     for (int kt = 0; kt < nkt; ++kt) {
       const int slot = kt % kTcStages;
-      if (!mbar_wait(full + slot, (unsigned)((kt / kTcStages) & 1), p.spin_limit, s_abort)) { failed = true; break; }
+      const unsigned par = (unsigned)((kt / kTcStages) & 1);
+      if (!__all_sync(0xffffffffu, mbar_wait(full + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
-      // warp ww owns the bands of the tile whose index is ww mod 4: it clears their rows, then fills them, so no
-      // barrier between warps is needed
-      const int band_bytes = p.bh * 128;  // bh rows of 64 bf16
-      for (int ts = ww; ts < p.slots_per_tile; ts += 4) {
-        uint4* rows16 = reinterpret_cast<uint4*>(st + ts * band_bytes);
-        for (int i = lane; i < band_bytes / 16; i += 32) rows16[i] = make_uint4(0u, 0u, 0u, 0u);
-      }
+      uint4* a4 = reinterpret_cast<uint4*>(st);
+#pragma unroll
+      for (int i = 0; i < kATileBytes / 16 / (32 * kTcWorkers); ++i) a4[wt + i * 32 * kTcWorkers] = make_uint4(0u, 0u, 0u, 0u);
       __syncwarp();
-      for (int bi = 0; bi < p.groups_per_tile * p.j_per_tile; ++bi) {
-        if (s_meta[slot * kMaxBlobs + bi] == 0) continue;
-        const int gi = bi / p.j_per_tile, jj = bi - gi * p.j_per_tile;
-        const uint8_t* blob = st + kATileBytes + kBTileBytes + bi * p.blob_stride;
-        // band slots of group (g_first + gi) that belong to this tile
-        const int gpos0 = (pos0 / kRcBands + gi) * kRcBands;
-        for (int sl = ww; sl < kRcBands; sl += 4) {
-          const int tslot = gpos0 + sl - pos0;  // band index inside the tile
-          if (tslot < 0 || tslot >= p.slots_per_tile) continue;
-          const uint32_t hdr = reinterpret_cast<const uint32_t*>(blob)[sl];
-          const int kr = (hdr >> 16) & 0xFF, nch = hdr >> 24;
-          if (kr == 0) continue;
-          const uint8_t* rec = blob + (hdr & 0xFFFFu) * 16;
-          const uint32_t rowmask = reinterpret_cast<const uint32_t*>(rec)[0];
-          const int kc = (int)reinterpret_cast<const uint32_t*>(rec)[1];
-          const uint8_t* cols = rec + 8;
-          const float* w = reinterpret_cast<const float*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
-          const int n = nch * kr * kRcChunk;
-          for (int i = lane; i < n; i += 32) {
-            const int e = i & 7, ar = i >> 3;
-            const int ch = ar / kr, ai = ar - ch * kr;
-            const int c = ch * kRcChunk + e;
-            if (c >= kc) continue;  // padding of the last chunk
-            const int r = __fns(rowmask, 0, ai + 1);
-            const int row = (tslot << p.bh_shift) + r;
-            const int k = jj * p.bw + cols[c];
-            const uint32_t byte = row * 128 + ((((unsigned)k >> 3) ^ ((unsigned)row & 7u)) << 4) + ((k & 7) << 1);
-            *reinterpret_cast<__nv_bfloat16*>(st + byte) = __float2bfloat16_rn(w[i]);  // exact: the value is bf16 already
+      if (lane == 0) mbar_arrive(zeroed + slot);
+      if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
+      if (s_meta[slot]) {
+        // a thread takes kept columns of the tile: it walks the column's row mask and drops the column's values
+        // into the swizzled K-major tile (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits)
+        const uint32_t* rec = reinterpret_cast<const uint32_t*>(st + kATileBytes + kBTileBytes);
+        const int ncols = (int)rec[0];
+        const uint32_t* cw = rec + 4;
+        const uint16_t* vo = reinterpret_cast<const uint16_t*>(cw + ((ncols + 3) & ~3));
+        const uint16_t* vals = vo + ((ncols + 7) & ~7);
+        for (int c = wt; c < ncols; c += 32 * kTcWorkers) {
+          const uint32_t w = cw[c];
+          uint32_t o = vo[c];
+          const uint32_t k = w & 63u;
+          const uint32_t rowbase = ((w >> 6) & 31u) << p.bh_shift;
+          const uint32_t kbyte = (k & 7u) << 1, kchunk = k >> 3;
+          uint32_t rm = w >> 16;
+          while (rm) {
+            const uint32_t row = rowbase + (uint32_t)__ffs((int)rm) - 1u;
+            rm &= rm - 1u;
+            *reinterpret_cast<uint16_t*>(st + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = vals[o++];
           }
         }
       }
@@ -263,7 +241,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
     }
     // ------------------------------------------------------------------ epilogue
     if (!__any_sync(0xffffffffu, failed)) {
-      if (!mbar_wait(acc_done, 0, p.spin_limit, s_abort)) failed = true;
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_done, 0, p.spin_limit, s_abort))) failed = true;
     }
     if (!__any_sync(0xffffffffu, failed)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -275,7 +253,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
       if (pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + r;
       const bool row_ok = row >= 0 && row < p.M;
       const float bias = (row_ok && a.bias) ? __ldg(a.bias + row) : 0.f;
-      for (int cb = 0; cb < kTQ / 32; ++cb) {
+      const int cb0 = ((warp - 2) >> 2) * (kTQ / 64), cb1 = cb0 + kTQ / 64;  // warps 2-5: columns 0-127, warps 6-9: 128-255
+      for (int cb = cb0; cb < cb1; ++cb) {
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 32), v);
         const int64_t q = q0 + cb * 32;
@@ -345,39 +324,28 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-int tc_blobs_per_stage(const grim_bcr* h) { return std::max(1, (kTM / h->bh) / kRcBands) * (kTK / h->bw); }
-size_t tc_stage_bytes(const grim_bcr* h) {
-  const size_t blob_stride = ((size_t)h->rc_max_blob + 127) & ~size_t(127);
-  return (kATileBytes + kBTileBytes + tc_blobs_per_stage(h) * blob_stride + 1023) & ~size_t(1023);
-}
+size_t tc_stage_bytes(const grim_bcr* h) { return (kATileBytes + kBTileBytes + (size_t)h->tc_max_rec + 1023) & ~size_t(1023); }
 size_t tc_smem_need(const grim_bcr* h) { return 1024 + kTcHdrBytes + (size_t)kTcStages * tc_stage_bytes(h); }
 
 }  // namespace
 
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
-  if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_rc_stage || !h->d_status) return false;
-  if (h->bh != 4 && h->bh != 8 && h->bh != 16) return false;
-  if (h->bw != 16 && h->bw != 32 && h->bw != 64) return false;
+  if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_tc_stage || !h->d_status) return false;
   if (a.conv || a.x_dtype != GRIM_BF16 || a.x_sq != 1 || a.y_sq != 1) return false;
   if (reinterpret_cast<uintptr_t>(a.X) % 16 != 0 || (a.x_sk * 2) % 16 != 0) return false;
-  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->rc_max_blob == 0) return false;
-  if (tc_blobs_per_stage(h) > kMaxBlobs) return false;
+  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
   if (tc_smem_need(h) > 225 * 1024) return false;
-  if ((h->nbr + (kTM / h->bh) - 1) / (kTM / h->bh) > 65535) return false;
+  if (h->tc_mtiles > 65535) return false;
   return encode_tiled_fn() != nullptr;
 }
 
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
   if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
   TcParams p;
-  p.stage = h->d_rc_stage; p.blob = h->d_rc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
-  p.nbr = (int)h->nbr; p.nbc = (int)h->nbc; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.bw = h->bw;
-  p.ngroups = (int)h->rc_groups;
+  p.stage = h->d_tc_stage; p.blob = h->d_tc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
+  p.nbr = (int)h->nbr; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.nkt = (int)h->tc_ktiles;
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;
-  p.groups_per_tile = std::max(1, p.slots_per_tile / kRcBands);
-  p.j_per_tile = kTK / h->bw;
-  p.blob_stride = (h->rc_max_blob + 127u) & ~127u;
   p.stage_bytes = (uint32_t)tc_stage_bytes(h);
   p.spin_limit = 1u << 20;
   p.a = a;
@@ -395,7 +363,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   cudaError_t e = cudaFuncSetAttribute(bcr_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
-  const int64_t mtiles = (h->nbr + p.slots_per_tile - 1) / p.slots_per_tile;
+  const int64_t mtiles = h->tc_mtiles;
   dim3 grid((unsigned)qtiles, (unsigned)mtiles);
   bcr_tc_kernel<<<grid, kTcThreads, smem, s>>>(tm, p);
   count_launch();
