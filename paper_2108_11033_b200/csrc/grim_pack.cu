@@ -376,7 +376,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
           if (cols.empty()) continue;
           if (tc_blob.size() / 16 >= (uint64_t(1) << 32) || nvals > 0xFFFFu) { st = GRIM_ERR_UNSUPPORTED; break; }
           std::stable_sort(cols.begin(), cols.end(), [](const Col& x, const Col& y) { return x.kr > y.kr; });
-          const size_t n = cols.size(), n4 = (n + 3) / 4 * 4, n8 = (n + 7) / 8 * 8, v8 = ((size_t)nvals + 7) / 8 * 8;
+          const size_t n = cols.size(), n4 = (n + 3) / 4 * 4, n8 = (n + 7) / 8 * 8, v8 = ((size_t)nvals + 8) / 8 * 8;  // at least one spare value: the kernel reads one past a column's last
           const size_t start = tc_blob.size();
           tc_blob.resize(start + 16 + n4 * 4 + n8 * 2 + v8 * 2, 0);
           uint32_t* hdr = reinterpret_cast<uint32_t*>(&tc_blob[start]);

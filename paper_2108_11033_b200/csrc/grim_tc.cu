@@ -26,11 +26,14 @@ namespace grim {
 namespace {
 
 constexpr int kTcWorkers = 8;      // warps that expand the packed weights and later run the epilogue
+constexpr int kTcGroups = 2;       // the workers form groups that take K tiles in turn, so that expansions overlap
+constexpr int kTcGroupWarps = kTcWorkers / kTcGroups;
+constexpr int kTcGroupThreads = 32 * kTcGroupWarps;
 constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
 constexpr int kTM = 128;          // rows of W per thread block
 constexpr int kTQ = 256;          // output columns per thread block
 constexpr int kTK = 64;           // K per stage
-constexpr int kTcStages = 4;
+constexpr int kTcStages = 4;        // ring slots at most; fewer when the packed records are large
 constexpr int kATileBytes = kTM * kTK * 2;   // 16 KiB
 constexpr int kBTileBytes = kTQ * kTK * 2;   // 32 KiB
 constexpr int kTcHdrBytes = 1024;
@@ -42,7 +45,7 @@ struct TcParams {
   const uint32_t* band_order;
   unsigned* status;
   int nbr, M, K, bh, nkt;
-  int bh_shift, slots_per_tile;
+  int bh_shift, slots_per_tile, nstages;
   uint32_t stage_bytes;
   unsigned spin_limit;
   SpmmArgs a;
@@ -118,6 +121,7 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+template <int BH>
 __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
@@ -138,13 +142,13 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
   const SpmmArgs& a = p.a;
   const int64_t q0 = (int64_t)blockIdx.x * kTQ;
   const int pos0 = blockIdx.y * p.slots_per_tile;  // first band (schedule position) of this tile
-  const int nkt = p.nkt;
+  const int nkt = p.nkt, ns = p.nstages;
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full + s, 1);
-      mbar_init(zeroed + s, kTcWorkers);
-      mbar_init(ready + s, kTcWorkers);
+      mbar_init(zeroed + s, kTcGroupWarps);
+      mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
     }
     mbar_init(acc_done, 1);
@@ -165,8 +169,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
       for (int kt = 0; kt < nkt; ++kt) {
-        const int slot = kt % kTcStages;
-        if (kt >= kTcStages && !mbar_wait(empty + slot, (unsigned)((kt / kTcStages - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
+        const int slot = kt % ns;
+        if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
         uint8_t* st = stages + (size_t)slot * stage_bytes;
         const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt];
         s_meta[slot] = se.bytes;
@@ -181,8 +185,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
     // ------------------------------------------------------------------ tensor core
     if (lane == 0) {
       for (int kt = 0; kt < nkt; ++kt) {
-        const int slot = kt % kTcStages;
-        const unsigned par = (unsigned)((kt / kTcStages) & 1);
+        const int slot = kt % ns;
+        const unsigned par = (unsigned)((kt / ns) & 1);
         if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort)) { failed = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(stages + (size_t)slot * stage_bytes);
@@ -201,37 +205,42 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
     }
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
-    const int wt = tid - 64;   // 0 .. 32 * kTcWorkers - 1
-    for (int kt = 0; kt < nkt; ++kt) {
-      const int slot = kt % kTcStages;
-      const unsigned par = (unsigned)((kt / kTcStages) & 1);
+    const int grp = (warp - 2) / kTcGroupWarps;               // this warp's group
+    const int wt = tid - 64 - grp * kTcGroupThreads;           // 0 .. kTcGroupThreads - 1 inside the group
+    for (int kt = grp; kt < nkt; kt += kTcGroups) {
+      const int slot = kt % ns;
+      const unsigned par = (unsigned)((kt / ns) & 1);
       if (!__all_sync(0xffffffffu, mbar_wait(full + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
       uint4* a4 = reinterpret_cast<uint4*>(st);
 #pragma unroll
-      for (int i = 0; i < kATileBytes / 16 / (32 * kTcWorkers); ++i) a4[wt + i * 32 * kTcWorkers] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = 0; i < kATileBytes / 16 / kTcGroupThreads; ++i) a4[wt + i * kTcGroupThreads] = make_uint4(0u, 0u, 0u, 0u);
       __syncwarp();
       if (lane == 0) mbar_arrive(zeroed + slot);
       if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
       if (s_meta[slot]) {
-        // a thread takes kept columns of the tile: it walks the column's row mask and drops the column's values
-        // into the swizzled K-major tile (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits)
+        // a thread takes kept columns of the tile and drops each column's values into the swizzled K-major tile
+        // (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits).  All loads of a column are
+        // issued before its stores: the value of row r sits popcount(mask below r) places after the first
         const uint32_t* rec = reinterpret_cast<const uint32_t*>(st + kATileBytes + kBTileBytes);
         const int ncols = (int)rec[0];
         const uint32_t* cw = rec + 4;
         const uint16_t* vo = reinterpret_cast<const uint16_t*>(cw + ((ncols + 3) & ~3));
         const uint16_t* vals = vo + ((ncols + 7) & ~7);
-        for (int c = wt; c < ncols; c += 32 * kTcWorkers) {
+        for (int c = wt; c < ncols; c += kTcGroupThreads) {
           const uint32_t w = cw[c];
-          uint32_t o = vo[c];
+          const uint16_t* v = vals + vo[c];
           const uint32_t k = w & 63u;
-          const uint32_t rowbase = ((w >> 6) & 31u) << p.bh_shift;
+          const uint32_t rowbase = ((w >> 6) & 31u) * BH;
           const uint32_t kbyte = (k & 7u) << 1, kchunk = k >> 3;
-          uint32_t rm = w >> 16;
-          while (rm) {
-            const uint32_t row = rowbase + (uint32_t)__ffs((int)rm) - 1u;
-            rm &= rm - 1u;
-            *reinterpret_cast<uint16_t*>(st + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = vals[o++];
+          const uint32_t rm = w >> 16;
+          uint16_t val[BH];
+#pragma unroll
+          for (int r = 0; r < BH; ++r) val[r] = v[__popc(rm & ((1u << r) - 1u))];  // in bounds for every r (< kr + pad)
+#pragma unroll
+          for (int r = 0; r < BH; ++r) {
+            const uint32_t row = rowbase + r;
+            if ((rm >> r) & 1u) *reinterpret_cast<uint16_t*>(st + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = val[r];
           }
         }
       }
@@ -248,7 +257,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
       const int quarter = warp & 3;                 // the tensor-memory lanes this warp may read
       const int trow = quarter * 32 + lane;         // row of the tile held by this thread's lane
       const int pos = pos0 + (trow >> p.bh_shift);
-      const int r = trow & (p.bh - 1);
+      const int r = trow & (BH - 1);
       int64_t row = -1;
       if (pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + r;
       const bool row_ok = row >= 0 && row < p.M;
@@ -325,7 +334,12 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 size_t tc_stage_bytes(const grim_bcr* h) { return (kATileBytes + kBTileBytes + (size_t)h->tc_max_rec + 1023) & ~size_t(1023); }
-size_t tc_smem_need(const grim_bcr* h) { return 1024 + kTcHdrBytes + (size_t)kTcStages * tc_stage_bytes(h); }
+size_t tc_smem_need(const grim_bcr* h, int stages) { return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(h); }
+int tc_stages(const grim_bcr* h) {
+  for (int s = kTcStages; s >= 2; --s)
+    if (tc_smem_need(h, s) <= 225 * 1024) return s;
+  return 0;
+}
 
 }  // namespace
 
@@ -334,7 +348,7 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (a.conv || a.x_dtype != GRIM_BF16 || a.x_sq != 1 || a.y_sq != 1) return false;
   if (reinterpret_cast<uintptr_t>(a.X) % 16 != 0 || (a.x_sk * 2) % 16 != 0) return false;
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
-  if (tc_smem_need(h) > 225 * 1024) return false;
+  if (tc_stages(h) == 0) return false;
   if (h->tc_mtiles > 65535) return false;
   return encode_tiled_fn() != nullptr;
 }
@@ -347,6 +361,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;
   p.stage_bytes = (uint32_t)tc_stage_bytes(h);
+  p.nstages = tc_stages(h);
   p.spin_limit = 1u << 20;
   p.a = a;
 
@@ -359,13 +374,14 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
-  const size_t smem = tc_smem_need(h);
-  cudaError_t e = cudaFuncSetAttribute(bcr_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  const size_t smem = tc_smem_need(h, p.nstages);
+  auto kern = h->bh == 4 ? bcr_tc_kernel<4> : (h->bh == 8 ? bcr_tc_kernel<8> : bcr_tc_kernel<16>);
+  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
   const int64_t mtiles = h->tc_mtiles;
   dim3 grid((unsigned)qtiles, (unsigned)mtiles);
-  bcr_tc_kernel<<<grid, kTcThreads, smem, s>>>(tm, p);
+  kern<<<grid, kTcThreads, smem, s>>>(tm, p);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
 }
