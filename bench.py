@@ -38,8 +38,8 @@ def measured_peaks():
         with open(p) as f:
             d = json.load(f)
         return dict(hbm_gbs=float(d["hbm_gbs"]), bf16_tflops=float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
-                    source="measured")
-    return dict(hbm_gbs=6650.0, bf16_tflops=1590.0, source="fallback")
+                    bf16_tflops_burst=float(d["bf16_tflops"]), source="measured")
+    return dict(hbm_gbs=6650.0, bf16_tflops=1400.0, bf16_tflops_burst=1590.0, source="fallback")
 
 
 class ClockSampler:
@@ -119,8 +119,9 @@ class GruWorkload:
             self.kernel_bytes += self.T * (i.value_bytes + i.index_bytes_gemv + 3 * self.H * 4 + 2 * self.H * 4)
         self.h2d = self.x_host.numel() * 4
         self.d2h = self.y_host.numel() * 4
-        self.kernel = "gru_recurrent_kernel"
-        self.bound = "hbm"
+        self.kernel = "gru_cluster_reg_kernel"
+        self.peak_kind = "alu"
+        self.force_bound = "hbm"  # a chain of dependent steps: reported against the streamed-bytes figure
 
     def step(self):
         self.B.grim_gru_seq(self.g, self.x, self.y)
@@ -171,12 +172,15 @@ class SpmmWorkload:
         self.y_host = torch.empty(self.M, self.N).pin_memory()
         i = B.grim_bcr_info(self.h)
         esz = 2 if self.bf16 else 4
-        idx = i.index_bytes_gemv if self.N == 1 else i.index_bytes_spmm
+        idx = i.index_bytes_gemv if self.N <= 16 else i.index_bytes_spmm
         self.kernel_bytes = float(i.value_bytes + idx + i.k_used * self.N * esz + self.M * self.N * 4)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * 4
-        self.kernel = "bcr_gemv_kernel" if self.N == 1 else "bcr_spmm_kernel"
-        self.bound = "hbm" if self.N <= 16 else "alu"
+        tc = self.bf16 and self.N >= 256 and self.bh in (4, 8, 16) and self.bw in (16, 32, 64)
+        self.kernel = "bcr_skinny_kernel" if self.N <= 16 else ("bcr_tc_kernel" if tc else "bcr_ffma_kernel")
+        self.peak_kind = "tensor" if tc else "alu"
+        if tc:
+            self.kernel_bytes = float(i.value_bytes + i.index_bytes_tc + i.k_used * self.N * esz + self.M * self.N * 4)
         self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
 
     def step(self):
@@ -231,8 +235,8 @@ class ConvWorkload:
         self.kernel_bytes = float(i.value_bytes + i.index_bytes_spmm + self.x.numel() * esz + self.y.numel() * esz)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * esz
-        self.kernel = "bcr_spmm_kernel<conv>"
-        self.bound = "alu"
+        self.kernel = "bcr_ffma_kernel (implicit im2col)"
+        self.peak_kind = "alu"
         self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
 
     def step(self):
@@ -260,6 +264,107 @@ class ConvWorkload:
         dt = time.perf_counter() - t0
         return 2.0 * self.nnz * 28 * 28 / dt / 1e9, f"1 of {self.batch} images, direct fp64 NumPy convolution with the masked dense weight"
 
+class VggWorkload:
+    """The 13 convolution layers of VGG-16 (3x3, stride 1, pad 1, ReLU; 2x2 max-pool after layers 2, 4, 7, 10, 13),
+    every layer BCR-pruned 8x with 8x32 blocks, bf16 activations and weights, fp32 accumulation."""
+
+    def __init__(self, batch=1, image=224):
+        from workloads import generators as gen
+        self.net = gen.vgg16_stack(batch, image=image)
+        self.batch, self.image = batch, image
+        self.name = f"vgg16_convstack_{image}x{image}_b{batch}_bcr8x32_c8_bf16"
+        self.dtype = "bf16"
+        self.nnz = sum(int(L["mask"].sum()) for L in self.net["layers"])
+        self.flops = sum(2.0 * int(L["mask"].sum()) * batch * L["hw"] * L["hw"] for L in self.net["layers"])
+        self.peak_kind = "alu"
+        self.kernel = "bcr_ffma_kernel (implicit im2col, per layer)"
+
+    def setup(self, B, torch):
+        self.B, self.torch = B, torch
+        net = self.net
+        self.h, self.bias, self.bufs, self.info = [], [], [], []
+        self.x_host = torch.from_numpy(net["x"]).to(torch.bfloat16).pin_memory()
+        self.x = self.x_host.cuda()
+        cur_hw = self.image
+        for L in net["layers"]:
+            self.h.append(B.grim_bcr_pack(L["W"], L["mask"], net["bh"], net["bw"], B.GRIM_BF16, B.GRIM_PACK_REORDER))
+            self.bias.append(torch.from_numpy(L["bias"]).cuda())
+            out = torch.empty(self.batch, L["cout"], cur_hw, cur_hw, device="cuda", dtype=torch.bfloat16)
+            pooled = None
+            if L["pool"]:
+                cur_hw //= 2
+                pooled = torch.empty(self.batch, L["cout"], cur_hw, cur_hw, device="cuda", dtype=torch.bfloat16)
+            self.bufs.append((out, pooled))
+            self.info.append(B.grim_bcr_info(self.h[-1]))
+        self.y_host = torch.empty_like(self.bufs[-1][1], device="cpu").pin_memory()
+        self.ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in net["layers"]]
+        self.layer_bytes, self.layer_flops = [], []
+        for L, i in zip(net["layers"], self.info):
+            npx = self.batch * L["hw"] * L["hw"]
+            self.layer_bytes.append(float(i.value_bytes + i.index_bytes_spmm + 2 * L["cin"] * npx + 2 * L["cout"] * npx))
+            self.layer_flops.append(2.0 * i.nnz * npx)
+        self.kernel_bytes = sum(self.layer_bytes)
+        self.h2d = self.x_host.numel() * 2
+        self.d2h = self.y_host.numel() * 2
+        self.layer_ms = [[] for _ in net["layers"]]
+
+    def _run(self, x):
+        B = self.B
+        cur = x
+        for li, L in enumerate(self.net["layers"]):
+            out, pooled = self.bufs[li]
+            self.ev[li][0].record()
+            B.grim_bcr_conv2d(self.h[li], cur, out, 3, 1, 1, bias=self.bias[li], relu=True)
+            self.ev[li][1].record()
+            if pooled is not None:
+                B.grim_maxpool2x2(out, pooled)
+                cur = pooled
+            else:
+                cur = out
+        return cur
+
+    def step(self):
+        self._run(self.x)
+
+    def step_e2e(self):
+        xd = self.x_host.cuda(non_blocking=True)
+        self.y_host.copy_(self._run(xd), non_blocking=True)
+
+    def kernel_ms(self):
+        self.ev[-1][1].synchronize()
+        ms = [a.elapsed_time(b) for a, b in self.ev]
+        for li, m in enumerate(ms):
+            self.layer_ms[li].append(m)
+        return sum(ms)
+
+    def check(self):
+        pass
+
+    def extra(self, peaks):
+        """Per-layer time and fraction of the binding roofline (HBM bytes vs fp32 FMA rate)."""
+        import statistics
+        alu_peak = 148 * 128 * 2 * 1.965e9
+        rows = []
+        for li, L in enumerate(self.net["layers"]):
+            ms = statistics.mean(self.layer_ms[li]) if self.layer_ms[li] else None
+            t_hbm = self.layer_bytes[li] / (peaks["hbm_gbs"] * 1e9)
+            t_alu = self.layer_flops[li] / alu_peak
+            rows.append(dict(layer=li + 1, cout=L["cout"], cin=L["cin"], hw=L["hw"], ms=ms,
+                             bound="hbm" if t_hbm >= t_alu else "alu",
+                             frac=(max(t_hbm, t_alu) / (ms * 1e-3)) if ms else None))
+        return dict(layers=rows)
+
+    def oracle_sample(self):
+        from oracle import bcr_oracle as orc
+        L = self.net["layers"][7]  # conv 8 (256 -> 512 at 1/8 resolution): a mid-sized layer
+        hw = L["hw"]
+        x = np.maximum(np.random.default_rng(0).standard_normal((1, L["cin"], hw, hw)).astype(np.float32), 0)
+        t0 = time.perf_counter()
+        orc.conv2d(L["W"], L["mask"], x, L["bias"], ksize=3, stride=1, pad=1, relu=True, dtype=1)
+        dt = time.perf_counter() - t0
+        return 2.0 * int(L["mask"].sum()) * hw * hw / dt / 1e9, \
+            f"layer 8 of 13 on one image ({L['cin']}->{L['cout']} at {hw}x{hw}), direct fp64 NumPy convolution with the masked dense weight"
+
 
 def make_workload(args):
     w = args.workload
@@ -271,6 +376,8 @@ def make_workload(args):
         return SpmmWorkload(M=args.size, N=args.ncols, c=args.compression, bh=args.bh, bw=args.bw, dist=args.dist, bf16=args.bf16)
     if w == "conv":
         return ConvWorkload(batch=args.batch, bf16=args.bf16)
+    if w == "vgg":
+        return VggWorkload(batch=args.batch if args.batch != 32 else 1, image=args.image)
     raise SystemExit(f"unknown workload {w}")
 
 
@@ -376,17 +483,29 @@ def run_ours(args):
         value = world * wl.flops * args.steps / (total_ms * 1e-3) / 1e9
         e2e_value = world * wl.flops * args.steps / (e2e_ms * 1e-3) / 1e9
         k_ms = statistics.mean(kernel_ms)
-        if wl.bound == "hbm":
+        # binding roofline of the dominant kernel: the slower of (algorithmic bytes at the measured HBM bandwidth) and
+        # (effective flops 2*nnz*N at the peak of the unit that does the arithmetic: plain fp32 FMA pipes, derived as
+        # 148 SMs x 128 lanes x 2 flop x 1.965 GHz, or the measured dense bf16 tensor rate for the tcgen05 kernel)
+        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        flop_peak = peaks["bf16_tflops_burst"] if wl.peak_kind == "tensor" else alu_peak
+        t_hbm = wl.kernel_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_flop = wl.flops / (flop_peak * 1e12)
+        bound = getattr(wl, "force_bound", None) or ("hbm" if t_hbm >= t_flop else wl.peak_kind)
+        if bound == "hbm":
             achieved = wl.kernel_bytes / (k_ms * 1e-3) / 1e9
             roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
                         traffic=None, kernel=wl.kernel, kernel_ms=k_ms, algorithmic_bytes=wl.kernel_bytes,
                         peak_source=peaks["source"])
         else:
-            # plain fp32 FMA pipes: 148 SMs x 128 lanes x 2 flop x 1.965 GHz
-            peak = 148 * 128 * 2 * 1.965e9 / 1e12
             achieved = wl.flops / (k_ms * 1e-3) / 1e12
-            roof = dict(bound="alu", achieved=achieved, peak=peak, unit="TFLOP/s", frac=achieved / peak, traffic=None,
-                        kernel=wl.kernel, kernel_ms=k_ms, peak_source="derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz")
+            roof = dict(bound=bound, achieved=achieved, peak=flop_peak, unit="TFLOP/s", frac=achieved / flop_peak, traffic=None,
+                        kernel=wl.kernel, kernel_ms=k_ms,
+                        peak_source=("measured dense bf16 (burst)" if bound == "tensor"
+                                     else "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"))
+        roof["t_hbm_us"] = t_hbm * 1e6
+        roof["t_flop_us"] = t_flop * 1e6
+        if hasattr(wl, "extra"):
+            roof.update(wl.extra(peaks))
         cpu_v, cpu_what = wl.oracle_sample()
         line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
                     ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
@@ -410,7 +529,8 @@ def main():
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gru", choices=["gru", "gemv", "spmm", "conv"])
+    ap.add_argument("--workload", default="gru", choices=["gru", "gemv", "spmm", "conv", "vgg"])
+    ap.add_argument("--image", type=int, default=224)
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--ncols", type=int, default=128)
     ap.add_argument("--compression", type=float, default=8.0)

@@ -77,9 +77,10 @@ typedef struct {
   int32_t on_device;        /* 0 for GRIM_PACK_HOST_ONLY handles */
   int32_t reserved;
   int64_t value_bytes;      /* nnz * sizeof(value) */
-  int64_t index_bytes_spmm; /* bytes of block descriptors / tables read by the N > 1 kernels */
-  int64_t index_bytes_gemv; /* bytes of column words / chunk tables read by the N = 1 kernel */
+  int64_t index_bytes_spmm; /* bytes of headers / column lists / padding read by the register-tiled N > 16 kernel */
+  int64_t index_bytes_gemv; /* bytes of column words / chunk tables read by the N <= 16 kernel */
   int64_t export_bytes;     /* size of the canonical byte string written by grim_bcr_export */
+  int64_t index_bytes_tc;   /* bytes of column words / tables read by the tensor-core kernel (0: layout not built) */
 } grim_bcr_info_t;
 
 /* Tile-shape choice for the N > 1 kernel (Section 4.5: tile sizes are tuned per kernel).

@@ -52,7 +52,7 @@ class grim_bcr_info_t(C.Structure):
                 ("nbc", C.c_int64), ("nnz", C.c_int64), ("nonempty_blocks", C.c_int64), ("k_used", C.c_int64),
                 ("dtype", C.c_int32), ("flags", C.c_uint32), ("on_device", C.c_int32), ("reserved", C.c_int32),
                 ("value_bytes", C.c_int64), ("index_bytes_spmm", C.c_int64), ("index_bytes_gemv", C.c_int64),
-                ("export_bytes", C.c_int64)]
+                ("export_bytes", C.c_int64), ("index_bytes_tc", C.c_int64)]
 
 
 class grim_tune_t(C.Structure):

@@ -89,6 +89,17 @@ __device__ __forceinline__ void cp_async4_zfill(void* dst, const void* src, bool
   const unsigned n = valid ? 4u : 0u;
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
 }
+// One slab element: fp32 activations go through cp.async; bf16 activations are widened on the way (a 2-byte
+// cp.async does not exist), so the slab always holds fp32.
+__device__ __forceinline__ void gather_elem(float* dst, const void* X, int64_t off, bool valid, bool x_bf16) {
+  if (!x_bf16) {
+    cp_async4_zfill(dst, static_cast<const float*>(X) + (valid ? off : 0), valid);
+  } else {
+    unsigned short u = 0;
+    if (valid) u = __ldg(static_cast<const unsigned short*>(X) + off);
+    *dst = __uint_as_float((unsigned)u << 16);
+  }
+}
 __device__ __forceinline__ void cp_async16_cg(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
@@ -213,7 +224,8 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
         if (bytes[b]) bulk_load(base + p.slab_bytes + b * p.blob_stride, p.blob + (size_t)off[b] * 16, bytes[b], full + slot);
     } else {
       float* slab = reinterpret_cast<float*>(base);
-      const float* X = static_cast<const float*>(a.X);
+      const void* X = a.X;
+      const bool xb = a.x_dtype == GRIM_BF16;
       int64_t k = (int64_t)j * p.bw + kk0;
       if (a.conv) {
         const int khw = a.KH * a.KW;
@@ -223,8 +235,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
         for (int kk = kk0; kk < p.bw; kk += 4, k += 4) {
           const int ih = ih0 + kh, iw = iw0 + kw;
           const bool ok = q_ok && k < p.K && ih >= 0 && ih < a.H && iw >= 0 && iw < a.W;
-          const float* src = ok ? X + qoff + ((int64_t)c * a.H + kh) * a.W + kw : X;
-          cp_async4_zfill(slab + kk * sld + qq, src, ok);
+          gather_elem(slab + kk * sld + qq, X, qoff + ((int64_t)c * a.H + kh) * a.W + kw, ok, xb);
           kw += 4;
           while (kw >= a.KW) { kw -= a.KW; ++kh; }
           while (kh >= a.KH) { kh -= a.KH; ++c; }
@@ -232,7 +243,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
       } else if (a.x_sq == 1) {
         for (int kk = kk0; kk < p.bw; kk += 4, k += 4) {
           const bool ok = q_ok && k < p.K;
-          cp_async4_zfill(slab + kk * sld + qq, ok ? X + k * a.x_sk + qoff : X, ok);
+          gather_elem(slab + kk * sld + qq, X, k * a.x_sk + qoff, ok, xb);
         }
       } else {
         // X stored q-major: consecutive threads take consecutive k so that the reads coalesce; the padded row
@@ -241,7 +252,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
           const int kk = e % p.bw, qe = e / p.bw;
           const int64_t ke = (int64_t)j * p.bw + kk, q = q0 + qe;
           const bool ok = q < a.ncols && ke < p.K;
-          cp_async4_zfill(slab + kk * sld + qe, ok ? X + ke * a.x_sk + q * a.x_sq : X, ok);
+          gather_elem(slab + kk * sld + qe, X, ke * a.x_sk + q * a.x_sq, ok, xb);
         }
       }
 #pragma unroll
@@ -256,6 +267,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
         const uint8_t* src = p.blob + (size_t)off * 16;
         for (uint32_t i = tid * 16; i < bytes; i += kFThreads * 16) cp_async16_cg(dst + i, src + i);
       }
+      if (xb) __threadfence_block();  // the widened elements were written with ordinary stores
       cp_async_arrive_noinc(full + slot);
     }
   };
@@ -522,14 +534,13 @@ bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (h->nbc > kJlistCap || h->rc_max_blob == 0 || h->rc_max_blob > 0xFFFF * 16u) return false;
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTN) return false;
   const bool tma = tma_eligible(a);
-  if (!tma && a.x_dtype != GRIM_F32) return false;  // the gather loader moves 4-byte elements
-  return smem_need(h, 1, a.x_dtype == GRIM_F32 ? 4 : 2) <= kSmemBudget;
+  return smem_need(h, 1, (tma && a.x_dtype == GRIM_BF16) ? 2 : 4) <= kSmemBudget;
 }
 
 grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
   if (!ffma_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
   const bool tma = tma_eligible(a);
-  const int esz = a.x_dtype == GRIM_F32 ? 4 : 2;
+  const int esz = (tma && a.x_dtype == GRIM_BF16) ? 2 : 4;  // bytes per slab element (the gather loader widens bf16)
   const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);
   const int64_t qtiles = (a.ncols + kTN - 1) / kTN;
   // band groups per thread block: as many as the accumulators allow, fewer when the grid would not fill the GPU

@@ -464,6 +464,7 @@ extern "C" grim_status_t grim_bcr_info(grim_bcr_t h, grim_bcr_info_t* info) {
   info->index_bytes_spmm = h->index_bytes_rc;
   info->index_bytes_gemv = h->index_bytes_gemv;
   info->export_bytes = export_size(h);
+  info->index_bytes_tc = h->index_bytes_tc;
   return GRIM_OK;
 }
 
