@@ -136,6 +136,7 @@ extern "C" grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d
   a.bias = d->bias_dev; a.relu = (d->flags & GRIM_CONV_RELU) ? 1 : 0;
   a.conv = 1; a.C = (int)d->C; a.H = (int)d->H; a.W = (int)d->W; a.KH = d->KH; a.KW = d->KW;
   a.stride = d->stride; a.pad = d->pad; a.OH = (int)OH; a.OW = (int)OW;
+  if (tc_path_supported(h, a) && a.ncols >= 128) return launch_spmm_tc(h, a, (cudaStream_t)stream);
   if (ffma_path_supported(h, a)) return launch_ffma(h, a, (cudaStream_t)stream);
   return launch_spmm(h, a, (cudaStream_t)stream);
 }

@@ -30,6 +30,9 @@ constexpr int kTcGroups = 2;       // the workers form groups that take K tiles 
 constexpr int kTcGroupWarps = kTcWorkers / kTcGroups;
 constexpr int kTcGroupThreads = 32 * kTcGroupWarps;
 constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
+constexpr int kTcBuilders = 8;     // convolution only: warps that build the X tile from the NCHW input
+constexpr int kTcBuildGroupWarps = kTcBuilders / kTcGroups;
+constexpr int kTcConvThreads = kTcThreads + 32 * kTcBuilders;
 constexpr int kTM = 128;          // rows of W per thread block
 constexpr int kTQ = 256;          // output columns per thread block
 constexpr int kTK = 64;           // K per stage
@@ -48,6 +51,7 @@ struct TcParams {
   int bh_shift, slots_per_tile, nstages;
   uint32_t stage_bytes;
   unsigned spin_limit;
+  int64_t in_elems;  // convolution: elements of the input tensor
   SpmmArgs a;
 };
 
@@ -121,8 +125,8 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-template <int BH>
-__global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
+template <int BH, bool CONV>
+__global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
@@ -130,7 +134,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
   uint64_t* zeroed = full + kTcStages;                         // every worker has cleared its part of the weight tile
   uint64_t* ready = zeroed + kTcStages;                        // the expanded weight tile of a stage is written
   uint64_t* empty = ready + kTcStages;                         // the tensor core is done with a stage
-  uint64_t* acc_done = empty + kTcStages;                      // all multiplies of the tile are complete
+  uint64_t* built = empty + kTcStages;                         // convolution: the X tile of a stage is written
+  uint64_t* acc_done = built + kTcStages;                      // all multiplies of the tile are complete
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 192);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 196);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 256);  // [stage] bytes of the stage's packed record (0: none)
@@ -150,6 +155,7 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
       mbar_init(zeroed + s, kTcGroupWarps);
       mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
+      mbar_init(built + s, kTcBuildGroupWarps);
     }
     mbar_init(acc_done, 1);
     *s_abort = 0;
@@ -174,10 +180,12 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
         uint8_t* st = stages + (size_t)slot * stage_bytes;
         const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt];
         s_meta[slot] = se.bytes;
-        mbar_arrive_expect_tx(full + slot, kBTileBytes + se.bytes);
+        mbar_arrive_expect_tx(full + slot, (CONV ? 0u : (unsigned)kBTileBytes) + se.bytes);
+        if (!CONV) {
 #pragma unroll
-        for (int i = 0; i < kTQ / 64; ++i)
-          tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+          for (int i = 0; i < kTQ / 64; ++i)
+            tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+        }
         if (se.bytes) bulk_load(st + kATileBytes + kBTileBytes, p.blob + (size_t)se.off16 * 16, se.bytes, full + slot);
       }
     }
@@ -187,7 +195,8 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
       for (int kt = 0; kt < nkt; ++kt) {
         const int slot = kt % ns;
         const unsigned par = (unsigned)((kt / ns) & 1);
-        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort)) { failed = true; break; }
+        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort) ||
+            (CONV && !mbar_wait(built + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(stages + (size_t)slot * stage_bytes);
         const uint32_t b_addr = a_addr + kATileBytes;
@@ -202,6 +211,116 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
         umma_commit(empty + slot);  // arrives when the multiplies above have read their operands
       }
       if (!failed) umma_commit(acc_done);
+    }
+  } else if (CONV && warp >= 2 + kTcWorkers) {
+    // ------------------------------------------------------------------ implicit im2col (3x3, stride 1, pad 1)
+    // With W = OW the input element of tap (kh, kw) for output pixel pix is plane[pix + (kh-1)*W + (kw-1)], so a
+    // row of the X tile (one k = (c, kh, kw), 256 consecutive pixels) is a shifted copy of the input plane with
+    // zeros where the tap leaves the image.  A thread owns one 16-byte piece (8 pixels) of the row: it reads
+    // the two aligned 16-byte vectors that cover it, shifts, clears the out-of-image pixels (four byte masks,
+    // fixed per thread: pixel on the left / right / top / bottom edge) and stores the piece where the 128-byte
+    // swizzled N-major layout wants it.
+    const int bgrp = (warp - 2 - kTcWorkers) / kTcBuildGroupWarps;
+    const int bt = tid - kTcThreads - bgrp * (32 * kTcBuildGroupWarps);  // 0 .. 127 inside the group
+    const int cq = bt & 31;                                               // this thread's piece of the row
+    const int64_t qc = q0 + cq * 8;
+    const int ohw = a.OH * a.OW;
+    const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(a.X);
+    const int64_t in_elems = p.in_elems;
+    uint32_t m_left = 0, m_right = 0, m_top = 0, m_bottom = 0, m_off = 0;  // bit e: pixel e of the piece
+    int64_t img_of[2];   // image of the first pixel and of the last (a piece can cross into the next image)
+    int pix0;
+    {
+      const int64_t img = qc / ohw;
+      pix0 = (int)(qc - img * ohw);
+      img_of[0] = img;
+      img_of[1] = (qc + 7) / ohw;
+#pragma unroll
+      for (int e = 0; e < 8; ++e) {
+        const int64_t q = qc + e;
+        if (q >= a.ncols) { m_off |= 1u << e; continue; }
+        const int pe = (int)(q - (q / ohw) * ohw);
+        const int oh = pe / a.OW, ow = pe - oh * a.OW;
+        if (ow == 0) m_left |= 1u << e;
+        if (ow == a.OW - 1) m_right |= 1u << e;
+        if (oh == 0) m_top |= 1u << e;
+        if (oh == a.OH - 1) m_bottom |= 1u << e;
+      }
+    }
+    const int split = (img_of[1] != img_of[0]) ? (ohw - pix0) : 8;  // pixels of the piece that lie in the first image
+    const uint32_t panel_off = (uint32_t)(cq >> 3) * (64 * kTK * 2);  // 64-pixel panel of the tile
+    const uint32_t piece = (uint32_t)(cq & 7);
+    for (int kt = bgrp; kt < nkt; kt += kTcGroups) {
+      const int slot = kt % ns;
+      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
+      uint8_t* bt_base = stages + (size_t)slot * stage_bytes + kATileBytes + panel_off;
+      for (int kk = bt >> 5; kk < kTK; kk += kTcBuildGroupWarps) {
+        const int kg = kt * kTK + kk;
+        uint4 out = make_uint4(0u, 0u, 0u, 0u);
+        if (kg < p.K && m_off != 0xFFu) {
+          const int c = kg / 9, tap = kg - c * 9;
+          const int kh = tap / 3, kw = tap - kh * 3;
+          uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
+          if (bad != 0xFFu) {
+            const int shift = (kh - 1) * a.W + (kw - 1);
+            uint32_t w[4] = {0u, 0u, 0u, 0u};
+            if (split == 8) {
+              // element index of the piece's first pixel in the input tensor
+              const int64_t e0 = (img_of[0] * a.C + c) * (int64_t)ohw + pix0 + shift;
+              const int64_t v0 = e0 >> 3;  // floor: the vector that holds it (e0 may be negative at the very start)
+              const int sh = (int)(e0 - v0 * 8);
+              const uint4* in16 = reinterpret_cast<const uint4*>(in);
+              uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
+              if (v0 >= 0 && (v0 + 1) * 8 <= in_elems) lo = __ldg(in16 + v0);
+              if (sh != 0 && v0 + 1 >= 0 && (v0 + 2) * 8 <= in_elems) hi = __ldg(in16 + v0 + 1);
+              const bool tail = (v0 >= 0 && (v0 + 1) * 8 > in_elems) || (sh != 0 && v0 + 1 >= 0 && (v0 + 2) * 8 > in_elems);
+              if (tail) {
+                // the last vector of the tensor is incomplete: element-wise reads inside the tensor only
+                const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
+#pragma unroll
+                for (int e = 0; e < 8; ++e) {
+                  const int64_t ee = e0 + e;
+                  const uint32_t val = (ee >= 0 && ee < in_elems && !((bad >> e) & 1u)) ? in1[ee] : 0u;
+                  w[e >> 1] |= val << ((e & 1) * 16);
+                }
+              } else {
+                const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+                const int sw = sh >> 1, sb = (sh & 1) * 16;
+                uint32_t t[5];
+#pragma unroll
+                for (int i = 0; i < 5; ++i) {
+                  const uint32_t c0 = x[i], c1 = x[(i + 1) & 7], c2 = x[(i + 2) & 7], c3 = x[(i + 3) & 7];
+                  t[i] = sw == 0 ? c0 : (sw == 1 ? c1 : (sw == 2 ? c2 : c3));
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) w[i] = __funnelshift_r(t[i], t[i + 1], sb);
+              }
+            } else {
+              // the piece crosses an image boundary: element-wise
+              const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                const int64_t img = e < split ? img_of[0] : img_of[1];
+                const int pe = e < split ? pix0 + e : e - split;
+                const int64_t ee = (img * a.C + c) * (int64_t)ohw + pe + shift;
+                const uint32_t val = (!((bad >> e) & 1u) && ee >= 0 && ee < in_elems) ? in1[ee] : 0u;
+                w[e >> 1] |= val << ((e & 1) * 16);
+              }
+            }
+            // clear the pixels whose tap lies outside the image
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+              const uint32_t b2 = (bad >> (2 * i)) & 3u;
+              w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
+            }
+            out = make_uint4(w[0], w[1], w[2], w[3]);
+          }
+        }
+        *reinterpret_cast<uint4*>(bt_base + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4)) = out;
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0) mbar_arrive(built + slot);
     }
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
@@ -274,8 +393,23 @@ __global__ void __launch_bounds__(kTcThreads, 1) bcr_tc_kernel(const __grid_cons
           t[i] = __uint_as_float(v[i]) + bias;
           if (a.relu) t[i] = fmaxf(t[i], 0.f);
         }
-        const int64_t off0 = row * a.y_sr + q;
-        const bool full_chunk = q + 31 < a.ncols;
+        int64_t off0 = row * a.y_sr + q;
+        bool full_chunk = q + 31 < a.ncols;
+        if (CONV) {
+          // NCHW output: 32 consecutive pixels of one channel are contiguous while they stay inside one image
+          const int64_t ohw = (int64_t)a.OH * a.OW;
+          const int64_t img = q / ohw, pix = q - img * ohw;
+          off0 = (img * p.M + row) * ohw + pix;
+          if (pix + 31 >= ohw || !full_chunk) {
+            for (int i = 0; i < 32 && q + i < a.ncols; ++i) {
+              const int64_t im = (q + i) / ohw, px = (q + i) - im * ohw;
+              const int64_t o = (im * p.M + row) * ohw + px;
+              if (a.y_dtype == GRIM_F32) static_cast<float*>(a.Y)[o] = t[i];
+              else static_cast<__nv_bfloat16*>(a.Y)[o] = __float2bfloat16_rn(t[i]);
+            }
+            continue;
+          }
+        }
         if (a.y_dtype == GRIM_F32) {
           float* y = static_cast<float*>(a.Y) + off0;
           if (full_chunk && ((reinterpret_cast<uintptr_t>(y) & 15) == 0)) {
@@ -345,8 +479,13 @@ int tc_stages(const grim_bcr* h) {
 
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_tc_stage || !h->d_status) return false;
-  if (a.conv || a.x_dtype != GRIM_BF16 || a.x_sq != 1 || a.y_sq != 1) return false;
-  if (reinterpret_cast<uintptr_t>(a.X) % 16 != 0 || (a.x_sk * 2) % 16 != 0) return false;
+  if (a.x_dtype != GRIM_BF16 || reinterpret_cast<uintptr_t>(a.X) % 16 != 0) return false;
+  if (a.conv) {
+    // the tile builder covers the common same-size 3x3 convolution; other geometries use the CUDA-core kernel
+    if (a.KH != 3 || a.KW != 3 || a.stride != 1 || a.pad != 1 || a.OH != a.H || a.OW != a.W) return false;
+  } else if (a.x_sq != 1 || a.y_sq != 1 || (a.x_sk * 2) % 16 != 0) {
+    return false;
+  }
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
   if (tc_stages(h) == 0) return false;
   if (h->tc_mtiles > 65535) return false;
@@ -365,7 +504,18 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.spin_limit = 1u << 20;
   p.a = a;
 
+  p.in_elems = a.conv ? a.ncols / ((int64_t)a.OH * a.OW) * a.C * a.H * a.W : 0;
   CUtensorMap tm;
+  memset(&tm, 0, sizeof(tm));
+  if (a.conv) {
+    auto kern = h->bh == 4 ? bcr_tc_kernel<4, true> : (h->bh == 8 ? bcr_tc_kernel<8, true> : bcr_tc_kernel<16, true>);
+    const size_t smem = tc_smem_need(h, p.nstages);
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
+    dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)h->tc_mtiles);
+    kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+  }
   const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
   const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * 2)};
   const cuuint32_t box[2] = {64, (cuuint32_t)kTK};
@@ -375,7 +525,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
   const size_t smem = tc_smem_need(h, p.nstages);
-  auto kern = h->bh == 4 ? bcr_tc_kernel<4> : (h->bh == 8 ? bcr_tc_kernel<8> : bcr_tc_kernel<16>);
+  auto kern = h->bh == 4 ? bcr_tc_kernel<4, false> : (h->bh == 8 ? bcr_tc_kernel<8, false> : bcr_tc_kernel<16, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
