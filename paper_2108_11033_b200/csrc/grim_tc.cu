@@ -125,6 +125,20 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// Element-wise construction of one 8-pixel piece of an im2col row (pieces that cross into the next image or touch
+// the end of the tensor).  Kept out of line so that the common vector path stays short.
+__device__ __noinline__ uint4 im2col_piece_slow(const unsigned short* in1, int in_elems, int plane0, int plane1, int c_off,
+                                                int pix0, int split, int shift, uint32_t bad) {
+  uint32_t w[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+  for (int e = 0; e < 8; ++e) {
+    const int ee = (e < split ? plane0 + pix0 + e : plane1 + e - split) + c_off + shift;
+    const uint32_t val = (!((bad >> e) & 1u) && ee >= 0 && ee < in_elems) ? in1[ee] : 0u;
+    w[e >> 1] |= val << ((e & 1) * 16);
+  }
+  return make_uint4(w[0], w[1], w[2], w[3]);
+}
+
 template <int BH, bool CONV>
 __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -226,15 +240,14 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int64_t qc = q0 + cq * 8;
     const int ohw = a.OH * a.OW;
     const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(a.X);
-    const int64_t in_elems = p.in_elems;
+    const int in_elems = (int)p.in_elems;  // < 2^31 (checked on the host)
     uint32_t m_left = 0, m_right = 0, m_top = 0, m_bottom = 0, m_off = 0;  // bit e: pixel e of the piece
-    int64_t img_of[2];   // image of the first pixel and of the last (a piece can cross into the next image)
-    int pix0;
+    int plane0, plane1, pix0;  // element offsets of channel 0 of the image of the first / last pixel; first pixel
     {
-      const int64_t img = qc / ohw;
+      const int64_t img = qc / ohw, img1 = (qc + 7) / ohw;
       pix0 = (int)(qc - img * ohw);
-      img_of[0] = img;
-      img_of[1] = (qc + 7) / ohw;
+      plane0 = (int)(img * a.C * ohw);
+      plane1 = (int)(img1 * a.C * ohw);
 #pragma unroll
       for (int e = 0; e < 8; ++e) {
         const int64_t q = qc + e;
@@ -246,77 +259,77 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         if (oh == 0) m_top |= 1u << e;
         if (oh == a.OH - 1) m_bottom |= 1u << e;
       }
+      if (qc >= a.ncols) { plane0 = plane1 = 0; pix0 = 0; }
     }
-    const int split = (img_of[1] != img_of[0]) ? (ohw - pix0) : 8;  // pixels of the piece that lie in the first image
+    const int split = (plane1 != plane0) ? (ohw - pix0) : 8;  // pixels of the piece that lie in the first image
     const uint32_t panel_off = (uint32_t)(cq >> 3) * (64 * kTK * 2);  // 64-pixel panel of the tile
     const uint32_t piece = (uint32_t)(cq & 7);
+    const uint4* in16 = reinterpret_cast<const uint4*>(in);
+    const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
+    const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
     for (int kt = bgrp; kt < nkt; kt += kTcGroups) {
       const int slot = kt % ns;
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
       uint8_t* bt_base = stages + (size_t)slot * stage_bytes + kATileBytes + panel_off;
-      for (int kk = bt >> 5; kk < kTK; kk += kTcBuildGroupWarps) {
-        const int kg = kt * kTK + kk;
-        uint4 out = make_uint4(0u, 0u, 0u, 0u);
-        if (kg < p.K && m_off != 0xFFu) {
+      // The thread's 16 rows of the stage are taken in batches: first the address arithmetic and the vector loads
+      // of the whole batch (so that they are in flight together), then shifting, masking, storing.
+      constexpr int kBatch = 4;
+      for (int kk0 = bt >> 5; kk0 < kTK; kk0 += kTcBuildGroupWarps * kBatch) {
+        uint4 lo[kBatch], hi[kBatch];
+        uint32_t info[kBatch];  // bits 0-7: pixels to clear, 8-10: shift inside the vector, 12-13: 0 zeros / 1 vectors / 2 element-wise
+#pragma unroll
+        for (int bb = 0; bb < kBatch; ++bb) {
+          const int kk = kk0 + bb * kTcBuildGroupWarps;
+          const int kg = kt * kTK + kk;
+          lo[bb] = make_uint4(0u, 0u, 0u, 0u);
+          hi[bb] = make_uint4(0u, 0u, 0u, 0u);
+          info[bb] = 0;
+          if (kg >= p.K || m_off == 0xFFu) continue;
           const int c = kg / 9, tap = kg - c * 9;
           const int kh = tap / 3, kw = tap - kh * 3;
-          uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
-          if (bad != 0xFFu) {
-            const int shift = (kh - 1) * a.W + (kw - 1);
-            uint32_t w[4] = {0u, 0u, 0u, 0u};
-            if (split == 8) {
-              // element index of the piece's first pixel in the input tensor
-              const int64_t e0 = (img_of[0] * a.C + c) * (int64_t)ohw + pix0 + shift;
-              const int64_t v0 = e0 >> 3;  // floor: the vector that holds it (e0 may be negative at the very start)
-              const int sh = (int)(e0 - v0 * 8);
-              const uint4* in16 = reinterpret_cast<const uint4*>(in);
-              uint4 lo = make_uint4(0u, 0u, 0u, 0u), hi = make_uint4(0u, 0u, 0u, 0u);
-              if (v0 >= 0 && (v0 + 1) * 8 <= in_elems) lo = __ldg(in16 + v0);
-              if (sh != 0 && v0 + 1 >= 0 && (v0 + 2) * 8 <= in_elems) hi = __ldg(in16 + v0 + 1);
-              const bool tail = (v0 >= 0 && (v0 + 1) * 8 > in_elems) || (sh != 0 && v0 + 1 >= 0 && (v0 + 2) * 8 > in_elems);
-              if (tail) {
-                // the last vector of the tensor is incomplete: element-wise reads inside the tensor only
-                const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
-#pragma unroll
-                for (int e = 0; e < 8; ++e) {
-                  const int64_t ee = e0 + e;
-                  const uint32_t val = (ee >= 0 && ee < in_elems && !((bad >> e) & 1u)) ? in1[ee] : 0u;
-                  w[e >> 1] |= val << ((e & 1) * 16);
-                }
-              } else {
-                const uint32_t x[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
-                const int sw = sh >> 1, sb = (sh & 1) * 16;
-                uint32_t t[5];
-#pragma unroll
-                for (int i = 0; i < 5; ++i) {
-                  const uint32_t c0 = x[i], c1 = x[(i + 1) & 7], c2 = x[(i + 2) & 7], c3 = x[(i + 3) & 7];
-                  t[i] = sw == 0 ? c0 : (sw == 1 ? c1 : (sw == 2 ? c2 : c3));
-                }
-#pragma unroll
-                for (int i = 0; i < 4; ++i) w[i] = __funnelshift_r(t[i], t[i + 1], sb);
-              }
-            } else {
-              // the piece crosses an image boundary: element-wise
-              const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                const int64_t img = e < split ? img_of[0] : img_of[1];
-                const int pe = e < split ? pix0 + e : e - split;
-                const int64_t ee = (img * a.C + c) * (int64_t)ohw + pe + shift;
-                const uint32_t val = (!((bad >> e) & 1u) && ee >= 0 && ee < in_elems) ? in1[ee] : 0u;
-                w[e >> 1] |= val << ((e & 1) * 16);
-              }
-            }
-            // clear the pixels whose tap lies outside the image
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              const uint32_t b2 = (bad >> (2 * i)) & 3u;
-              w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
-            }
-            out = make_uint4(w[0], w[1], w[2], w[3]);
-          }
+          const uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
+          if (bad == 0xFFu) continue;
+          const int e0 = plane0 + c * ohw + pix0 + (kh - 1) * a.W + (kw - 1);
+          const int v0 = e0 >> 3;  // floor: the vector that holds the first pixel (negative at the very start)
+          const int sh = e0 & 7;
+          // pieces that cross into the next image, or whose vectors are not both complete vectors of the tensor
+          // (its very end), are built element by element
+          if (split != 8 || v0 + 1 >= nvec) { info[bb] = bad | (2u << 12); continue; }
+          if (v0 >= 0) lo[bb] = __ldg(in16 + v0);
+          if (sh != 0 && v0 + 1 >= 0) hi[bb] = __ldg(in16 + v0 + 1);
+          info[bb] = bad | ((uint32_t)sh << 8) | (1u << 12);
         }
-        *reinterpret_cast<uint4*>(bt_base + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4)) = out;
+#pragma unroll
+        for (int bb = 0; bb < kBatch; ++bb) {
+          const int kk = kk0 + bb * kTcBuildGroupWarps;
+          const uint32_t bad = info[bb] & 0xFFu, mode = info[bb] >> 12;
+          uint4 out = make_uint4(0u, 0u, 0u, 0u);
+          if (mode == 1u) {
+            const uint4 l = lo[bb], h = hi[bb];
+            const int sb = (int)((info[bb] >> 8) & 1u) * 16;
+            switch ((info[bb] >> 9) & 3u) {  // 32-bit word of the vector pair at which the piece starts
+              case 0: out = make_uint4(__funnelshift_r(l.x, l.y, sb), __funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb)); break;
+              case 1: out = make_uint4(__funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb)); break;
+              case 2: out = make_uint4(__funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb)); break;
+              default: out = make_uint4(__funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb), __funnelshift_r(h.z, h.w, sb)); break;
+            }
+            if (bad) {  // clear the pixels whose tap lies outside the image
+              uint32_t w[4] = {out.x, out.y, out.z, out.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                const uint32_t b2 = (bad >> (2 * i)) & 3u;
+                w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
+              }
+              out = make_uint4(w[0], w[1], w[2], w[3]);
+            }
+          } else if (mode == 2u) {
+            const int kg = kt * kTK + kk;
+            const int c = kg / 9, tap = kg - c * 9;
+            const int kh = tap / 3, kw = tap - kh * 3;
+            out = im2col_piece_slow(in1, in_elems, plane0, plane1, c * ohw, pix0, split, (kh - 1) * a.W + (kw - 1), bad);
+          }
+          *reinterpret_cast<uint4*>(bt_base + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4)) = out;
+        }
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
@@ -483,6 +496,7 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (a.conv) {
     // the tile builder covers the common same-size 3x3 convolution; other geometries use the CUDA-core kernel
     if (a.KH != 3 || a.KW != 3 || a.stride != 1 || a.pad != 1 || a.OH != a.H || a.OW != a.W) return false;
+    if (a.ncols / ((int64_t)a.OH * a.OW) * a.C * a.H * a.W >= (int64_t(1) << 31) - 64) return false;
   } else if (a.x_sq != 1 || a.y_sq != 1 || (a.x_sk * 2) % 16 != 0) {
     return false;
   }
