@@ -232,11 +232,12 @@ class ConvWorkload:
         self.y_host = torch.empty(self.batch, 512, 28, 28, dtype=tdt).pin_memory()
         i = B.grim_bcr_info(self.h)
         esz = 2 if self.bf16 else 4
-        self.kernel_bytes = float(i.value_bytes + i.index_bytes_spmm + self.x.numel() * esz + self.y.numel() * esz)
+        idx = i.index_bytes_tc if self.bf16 else i.index_bytes_spmm
+        self.kernel_bytes = float(i.value_bytes + idx + self.x.numel() * esz + self.y.numel() * esz)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * esz
-        self.kernel = "bcr_ffma_kernel (implicit im2col)"
-        self.peak_kind = "alu"
+        self.kernel = "bcr_tc_kernel (implicit im2col)" if self.bf16 else "bcr_ffma_kernel (implicit im2col)"
+        self.peak_kind = "tensor" if self.bf16 else "alu"
         self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
 
     def step(self):
@@ -276,8 +277,8 @@ class VggWorkload:
         self.dtype = "bf16"
         self.nnz = sum(int(L["mask"].sum()) for L in self.net["layers"])
         self.flops = sum(2.0 * int(L["mask"].sum()) * batch * L["hw"] * L["hw"] for L in self.net["layers"])
-        self.peak_kind = "alu"
-        self.kernel = "bcr_ffma_kernel (implicit im2col, per layer)"
+        self.peak_kind = "tensor"
+        self.kernel = "bcr_tc_kernel (implicit im2col, per layer)"
 
     def setup(self, B, torch):
         self.B, self.torch = B, torch
@@ -301,7 +302,7 @@ class VggWorkload:
         self.layer_bytes, self.layer_flops = [], []
         for L, i in zip(net["layers"], self.info):
             npx = self.batch * L["hw"] * L["hw"]
-            self.layer_bytes.append(float(i.value_bytes + i.index_bytes_spmm + 2 * L["cin"] * npx + 2 * L["cout"] * npx))
+            self.layer_bytes.append(float(i.value_bytes + i.index_bytes_tc + 2 * L["cin"] * npx + 2 * L["cout"] * npx))
             self.layer_flops.append(2.0 * i.nnz * npx)
         self.kernel_bytes = sum(self.layer_bytes)
         self.h2d = self.x_host.numel() * 2
@@ -341,16 +342,16 @@ class VggWorkload:
         pass
 
     def extra(self, peaks):
-        """Per-layer time and fraction of the binding roofline (HBM bytes vs fp32 FMA rate)."""
+        """Per-layer time and fraction of the binding roofline (HBM bytes vs the measured dense bf16 tensor rate)."""
         import statistics
-        alu_peak = 148 * 128 * 2 * 1.965e9
+        alu_peak = peaks["bf16_tflops_burst"] * 1e12
         rows = []
         for li, L in enumerate(self.net["layers"]):
             ms = statistics.mean(self.layer_ms[li]) if self.layer_ms[li] else None
             t_hbm = self.layer_bytes[li] / (peaks["hbm_gbs"] * 1e9)
             t_alu = self.layer_flops[li] / alu_peak
             rows.append(dict(layer=li + 1, cout=L["cout"], cin=L["cin"], hw=L["hw"], ms=ms,
-                             bound="hbm" if t_hbm >= t_alu else "alu",
+                             bound="hbm" if t_hbm >= t_alu else "tensor",
                              frac=(max(t_hbm, t_alu) / (ms * 1e-3)) if ms else None))
         return dict(layers=rows)
 
@@ -522,6 +523,72 @@ def run_ours(args):
     if world > 1:
         dist.destroy_process_group()
 
+def run_sweep(args):
+    """The SpMM sweep: square W with M = K in {1024, 4096, 8192}, N in {1, 16, 128, 1024}, compression in {4, 8, 16},
+    blocks in {4x16, 8x32, 16x64}, fp32 and bf16, kept-row counts uniform or Zipf(1.2), with and without reorder.
+    Writes one JSON line per run to --out and prints a one-line summary.  (--sweep-sizes etc. restrict the grid.)"""
+    import itertools
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2108_11033_b200.build import build_library
+    build_library()
+    from paper_2108_11033_b200 import binding as B
+    from workloads import generators as gen
+
+    peaks = measured_peaks()
+    alu_peak = 148 * 128 * 2 * 1.965e9
+    flush = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    sizes = [int(v) for v in args.sweep_sizes.split(",")]
+    ncols = [int(v) for v in args.sweep_ncols.split(",")]
+    comps = [float(v) for v in args.sweep_compressions.split(",")]
+    blocks = [tuple(int(t) for t in v.split("x")) for v in args.sweep_blocks.split(",")]
+    out = open(args.out, "w")
+    fracs, n_runs = [], 0
+    t_start = time.perf_counter()
+    for M, c, (bh, bw), dist_name in itertools.product(sizes, comps, blocks, ["uniform", "zipf"]):
+        W = gen.dense_weight(M, M, 5, 31)
+        mask = gen.bcr_mask(M, M, bh, bw, compression=c, dist=dist_name, seed=5, stream=32)
+        nnz = int(mask.sum())
+        Xf = gen.normal_f32((M, max(ncols)), 1.0, 5, 33)
+        for bf16, reorder in itertools.product([False, True], [1, 0]):
+            h = B.grim_bcr_pack(W, mask, bh, bw, B.GRIM_BF16 if bf16 else B.GRIM_F32, reorder)
+            info = B.grim_bcr_info(h)
+            esz = 2 if bf16 else 4
+            for N in ncols:
+                X = torch.from_numpy(np.ascontiguousarray(Xf[:, :N])).cuda()
+                if bf16:
+                    X = X.to(torch.bfloat16)
+                Y = torch.empty(M, N, device="cuda")
+                tc = bf16 and N >= 256
+                idx = info.index_bytes_gemv if N <= 16 else (info.index_bytes_tc if tc else info.index_bytes_spmm)
+                nbytes = float(info.value_bytes + idx + info.k_used * N * esz + M * N * 4)
+                flops = 2.0 * nnz * N
+                for _ in range(3):
+                    B.grim_bcr_spmm(h, X, Y)
+                ms = []
+                for _ in range(args.steps):
+                    flush.zero_()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    B.grim_bcr_spmm(h, X, Y)
+                    e1.record()
+                    e1.synchronize()
+                    ms.append(e0.elapsed_time(e1))
+                t = statistics.median(ms) * 1e-3
+                t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
+                t_flop = flops / (peaks["bf16_tflops_burst"] * 1e12 if tc else alu_peak)
+                rec = dict(M=M, N=N, c=c, block=f"{bh}x{bw}", dist=dist_name, dtype="bf16" if bf16 else "f32", reorder=reorder,
+                           nnz=nnz, ms=t * 1e3, gflops=flops / t / 1e9, bound="hbm" if t_hbm >= t_flop else ("tensor" if tc else "alu"),
+                           frac=max(t_hbm, t_flop) / t, kernel="skinny" if N <= 16 else ("tc" if tc else "ffma"))
+                out.write(json.dumps(rec) + "\n")
+                fracs.append(rec["frac"])
+                n_runs += 1
+            B.grim_bcr_destroy(h)
+        out.flush()
+    out.close()
+    print(json.dumps(dict(metric="SpMM sweep: fraction of the binding roofline", runs=n_runs, median_frac=statistics.median(fracs),
+                          min_frac=min(fracs), max_frac=max(fracs), wall_s=time.perf_counter() - t_start, out=args.out)))
+
 
 def main():
     ap = argparse.ArgumentParser()
@@ -539,7 +606,16 @@ def main():
     ap.add_argument("--dist", default="uniform", choices=["uniform", "zipf"])
     ap.add_argument("--bf16", action="store_true")
     ap.add_argument("--batch", type=int, default=32)
+    ap.add_argument("--sweep", action="store_true", help="run the SpMM sweep instead of one workload")
+    ap.add_argument("--sweep-sizes", default="1024,4096,8192")
+    ap.add_argument("--sweep-ncols", default="1,16,128,1024")
+    ap.add_argument("--sweep-compressions", default="4,8,16")
+    ap.add_argument("--sweep-blocks", default="4x16,8x32,16x64")
+    ap.add_argument("--out", default="sweep.jsonl")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.impl == "reference":
         run_reference(args)
     else:

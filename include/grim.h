@@ -219,6 +219,13 @@ grim_status_t grim_gru_seq(grim_gru_t g, const float* x_dev, int64_t T, const fl
 grim_status_t grim_gru_status(grim_gru_t g);
 grim_status_t grim_gru_destroy(grim_gru_t g);
 
+/* Layer pipelining of grim_gru_seq (execution detail, Section 4.2's concern with keeping all units busy; the paper
+ * has no multi-layer schedule).  With more than one layer the sequence is cut into `chunks` pieces in time and layer
+ * l works on piece k while layer l - 1 works on piece k + 1, each layer on an internal stream ordered by events; the
+ * caller's stream continues after the last layer.  chunks = 0 lets the library choose, 1 runs the layers one after the
+ * other on the caller's stream, at most 8.  Results do not depend on it. */
+grim_status_t grim_gru_set_pipeline(grim_gru_t g, int chunks);
+
 /* grim_gru_seq without any device allocation behind it.  (The paper has no counterpart: this entry
  * point exists for the way the library is deployed, not for the method.)
  *

@@ -32,7 +32,7 @@ EXPORTED = [
     "grim_bcr_pack", "grim_bcr_destroy", "grim_bcr_info", "grim_bcr_export", "grim_bcr_unpack_dense",
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
-    "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static",
+    "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
     "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version",
 ]
 
@@ -87,6 +87,7 @@ lib.grim_gru_status.argtypes = [_vp]
 lib.grim_gru_destroy.argtypes = [_vp]
 lib.grim_gru_debug_barrier.argtypes = [_vp, C.c_int, C.c_uint]
 lib.grim_gru_profile.argtypes = [_vp, C.c_int]
+lib.grim_gru_set_pipeline.argtypes = [_vp, C.c_int]
 lib.grim_gru_profile_read.argtypes = [_vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
 lib.grim_launch_count.restype = C.c_int64
 lib.grim_launch_count_reset.restype = None
@@ -249,6 +250,10 @@ def grim_gru_status(g: int) -> int:
 
 def grim_gru_debug_barrier(g: int, skip_cta: int, spin_limit: int):
     _check(lib.grim_gru_debug_barrier(g, skip_cta, spin_limit), "grim_gru_debug_barrier")
+
+
+def grim_gru_set_pipeline(g: int, chunks: int):
+    _check(lib.grim_gru_set_pipeline(g, chunks), "grim_gru_set_pipeline")
 
 
 def grim_gru_profile(g: int, enable: bool):

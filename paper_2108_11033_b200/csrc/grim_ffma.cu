@@ -10,8 +10,9 @@
 // A warp owns one band per group, a lane four output columns.  Per block the lane loads the slab rows of
 // eight kept columns into registers once (each needed input row is read once and reused by every kept row -
 // the load-redundancy idea of Section 4.4) and then, per kept row, reads the row's eight weights with two
-// broadcast 128-bit loads and issues 32 FMAs into that row's accumulators.  Which accumulator registers a
-// kept row uses is decided by one jump per (row, eight columns); everything inside is straight-line code.
+// broadcast 128-bit loads and issues 32 FMAs into that row's accumulators.  Accumulator registers are indexed
+// statically: the rows of the band are walked in order with one warp-uniform test of the block's row mask each.
+// Grids that would leave most SMs idle are split over block columns (partial sums added into a zeroed Y).
 #include <cuda.h>
 #include <cuda_bf16.h>
 

@@ -42,8 +42,15 @@ struct grim_gru {
   std::vector<const grim_bcr*> Wih, Whh;
   std::vector<float*> d_bih, d_bhh;
   std::vector<uint32_t*> d_pos_of_band;
-  float* d_gi = nullptr;
+  std::vector<float*> d_gi;  // per layer: hoisted pre-activations, T x 3H (layers overlap in time, so each has its own)
   float* d_seq[2] = {nullptr, nullptr};
+  // layer pipelining: layer l runs on its own stream, a chunk of time steps behind layer l - 1
+  std::vector<cudaStream_t> lstream;   // streams of layers 1 .. L-1 (layer 0 uses the caller's stream)
+  std::vector<cudaEvent_t> ev_chunk;   // [layer][chunk]: the layer's recurrence has produced the chunk
+  cudaEvent_t ev_fork = nullptr;
+  int max_chunks = 8;
+  bool pipeline = true;
+  int want_chunks = 0;  // 0: chosen from T
   unsigned* d_sync = nullptr;  // [0..L): barrier counters, [L]: status word
   ModeCfg grid, cluster;       // launch shapes of the shared-memory kernels
   ModeCfg regc;                // launch shape of the register-resident cluster kernel
@@ -54,7 +61,9 @@ struct grim_gru {
   unsigned spin_limit = 1u << 22;
   bool force_grid = false;
   bool profile = false;
-  std::vector<cudaEvent_t> ev;  // 3 per layer: before projection, before recurrent kernel, after it
+  std::vector<cudaEvent_t> ev;  // timing events, used in pairs: (before, after) each projection / recurrent launch
+  std::vector<int> ev_kind;     // 0 / 1: before / after a projection, 2 / 3: before / after a recurrent kernel
+  int ev_used = 0;
 };
 
 namespace {
@@ -573,7 +582,10 @@ void destroy(grim_gru* g) {
   for (float* p : g->d_bhh) cudaFree(p);
   for (uint32_t* p : g->d_pos_of_band) cudaFree(p);
   for (cudaEvent_t e : g->ev) cudaEventDestroy(e);
-  cudaFree(g->d_gi);
+  for (float* p : g->d_gi) cudaFree(p);
+  for (cudaStream_t st : g->lstream) cudaStreamDestroy(st);
+  for (cudaEvent_t e : g->ev_chunk) cudaEventDestroy(e);
+  if (g->ev_fork) cudaEventDestroy(g->ev_fork);
   cudaFree(g->d_seq[0]);
   cudaFree(g->d_seq[1]);
   cudaFree(g->d_sync);
@@ -582,6 +594,15 @@ void destroy(grim_gru* g) {
 
 constexpr size_t kSmemLimit = 200 * 1024;
 
+}  // namespace
+
+namespace {
+// Records the next timing event of the pool on stream s (profiling only).
+void profile_mark(grim_gru* g, int kind, cudaStream_t s) {
+  if (g->ev_used >= (int)g->ev.size()) return;
+  g->ev_kind[(size_t)g->ev_used] = kind;
+  cudaEventRecord(g->ev[(size_t)g->ev_used++], s);
+}
 }  // namespace
 
 extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, const grim_bcr_t* W_hh,
@@ -628,7 +649,23 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
       if (e != cudaSuccess) st = e == cudaErrorMemoryAllocation ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;
     }
     if (st == GRIM_OK) {
-      cudaError_t e = cudaMalloc((void**)&g->d_gi, (size_t)max_T * 3 * H * 4);
+      cudaError_t e = cudaSuccess;
+      for (int l = 0; l < layers && e == cudaSuccess; ++l) {
+        float* p = nullptr;
+        e = cudaMalloc((void**)&p, (size_t)max_T * 3 * H * 4);
+        if (e == cudaSuccess) g->d_gi.push_back(p);
+      }
+      for (int l = 1; l < layers && e == cudaSuccess; ++l) {
+        cudaStream_t st = nullptr;
+        e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking);
+        if (e == cudaSuccess) g->lstream.push_back(st);
+      }
+      for (int i = 0; i < layers * g->max_chunks && e == cudaSuccess; ++i) {
+        cudaEvent_t ev = nullptr;
+        e = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming);
+        if (e == cudaSuccess) g->ev_chunk.push_back(ev);
+      }
+      if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g->ev_fork, cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seq[0], (size_t)max_T * H * 4);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seq[1], (size_t)max_T * H * 4);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_sync, (size_t)(layers + 1) * 4);
@@ -702,39 +739,61 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
                                       grim_stream_t stream) {
   if (!g || !x || !y || T <= 0) return GRIM_ERR_INVALID_ARG;
   if (T > g->max_T) return GRIM_ERR_SHAPE;
-  cudaStream_t s = (cudaStream_t)stream;
-  g->last_stream = s;
+  cudaStream_t s0 = (cudaStream_t)stream;
+  g->last_stream = s0;
   const int64_t H = g->H;
+  const int L = g->L;
   // preference: weights in registers > cooperative grid > shared-memory cluster
   const bool want_grid = g->force_grid && g->grid.ok;
   const bool use_reg = g->regc.ok && !want_grid;
   const bool use_cluster = !use_reg && g->cluster.ok && !g->grid.ok;
   const ModeCfg& m = use_reg ? g->regc : (use_cluster ? g->cluster : g->grid);
   const int BHc = g->bh <= 4 ? 4 : (g->bh <= 8 ? 8 : 16);
-  if (cudaMemsetAsync(g->d_sync, 0, (size_t)(g->L + 1) * 4, s) != cudaSuccess) return GRIM_ERR_CUDA;
-  const float* seq_in = x;
-  for (int l = 0; l < g->L; ++l) {
-    const grim_bcr* wi = g->Wih[l];
-    // hoisted input projection: gi[t, :] = W_ih x_t + b_ih for all t (X given as T x in, output T x 3H)
+  if (cudaMemsetAsync(g->d_sync, 0, (size_t)(L + 1) * 4, s0) != cudaSuccess) return GRIM_ERR_CUDA;
+
+  // Time is cut into chunks; layer l works on chunk k while layer l - 1 works on chunk k + 1 (each layer on its own
+  // stream, ordered by events), so a stack of L layers takes about (1 + (L - 1) / chunks) single-layer times instead
+  // of L.  The kernels with a global barrier (fall-back) and single-layer models run as one chunk on one stream.
+  int chunks = 1;
+  if (g->pipeline && L > 1 && (use_reg || use_cluster))
+    chunks = g->want_chunks > 0 ? (int)std::min<int64_t>(g->want_chunks, T)
+                                : (int)std::max<int64_t>(1, std::min<int64_t>(3, T / 64));
+  const int64_t clen = (T + chunks - 1) / chunks;
+  auto stream_of = [&](int l) { return (chunks > 1 && l > 0) ? g->lstream[(size_t)l - 1] : s0; };
+  if (chunks > 1) {
+    if (cudaEventRecord(g->ev_fork, s0) != cudaSuccess) return GRIM_ERR_CUDA;
+    for (int l = 1; l < L; ++l)
+      if (cudaStreamWaitEvent(g->lstream[(size_t)l - 1], g->ev_fork, 0) != cudaSuccess) return GRIM_ERR_CUDA;
+  }
+  if (g->profile) g->ev_used = 0;
+
+  auto launch_projection = [&](int l, const float* seq_in, int64_t t0, int64_t n, cudaStream_t s) -> grim_status_t {
+    const grim_bcr* wi = g->Wih[(size_t)l];
+    // gi[t, :] = W_ih x_t + b_ih for the n steps from t0 (X given q-major as n x in, output n x 3H)
     SpmmArgs a;
-    a.X = seq_in; a.Y = g->d_gi; a.ncols = T;
+    a.X = seq_in + t0 * wi->K; a.Y = g->d_gi[(size_t)l] + t0 * 3 * H; a.ncols = n;
     a.x_sk = 1; a.x_sq = wi->K; a.y_sr = 1; a.y_sq = 3 * H;
-    a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32; a.bias = g->d_bih[l];
-    if (g->profile) cudaEventRecord(g->ev[3 * l], s);
-    grim_status_t st = ffma_path_supported(wi, a) ? launch_ffma(wi, a, s) : launch_spmm(wi, a, s);
-    if (st != GRIM_OK) return st;
-    if (g->profile) cudaEventRecord(g->ev[3 * l + 1], s);
-    float* seq_out = (l == g->L - 1) ? y : g->d_seq[l & 1];
-    const grim_bcr* wh = g->Whh[l];
+    a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32; a.bias = g->d_bih[(size_t)l];
+    if (g->profile) profile_mark(g, 0, s);
+    const grim_status_t st = ffma_path_supported(wi, a) ? launch_ffma(wi, a, s) : launch_spmm(wi, a, s);
+    if (g->profile) profile_mark(g, 1, s);
+    return st;
+  };
+  auto launch_recurrence = [&](int l, float* seq_out, int64_t t0, int64_t n, cudaStream_t s) -> grim_status_t {
+    const grim_bcr* wh = g->Whh[(size_t)l];
     GruParams p;
     p.band_ptr = wh->d_gemv_band_ptr; p.chunks = wh->d_chunks; p.colwords = wh->d_colwords;
-    p.vals = static_cast<const float*>(wh->d_gemv_vals); p.pos_of_band = g->d_pos_of_band[l];
-    p.b_hh = g->d_bhh[l]; p.gi = g->d_gi; p.h0 = h0 ? h0 + (int64_t)l * H : nullptr;
-    p.out = seq_out; p.hT = hT ? hT + (int64_t)l * H : nullptr;
-    p.bar = g->d_sync + l; p.status = g->d_sync + g->L;
-    p.H = (int)H; p.bh = g->bh; p.T = (int)T; p.tpc = m.tpc; p.ks = m.ks; p.resident = m.resident;
+    p.vals = static_cast<const float*>(wh->d_gemv_vals); p.pos_of_band = g->d_pos_of_band[(size_t)l];
+    p.b_hh = g->d_bhh[(size_t)l]; p.gi = g->d_gi[(size_t)l] + t0 * 3 * H;
+    // the state entering a later chunk is the previous chunk's last output row
+    p.h0 = t0 == 0 ? (h0 ? h0 + (int64_t)l * H : nullptr) : seq_out + (t0 - 1) * H;
+    p.out = seq_out + t0 * H;
+    p.hT = (hT && t0 + n == T) ? hT + (int64_t)l * H : nullptr;
+    p.bar = g->d_sync + l; p.status = g->d_sync + L;
+    p.H = (int)H; p.bh = g->bh; p.T = (int)n; p.tpc = m.tpc; p.ks = m.ks; p.resident = m.resident;
     p.max_chunks = m.max_chunks; p.max_cw = m.max_cw; p.max_vals = m.max_vals;
     p.skip_cta = g->dbg_skip_cta; p.spin_limit = g->spin_limit;
+    if (g->profile) profile_mark(g, 2, s);
     cudaError_t e;
     if (use_reg) {
       e = launch_cluster(reg_kernel(BHc, g->reg_ni, g->reg_s), m, p, s);
@@ -745,9 +804,39 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
       else if (g->bh <= 8) e = launch_grid<8>(g, p, s);
       else e = launch_grid<16>(g, p, s);
     }
+    if (g->profile) profile_mark(g, 3, s);
     if (e != cudaSuccess) { cudaGetLastError(); return e == cudaErrorCooperativeLaunchTooLarge ? GRIM_ERR_UNSUPPORTED : GRIM_ERR_CUDA; }
-    if (g->profile) cudaEventRecord(g->ev[3 * l + 2], s);
-    seq_in = seq_out;
+    return GRIM_OK;
+  };
+
+  // issue order: chunk-major over layers (a wavefront), so that every stream always has work queued
+  for (int k = 0; k < chunks + L - 1; ++k) {
+    for (int l = 0; l < L; ++l) {
+      const int c = k - l;  // the chunk layer l handles in this wave
+      if (c < 0 || c >= chunks) continue;
+      const int64_t t0 = (int64_t)c * clen, n = std::min<int64_t>(clen, T - t0);
+      if (n <= 0) continue;
+      cudaStream_t s = stream_of(l);
+      const float* seq_in = l == 0 ? x : g->d_seq[(l - 1) & 1];
+      float* seq_out = (l == L - 1) ? y : g->d_seq[l & 1];
+      grim_status_t st = GRIM_OK;
+      if (l == 0) {
+        if (c == 0) st = launch_projection(0, x, 0, T, s);  // the first layer's input is all there: one launch
+      } else {
+        if (chunks > 1 && cudaStreamWaitEvent(s, g->ev_chunk[(size_t)(l - 1) * g->max_chunks + c], 0) != cudaSuccess) return GRIM_ERR_CUDA;
+        st = launch_projection(l, seq_in, t0, n, s);
+      }
+      if (st != GRIM_OK) return st;
+      st = launch_recurrence(l, seq_out, t0, n, s);
+      if (st != GRIM_OK) return st;
+      if (chunks > 1 && cudaEventRecord(g->ev_chunk[(size_t)l * g->max_chunks + c], s) != cudaSuccess) return GRIM_ERR_CUDA;
+    }
+  }
+  if (chunks > 1) {
+    // join: the caller's stream continues when the last layer is done (lower layers finish earlier by construction,
+    // but their streams are joined too so that the handle's buffers are quiescent)
+    for (int l = 1; l < L; ++l)
+      if (cudaStreamWaitEvent(s0, g->ev_chunk[(size_t)l * g->max_chunks + chunks - 1], 0) != cudaSuccess) return GRIM_ERR_CUDA;
   }
   return GRIM_OK;
 }
@@ -773,26 +862,34 @@ extern "C" grim_status_t grim_gru_debug_barrier(grim_gru_t g, int skip_cta, unsi
   return GRIM_OK;
 }
 
+extern "C" grim_status_t grim_gru_set_pipeline(grim_gru_t g, int chunks) {
+  if (!g || chunks < 0 || chunks > g->max_chunks) return GRIM_ERR_INVALID_ARG;
+  g->pipeline = chunks != 1;
+  g->want_chunks = chunks;
+  return GRIM_OK;
+}
+
 extern "C" grim_status_t grim_gru_profile(grim_gru_t g, int enable) {
   if (!g) return GRIM_ERR_INVALID_ARG;
   if (enable && g->ev.empty()) {
-    g->ev.resize((size_t)3 * g->L);
+    g->ev.resize((size_t)4 * g->L * g->max_chunks);
+    g->ev_kind.assign(g->ev.size(), 0);
     for (cudaEvent_t& e : g->ev)
       if (cudaEventCreate(&e) != cudaSuccess) return GRIM_ERR_CUDA;
   }
   g->profile = enable != 0;
+  g->ev_used = 0;
   return GRIM_OK;
 }
 
 extern "C" grim_status_t grim_gru_profile_read(grim_gru_t g, float* projection_ms, float* recurrent_ms) {
   if (!g || !g->profile || g->ev.empty()) return GRIM_ERR_INVALID_ARG;
   float pj = 0.f, rc = 0.f;
-  for (int l = 0; l < g->L; ++l) {
-    float a = 0.f, b = 0.f;
-    if (cudaEventSynchronize(g->ev[3 * l + 2]) != cudaSuccess) return GRIM_ERR_CUDA;
-    if (cudaEventElapsedTime(&a, g->ev[3 * l], g->ev[3 * l + 1]) != cudaSuccess) return GRIM_ERR_CUDA;
-    if (cudaEventElapsedTime(&b, g->ev[3 * l + 1], g->ev[3 * l + 2]) != cudaSuccess) return GRIM_ERR_CUDA;
-    pj += a; rc += b;
+  for (int i = 0; i + 1 < g->ev_used; i += 2) {
+    float ms = 0.f;
+    if (cudaEventSynchronize(g->ev[(size_t)i + 1]) != cudaSuccess) return GRIM_ERR_CUDA;
+    if (cudaEventElapsedTime(&ms, g->ev[(size_t)i], g->ev[(size_t)i + 1]) != cudaSuccess) return GRIM_ERR_CUDA;
+    if (g->ev_kind[(size_t)i] == 0) pj += ms; else rc += ms;
   }
   if (projection_ms) *projection_ms = pj;
   if (recurrent_ms) *recurrent_ms = rc;
@@ -848,17 +945,21 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
     g_static_scratch_addr[dev] = static_cast<unsigned char*>(p);
   }
   unsigned char* base = g_static_scratch_addr[dev];
-  // Run the ordinary pass with the handle's scratch pointers pointing into the static array for the
-  // duration of the call.  Kernel arguments are copied at launch, so the handle can be put back at once.
-  float* const saved_gi = g->d_gi;
+  // Run the ordinary pass with the handle's scratch pointers pointing into the static array for the duration of
+  // the call (kernel arguments are copied at launch, so the handle can be put back at once).  All layers share one
+  // pre-activation buffer here, so the layers run one after the other on the caller's stream.
+  const std::vector<float*> saved_gi = g->d_gi;
   float* const saved_seq0 = g->d_seq[0];
   float* const saved_seq1 = g->d_seq[1];
-  g->d_gi = reinterpret_cast<float*>(base);
+  const bool saved_pipeline = g->pipeline;
+  for (float*& p : g->d_gi) p = reinterpret_cast<float*>(base);
   g->d_seq[0] = reinterpret_cast<float*>(base + gi_bytes);
   g->d_seq[1] = reinterpret_cast<float*>(base + gi_bytes + seq_bytes);
+  g->pipeline = false;
   const grim_status_t st = grim_gru_seq(g, x, T, h0, y, hT, stream);
   g->d_gi = saved_gi;
   g->d_seq[0] = saved_seq0;
   g->d_seq[1] = saved_seq1;
+  g->pipeline = saved_pipeline;
   return st;
 }

@@ -335,6 +335,25 @@ def test_vgg_stack_small_image_per_layer(B):
             cur = out
 
 
+@pytest.mark.parametrize("layer", [0, 1, 4, 8, 12])
+def test_vgg_full_size_layers(B, layer):
+    """Config-4 layers at their real 224x224 sizes (batch 1, the launch shapes the benchmark times): first layer
+    (K = 27, ragged), the widest pixel count, and one layer per resolution down to 14x14."""
+    net = gen.vgg16_stack(1)
+    L = net["layers"][layer]
+    x = gen.bf16_representable(np.maximum(gen.normal_f32((1, L["cin"], L["hw"], L["hw"]), 1.0, 93, layer), 0))
+    LL = dict(W=L["W"], mask=L["mask"], bias=L["bias"], bh=net["bh"], bw=net["bw"])
+    check_conv(B, LL, x, ksize=3, stride=1, pad=1, bf16=True, out_bf16=True)
+
+
+def test_conv_bf16_batch_crossing_images(B):
+    """Tensor-core convolution with an image size that is not a multiple of the 8-pixel pieces or of the 256-column
+    tile, several images, fp32 and bf16 outputs."""
+    L = gen.conv_layer(5, 24, 72, 15, ksize=3, bh=8, bw=32, compression=5, seed=94)
+    check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=True)
+    check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
+
+
 # ---------------------------------------------------------------------------------------- GRU
 
 
@@ -382,6 +401,30 @@ def test_gru_small(B, cfg):
 @pytest.mark.parametrize("grid_kernel", [False, True])
 def test_config2_gru_full(B, grid_kernel):
     check_gru(B, gen.gru_model(), grid_kernel=grid_kernel)
+
+
+@pytest.mark.parametrize("chunks", [1, 2, 5, 8])
+def test_gru_layer_pipelining_gives_the_same_result(B, chunks):
+    """Three layers cut into `chunks` pieces in time and run as a wavefront on internal streams: same outputs and
+    final states as the oracle, with and without an initial state, on a sequence length that does not divide."""
+    m = gen.gru_model(30, 128, 3, 53, bh=8, bw=32, compression=4, seed=95)
+    T, H, L = m["T"], m["hidden"], 3
+    g, handles = build_gru(B, m, T)
+    try:
+        B.grim_gru_set_pipeline(g, chunks)
+        h0 = gen.normal_f32((L, H), 0.5, 96, 0)
+        for init in (None, h0):
+            y = torch.full((T, H), float("nan"), device="cuda")
+            hT = torch.full((L, H), float("nan"), device="cuda")
+            B.grim_gru_seq(g, to_dev(m["x"]), y, h0=to_dev(init) if init is not None else None, hT=hT)
+            assert B.grim_gru_status(g) == B.GRIM_OK
+            want_y, want_h = orc.gru_seq(m["layers"], m["x"], h0=init)
+            assert rel_fro(y.cpu().numpy(), want_y) <= F32_TOL
+            assert rel_fro(hT.cpu().numpy(), want_h) <= F32_TOL
+    finally:
+        B.grim_gru_destroy(g)
+        for h in handles:
+            B.grim_bcr_destroy(h)
 
 
 def test_gru_bounded_wait_reports_timeout(B):
