@@ -590,7 +590,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   const size_t smem = smem_need(h, bpw, esz, p.slab_ld);
   dim3 grid((unsigned)qtiles, (unsigned)gy, (unsigned)ksplit);
   cudaError_t e = cudaSuccess;
-  if (ksplit > 1) {
+  if (ksplit > 1 && !(a.y_prefilled && !a.relu)) {
     e = zero_output(a, h->M, s);
     if (e != cudaSuccess) return GRIM_ERR_CUDA;
   }
@@ -601,7 +601,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
     e = launch_bh<float, kModeGather>(BHc, bpw, tm, p, smem, grid, s);
   }
   count_launch();
-  if (e == cudaSuccess && ksplit > 1 && (a.bias || a.relu)) {
+  if (e == cudaSuccess && ksplit > 1 && (a.bias || a.relu) && !(a.y_prefilled && !a.relu)) {
     const int64_t total = h->M * a.ncols;
     bcr_finalize_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8), 256, 0, s>>>(a, (int)h->M);
     count_launch();

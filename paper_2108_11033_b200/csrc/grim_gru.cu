@@ -42,6 +42,8 @@ struct grim_gru {
   std::vector<const grim_bcr*> Wih, Whh;
   std::vector<float*> d_bih, d_bhh;
   std::vector<uint32_t*> d_pos_of_band;
+  std::vector<float*> d_img_val;      // per layer: register image of the register-resident kernel (may be empty)
+  std::vector<uint32_t*> d_img_col;
   std::vector<float*> d_gi;  // per layer: hoisted pre-activations, T x 3H (layers overlap in time, so each has its own)
   float* d_seq[2] = {nullptr, nullptr};
   // layer pipelining: layer l runs on its own stream, a chunk of time steps behind layer l - 1
@@ -76,6 +78,7 @@ struct GruParams {
   const uint32_t* pos_of_band;
   const float* b_hh;
   const float* gi;   // T x 3H, b_ih already added
+  const float* b_ih; // 3H or null: added to gi here (not used by the register-resident kernel)
   const float* h0;   // H or null
   float* out;        // T x H
   float* hT;         // H or null
@@ -85,6 +88,10 @@ struct GruParams {
   uint32_t max_chunks, max_cw, max_vals;
   int skip_cta;
   unsigned spin_limit;
+  // register image of the register-resident kernel: what every thread keeps for the whole sequence, laid out
+  // so that the threads of a block read consecutive words ([cta][item][slot][row or column][thread])
+  const float* img_val;
+  const uint32_t* img_col;
 };
 
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
@@ -224,14 +231,17 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
   const int g_tri = tid / p.bh, g_r = tid % p.bh;
   const int unit = (blockIdx.x * p.tpc + g_tri) * p.bh + g_r;
   const bool gate_live = gate_thread && unit < p.H;
-  float bq[3] = {0.f, 0.f, 0.f};
+  float bq[3] = {0.f, 0.f, 0.f}, bi[3] = {0.f, 0.f, 0.f};
   if (gate_live)
-    for (int g = 0; g < 3; ++g) bq[g] = p.b_hh[g * p.H + unit];
+    for (int g = 0; g < 3; ++g) {
+      bq[g] = p.b_hh[g * p.H + unit];
+      if (p.b_ih) bi[g] = p.b_ih[g * p.H + unit];
+    }
 
   for (int t = 0; t < p.T; ++t) {
     float gi[3] = {0.f, 0.f, 0.f};
     if (gate_live)
-      for (int g = 0; g < 3; ++g) gi[g] = __ldg(p.gi + (int64_t)t * 3 * p.H + g * p.H + unit);
+      for (int g = 0; g < 3; ++g) gi[g] = __ldg(p.gi + (int64_t)t * 3 * p.H + g * p.H + unit) + bi[g];
     // h_{t-1}: written by other blocks during this launch -> read through L2
     const float* hprev = t == 0 ? p.h0 : p.out + (int64_t)(t - 1) * p.H;
     for (int i = tid; i < p.H; i += blockDim.x) hs[i] = hprev ? __ldcg(hprev + i) : 0.f;
@@ -284,9 +294,12 @@ __global__ void __launch_bounds__(1024, 1) gru_cluster_kernel(const GruParams p)
   const bool gate_live = tid < U;
   const int g_tri = tid / p.bh, g_r = tid % p.bh;
   const int unit = rank * U + tid;
-  float bq[3] = {0.f, 0.f, 0.f};
+  float bq[3] = {0.f, 0.f, 0.f}, bi[3] = {0.f, 0.f, 0.f};
   if (gate_live)
-    for (int g = 0; g < 3; ++g) bq[g] = p.b_hh[g * p.H + unit];
+    for (int g = 0; g < 3; ++g) {
+      bq[g] = p.b_hh[g * p.H + unit];
+      if (p.b_ih) bi[g] = p.b_ih[g * p.H + unit];
+    }
   for (int i = tid; i < p.H; i += blockDim.x) hs[i] = p.h0 ? p.h0[i] : 0.f;
   cluster.sync();  // every CTA of the cluster is resident and has initialised its buffers
 
@@ -295,7 +308,7 @@ __global__ void __launch_bounds__(1024, 1) gru_cluster_kernel(const GruParams p)
     float* hnxt_local = hs + ((t + 1) & 1) * p.H;
     float gi[3] = {0.f, 0.f, 0.f};
     if (gate_live)
-      for (int g = 0; g < 3; ++g) gi[g] = __ldg(p.gi + (int64_t)t * 3 * p.H + g * p.H + unit);
+      for (int g = 0; g < 3; ++g) gi[g] = __ldg(p.gi + (int64_t)t * 3 * p.H + g * p.H + unit) + bi[g];
     for (int item = warp; item < nb * p.ks; item += nwarps) band_gemv<BH>(v, hcur, partial, item / p.ks, item % p.ks, p.ks, lane);
     __syncthreads();
     if (gate_live) {
@@ -349,48 +362,20 @@ __global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const G
   float* hnew = hs + 2 * H;                   // [U]
   float* partial = hnew + ((U + 3) & ~3);     // [nb][2][BH]
 
-  // ---- one-time: pull this warp's items out of the chunk layout into registers
+  // ---- one-time: this thread's share of W_hh (built on the host when the handle was created): coalesced loads
   float val[NI][S][BH];
   uint32_t col[NI][S];
+  {
+    const float* iv = p.img_val + (size_t)rank * NI * S * BH * kRegThreads + tid;
+    const uint32_t* ic = p.img_col + (size_t)rank * NI * S * kRegThreads + tid;
 #pragma unroll
-  for (int i = 0; i < NI; ++i) {
-    const int item = warp * NI + i;
-    uint32_t cb = 0, ce = 0;
-    if (item < nb * 2) {
-      const int lb = item >> 1;
-      const int tri = rank * p.tpc + lb / 3;
-      const uint32_t pos = p.pos_of_band[(lb % 3) * nbands_gate + tri];
-      cb = p.band_ptr[pos];
-      ce = p.band_ptr[pos + 1];
-    }
-    uint32_t n = 0;
-    for (uint32_t c = cb; c < ce; ++c) n += p.chunks[c].ncols_kr & 0xFFFFu;
-    const uint32_t mid = (n + 1) >> 1;
-    const uint32_t c0 = (item & 1) ? mid : 0u, c1 = (item & 1) ? n : mid;
+    for (int i = 0; i < NI; ++i)
 #pragma unroll
-    for (int s = 0; s < S; ++s) {
-      col[i][s] = 0;
+      for (int s = 0; s < S; ++s) {
+        col[i][s] = __ldg(ic + (size_t)(i * S + s) * kRegThreads);
 #pragma unroll
-      for (int r = 0; r < BH; ++r) val[i][s][r] = 0.f;
-      const uint32_t ci = c0 + s * 32 + lane;
-      if (ci < c1) {
-        uint32_t prefix = 0, c = cb;
-        uint32_t nk = p.chunks[c].ncols_kr;
-        while (ci >= prefix + (nk & 0xFFFFu)) {
-          prefix += nk & 0xFFFFu;
-          ++c;
-          nk = p.chunks[c].ncols_kr;
-        }
-        const uint32_t l = ci - prefix, ncols = nk & 0xFFFFu;
-        const ChunkDesc cd = p.chunks[c];
-        const uint32_t w = p.colwords[cd.cw_off + l];
-        const uint32_t rm = w >> 16;
-        col[i][s] = w & 0xFFFFu;
-#pragma unroll
-        for (int r = 0; r < BH; ++r)
-          if ((rm >> r) & 1u) val[i][s][r] = p.vals[cd.val_off + __popc(rm & ((1u << r) - 1u)) * ncols + l];
+        for (int r = 0; r < BH; ++r) val[i][s][r] = __ldg(iv + (size_t)((i * S + s) * BH + r) * kRegThreads);
       }
-    }
   }
 
   const bool gate_live = tid < U;
@@ -483,10 +468,12 @@ cudaError_t launch_grid(const grim_gru* g, const GruParams& p, cudaStream_t s) {
 
 template <typename Kern>
 cudaError_t cluster_launch_config(Kern kern, const ModeCfg& m, cudaLaunchConfig_t* cfg, cudaLaunchAttribute* attr,
-                                  cudaStream_t s) {
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m.smem);
-  if (e == cudaSuccess && m.ctas > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
-  if (e != cudaSuccess) return e;
+                                  cudaStream_t s, bool set_attributes) {
+  if (set_attributes) {  // once, when the handle is created (the kernel keeps them)
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)m.smem);
+    if (e == cudaSuccess && m.ctas > 8) e = cudaFuncSetAttribute(kern, cudaFuncAttributeNonPortableClusterSizeAllowed, 1);
+    if (e != cudaSuccess) return e;
+  }
   *cfg = cudaLaunchConfig_t{};
   cfg->gridDim = dim3(m.ctas);
   cfg->blockDim = dim3(m.threads);
@@ -506,7 +493,7 @@ template <typename Kern>
 bool cluster_fits(Kern kern, const ModeCfg& m) {
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
-  if (cluster_launch_config(kern, m, &cfg, attr, nullptr) != cudaSuccess) { cudaGetLastError(); return false; }
+  if (cluster_launch_config(kern, m, &cfg, attr, nullptr, true) != cudaSuccess) { cudaGetLastError(); return false; }
   int n = 0;
   if (cudaOccupancyMaxActiveClusters(&n, kern, &cfg) != cudaSuccess) { cudaGetLastError(); return false; }
   return n >= 1;
@@ -516,7 +503,7 @@ template <typename Kern>
 cudaError_t launch_cluster(Kern kern, const ModeCfg& m, const GruParams& p, cudaStream_t s) {
   cudaLaunchConfig_t cfg;
   cudaLaunchAttribute attr[1];
-  cudaError_t e = cluster_launch_config(kern, m, &cfg, attr, s);
+  cudaError_t e = cluster_launch_config(kern, m, &cfg, attr, s, false);
   if (e != cudaSuccess) return e;
   e = cudaLaunchKernelEx(&cfg, kern, p);
   count_launch();
@@ -581,6 +568,8 @@ void destroy(grim_gru* g) {
   for (float* p : g->d_bih) cudaFree(p);
   for (float* p : g->d_bhh) cudaFree(p);
   for (uint32_t* p : g->d_pos_of_band) cudaFree(p);
+  for (float* p : g->d_img_val) cudaFree(p);
+  for (uint32_t* p : g->d_img_col) cudaFree(p);
   for (cudaEvent_t e : g->ev) cudaEventDestroy(e);
   for (float* p : g->d_gi) cudaFree(p);
   for (cudaStream_t st : g->lstream) cudaStreamDestroy(st);
@@ -597,6 +586,12 @@ constexpr size_t kSmemLimit = 200 * 1024;
 }  // namespace
 
 namespace {
+// out[t, :] = bias for t < T (n = row length, a multiple of 4).
+__global__ void fill_rows_kernel(float* __restrict__ out, const float* __restrict__ bias, int64_t T, int64_t n) {
+  const int64_t total4 = T * n / 4, n4 = n / 4;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total4; i += (int64_t)gridDim.x * blockDim.x)
+    reinterpret_cast<float4*>(out)[i] = __ldg(reinterpret_cast<const float4*>(bias) + i % n4);
+}
 // Records the next timing event of the pool on stream s (profiling only).
 void profile_mark(grim_gru* g, int kind, cudaStream_t s) {
   if (g->ev_used >= (int)g->ev.size()) return;
@@ -725,7 +720,65 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
           break;
         }
       }
-      if (!g->grid.ok && !g->cluster.ok && !g->regc.ok) st = GRIM_ERR_UNSUPPORTED;
+      if (g->regc.ok) {
+        // register image: for every thread of every CTA the columns it owns (global index + values at row positions)
+        const int NI = g->reg_ni, S = g->reg_s, tpc = g->regc.tpc, cs = g->regc.ctas, nbb = 3 * tpc;
+        const size_t nval = (size_t)cs * NI * S * BHc * kRegThreads, ncol = (size_t)cs * NI * S * kRegThreads;
+        std::vector<float> iv(nval);
+        std::vector<uint32_t> ic(ncol);
+        struct ColRec { uint32_t col; float v[16]; };
+        std::vector<ColRec> cols;
+        for (int l = 0; l < layers && st == GRIM_OK; ++l) {
+          const grim_bcr* wh = W_hh[l];
+          std::fill(iv.begin(), iv.end(), 0.f);
+          std::fill(ic.begin(), ic.end(), 0u);
+          for (int rank = 0; rank < cs; ++rank)
+            for (int lb = 0; lb < nbb; ++lb) {
+              const int64_t band = (int64_t)(lb % 3) * ntri + (int64_t)rank * tpc + lb / 3;
+              cols.clear();
+              for (int64_t j = 0; j < wh->nbc; ++j) {
+                const HostBlock& hb = wh->blocks[(size_t)(band * wh->nbc + j)];
+                if (!(hb.kr && hb.kc)) continue;
+                int bidx = 0;
+                for (int c = 0; c < wh->bw; ++c) {
+                  if (!((hb.colmask >> c) & 1ull)) continue;
+                  ColRec cr;
+                  cr.col = (uint32_t)(j * wh->bw + c);
+                  int a = 0;
+                  for (int r = 0; r < 16; ++r) {
+                    cr.v[r] = 0.f;
+                    if ((hb.rowmask >> r) & 1u) cr.v[r] = wh->vals[(size_t)hb.val_off + (size_t)(a++) * hb.kc + (size_t)bidx];
+                  }
+                  cols.push_back(cr);
+                  ++bidx;
+                }
+              }
+              const size_t n = cols.size(), mid = (n + 1) / 2;
+              for (int half = 0; half < 2; ++half) {
+                const int item = lb * 2 + half, warp = item / NI, i = item % NI;
+                const size_t c0 = half ? mid : 0, c1 = half ? n : mid;
+                for (size_t ci = c0; ci < c1; ++ci) {
+                  const size_t k = ci - c0;
+                  const int sl = (int)(k / 32), lane = (int)(k % 32);
+                  if (sl >= S || warp >= kRegWarps) { st = GRIM_ERR_UNSUPPORTED; break; }
+                  const int tid = warp * 32 + lane;
+                  ic[((size_t)(rank * NI + i) * S + sl) * kRegThreads + tid] = cols[ci].col;
+                  for (int r = 0; r < BHc; ++r)
+                    iv[(((size_t)(rank * NI + i) * S + sl) * BHc + r) * kRegThreads + tid] = cols[ci].v[r];
+                }
+              }
+            }
+          if (st != GRIM_OK) break;
+          float* dv = nullptr;
+          uint32_t* dc = nullptr;
+          cudaError_t e = cudaMalloc((void**)&dv, nval * 4);
+          if (e == cudaSuccess) { g->d_img_val.push_back(dv); e = cudaMalloc((void**)&dc, ncol * 4); }
+          if (e == cudaSuccess) { g->d_img_col.push_back(dc); e = cudaMemcpy(dv, iv.data(), nval * 4, cudaMemcpyHostToDevice); }
+          if (e == cudaSuccess) e = cudaMemcpy(dc, ic.data(), ncol * 4, cudaMemcpyHostToDevice);
+          if (e != cudaSuccess) st = e == cudaErrorMemoryAllocation ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;
+        }
+      }
+      if (st == GRIM_OK && !g->grid.ok && !g->cluster.ok && !g->regc.ok) st = GRIM_ERR_UNSUPPORTED;
     }
   } catch (const std::bad_alloc&) {
     st = GRIM_ERR_ALLOC;
@@ -766,6 +819,17 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
       if (cudaStreamWaitEvent(g->lstream[(size_t)l - 1], g->ev_fork, 0) != cudaSuccess) return GRIM_ERR_CUDA;
   }
   if (g->profile) g->ev_used = 0;
+  // every row of a pre-activation buffer starts as b_ih: the projections may add partial sums onto it
+  auto prefill = [&](int l, cudaStream_t s) {
+    const int64_t total = T * 3 * H;
+    fill_rows_kernel<<<(unsigned)std::min<int64_t>((total / 4 + 255) / 256, 148 * 8), 256, 0, s>>>(g->d_gi[(size_t)l], g->d_bih[(size_t)l], T, 3 * H);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess;
+  };
+  for (int l = 0; l < L; ++l) {
+    if (l > 0 && g->d_gi[(size_t)l] == g->d_gi[0]) break;  // one shared buffer: filled per layer, below
+    if (!prefill(l, stream_of(l))) return GRIM_ERR_CUDA;
+  }
 
   auto launch_projection = [&](int l, const float* seq_in, int64_t t0, int64_t n, cudaStream_t s) -> grim_status_t {
     const grim_bcr* wi = g->Wih[(size_t)l];
@@ -773,7 +837,10 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     SpmmArgs a;
     a.X = seq_in + t0 * wi->K; a.Y = g->d_gi[(size_t)l] + t0 * 3 * H; a.ncols = n;
     a.x_sk = 1; a.x_sq = wi->K; a.y_sr = 1; a.y_sq = 3 * H;
-    a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32; a.bias = g->d_bih[(size_t)l];
+    a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32;
+    a.bias = g->d_bih[(size_t)l];
+    a.y_prefilled = 1;  // every row of the buffer already holds b_ih (below): a split multiply adds onto it and
+                        // needs neither its own clearing nor a bias pass; an unsplit one writes sum + bias as usual
     if (g->profile) profile_mark(g, 0, s);
     const grim_status_t st = ffma_path_supported(wi, a) ? launch_ffma(wi, a, s) : launch_spmm(wi, a, s);
     if (g->profile) profile_mark(g, 1, s);
@@ -784,7 +851,7 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     GruParams p;
     p.band_ptr = wh->d_gemv_band_ptr; p.chunks = wh->d_chunks; p.colwords = wh->d_colwords;
     p.vals = static_cast<const float*>(wh->d_gemv_vals); p.pos_of_band = g->d_pos_of_band[(size_t)l];
-    p.b_hh = g->d_bhh[(size_t)l]; p.gi = g->d_gi[(size_t)l] + t0 * 3 * H;
+    p.b_hh = g->d_bhh[(size_t)l]; p.b_ih = nullptr; p.gi = g->d_gi[(size_t)l] + t0 * 3 * H;
     // the state entering a later chunk is the previous chunk's last output row
     p.h0 = t0 == 0 ? (h0 ? h0 + (int64_t)l * H : nullptr) : seq_out + (t0 - 1) * H;
     p.out = seq_out + t0 * H;
@@ -793,6 +860,8 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     p.H = (int)H; p.bh = g->bh; p.T = (int)n; p.tpc = m.tpc; p.ks = m.ks; p.resident = m.resident;
     p.max_chunks = m.max_chunks; p.max_cw = m.max_cw; p.max_vals = m.max_vals;
     p.skip_cta = g->dbg_skip_cta; p.spin_limit = g->spin_limit;
+    p.img_val = use_reg ? g->d_img_val[(size_t)l] : nullptr;
+    p.img_col = use_reg ? g->d_img_col[(size_t)l] : nullptr;
     if (g->profile) profile_mark(g, 2, s);
     cudaError_t e;
     if (use_reg) {
@@ -820,6 +889,8 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
       const float* seq_in = l == 0 ? x : g->d_seq[(l - 1) & 1];
       float* seq_out = (l == L - 1) ? y : g->d_seq[l & 1];
       grim_status_t st = GRIM_OK;
+      if (l > 0 && c == 0 && g->d_gi[(size_t)l] == g->d_gi[0] && !prefill(l, s))
+        return GRIM_ERR_CUDA;  // layers share one buffer (allocation-free variant): fill it again for this layer
       if (l == 0) {
         if (c == 0) st = launch_projection(0, x, 0, T, s);  // the first layer's input is all there: one launch
       } else {

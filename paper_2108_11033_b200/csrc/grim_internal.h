@@ -151,6 +151,8 @@ struct SpmmArgs {
   int conv = 0;
   int C = 0, H = 0, W = 0, KH = 0, KW = 0, stride = 1, pad = 0, OH = 0, OW = 0;
   int tile_n = 0;  // 0 = default
+  int y_prefilled = 0;  // Y already holds the bias in every column: a split multiply adds onto it (no clearing, no
+                        // bias pass; not with relu); an unsplit multiply ignores the flag
 };
 
 grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
