@@ -29,6 +29,15 @@ if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
 METRIC = "BCR SpMM/GEMV effective GFLOP/s (2*nnz*N)"
+
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes) of the dominant kernel per step, from one ncu
+# capture of the same command (summaries under profiles/); None where the kernel has changed since or was not captured.
+TRAFFIC = {
+    "gru_2x1024_in153_T200_bcr8x32_c10_fp32": 6 * 3.514e6,  # six launches (2 layers x 3 chunks) of 3.5 MB each
+    "spmm_M4096_K4096_N1024_c8_8x32_uniform_fp32": 27.68e6,
+    "spmm_M8192_K8192_N1_c4_8x32_uniform_fp32": 87.46e6,
+    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.70e6,
+}
 UNIT = "GFLOP/s"
 
 
@@ -503,6 +512,7 @@ def run_ours(args):
                         kernel=wl.kernel, kernel_ms=k_ms,
                         peak_source=("measured dense bf16 (burst)" if bound == "tensor"
                                      else "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"))
+        roof["traffic"] = TRAFFIC.get(wl.name)
         roof["t_hbm_us"] = t_hbm * 1e6
         roof["t_flop_us"] = t_flop * 1e6
         if hasattr(wl, "extra"):
