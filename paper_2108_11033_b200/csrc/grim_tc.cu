@@ -25,13 +25,14 @@
 namespace grim {
 namespace {
 
-constexpr int kTcWorkers = 8;      // warps that expand the packed weights and later run the epilogue
-constexpr int kTcGroups = 2;       // the workers form groups that take K tiles in turn, so that expansions overlap
+constexpr int kTcWorkers = 12;     // warps that expand the packed weights; the first eight also run the epilogue
+constexpr int kTcGroups = 3;       // the workers form groups that take K tiles in turn, so that expansions overlap
 constexpr int kTcGroupWarps = kTcWorkers / kTcGroups;
 constexpr int kTcGroupThreads = 32 * kTcGroupWarps;
 constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
 constexpr int kTcBuilders = 8;     // convolution only: warps that build the X tile from the NCHW input
-constexpr int kTcBuildGroupWarps = kTcBuilders / kTcGroups;
+constexpr int kTcBuildGroups = 2;
+constexpr int kTcBuildGroupWarps = kTcBuilders / kTcBuildGroups;
 constexpr int kTcConvThreads = kTcThreads + 32 * kTcBuilders;
 constexpr int kTM = 128;          // rows of W per thread block
 constexpr int kTQ = 256;          // output columns per thread block
@@ -40,6 +41,8 @@ constexpr int kTcStages = 4;        // ring slots at most; fewer when the packed
 constexpr int kATileBytes = kTM * kTK * 2;   // 16 KiB
 constexpr int kBTileBytes = kTQ * kTK * 2;   // 32 KiB
 constexpr int kTcHdrBytes = 1024;
+constexpr int kTcRecSlots = 8;      // ring of packed records (small), deeper than the ring of tiles so that records
+                                    // are on chip well before the weight tile they expand into becomes free
 constexpr unsigned kTmemCols = 256;
 
 struct TcParams {
@@ -48,8 +51,8 @@ struct TcParams {
   const uint32_t* band_order;
   unsigned* status;
   int nbr, M, K, bh, nkt;
-  int bh_shift, slots_per_tile, nstages;
-  uint32_t stage_bytes;
+  int bh_shift, slots_per_tile, nstages, nrec;
+  uint32_t stage_bytes, rec_stride;
   unsigned spin_limit;
   int64_t in_elems;  // convolution: elements of the input tensor
   SpmmArgs a;
@@ -144,24 +147,27 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   extern __shared__ uint8_t smem_raw[];
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // copies of a stage have landed
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // the X tile of a stage has landed
   uint64_t* zeroed = full + kTcStages;                         // every worker has cleared its part of the weight tile
   uint64_t* ready = zeroed + kTcStages;                        // the expanded weight tile of a stage is written
   uint64_t* empty = ready + kTcStages;                         // the tensor core is done with a stage
   uint64_t* built = empty + kTcStages;                         // convolution: the X tile of a stage is written
   uint64_t* acc_done = built + kTcStages;                      // all multiplies of the tile are complete
-  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 192);
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 196);
-  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 256);  // [stage] bytes of the stage's packed record (0: none)
+  uint64_t* rec_full = acc_done + 1;                           // a packed record has landed
+  uint64_t* rec_empty = rec_full + kTcRecSlots;                // a packed record has been expanded
+  uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
+  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 512);  // [record slot] bytes of the packed record (0: none)
   uint8_t* stages = smem + kTcHdrBytes;
   const uint32_t stage_bytes = p.stage_bytes;
+  uint8_t* recs = stages + (size_t)p.nstages * stage_bytes;
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   const SpmmArgs& a = p.a;
   const int64_t q0 = (int64_t)blockIdx.x * kTQ;
   const int pos0 = blockIdx.y * p.slots_per_tile;  // first band (schedule position) of this tile
-  const int nkt = p.nkt, ns = p.nstages;
+  const int nkt = p.nkt, ns = p.nstages, nr = p.nrec;
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
@@ -170,6 +176,10 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
       mbar_init(built + s, kTcBuildGroupWarps);
+    }
+    for (int s = 0; s < kTcRecSlots; ++s) {
+      mbar_init(rec_full + s, 1);
+      mbar_init(rec_empty + s, kTcGroupWarps);
     }
     mbar_init(acc_done, 1);
     *s_abort = 0;
@@ -188,19 +198,22 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   if (warp == 0) {
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
-      for (int kt = 0; kt < nkt; ++kt) {
+      // the first records (the ring of records is deeper than the ring of tiles); later ones are requested by the
+      // expansion warps as they free a record slot
+      for (int rk = 0; rk < nr && rk < nkt; ++rk) {
+        const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + rk];
+        s_meta[rk] = se.bytes;
+        mbar_arrive_expect_tx(rec_full + rk, se.bytes);
+        if (se.bytes) bulk_load(recs + (size_t)rk * p.rec_stride, p.blob + (size_t)se.off16 * 16, se.bytes, rec_full + rk);
+      }
+      for (int kt = 0; kt < nkt && !CONV; ++kt) {  // the convolution builds its X tiles itself
         const int slot = kt % ns;
         if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
         uint8_t* st = stages + (size_t)slot * stage_bytes;
-        const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt];
-        s_meta[slot] = se.bytes;
-        mbar_arrive_expect_tx(full + slot, (CONV ? 0u : (unsigned)kBTileBytes) + se.bytes);
-        if (!CONV) {
+        mbar_arrive_expect_tx(full + slot, (unsigned)kBTileBytes);
 #pragma unroll
-          for (int i = 0; i < kTQ / 64; ++i)
-            tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
-        }
-        if (se.bytes) bulk_load(st + kATileBytes + kBTileBytes, p.blob + (size_t)se.off16 * 16, se.bytes, full + slot);
+        for (int i = 0; i < kTQ / 64; ++i)
+          tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
       }
     }
   } else if (warp == 1) {
@@ -209,7 +222,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       for (int kt = 0; kt < nkt; ++kt) {
         const int slot = kt % ns;
         const unsigned par = (unsigned)((kt / ns) & 1);
-        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort) ||
+        if ((!CONV && !mbar_wait(full + slot, par, p.spin_limit, s_abort)) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort) ||
             (CONV && !mbar_wait(built + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(stages + (size_t)slot * stage_bytes);
@@ -267,7 +280,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const uint4* in16 = reinterpret_cast<const uint4*>(in);
     const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
     const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
-    for (int kt = bgrp; kt < nkt; kt += kTcGroups) {
+    for (int kt = bgrp; kt < nkt; kt += kTcBuildGroups) {
       const int slot = kt % ns;
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
       uint8_t* bt_base = stages + (size_t)slot * stage_bytes + kATileBytes + panel_off;
@@ -340,9 +353,12 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int grp = (warp - 2) / kTcGroupWarps;               // this warp's group
     const int wt = tid - 64 - grp * kTcGroupThreads;           // 0 .. kTcGroupThreads - 1 inside the group
     for (int kt = grp; kt < nkt; kt += kTcGroups) {
-      const int slot = kt % ns;
+      const int slot = kt % ns, rs = kt % nr;
       const unsigned par = (unsigned)((kt / ns) & 1);
-      if (!__all_sync(0xffffffffu, mbar_wait(full + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
+      // the weight tile of the slot is free once the multiplies of its previous use are done; the record is
+      // normally long there
+      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
       uint4* a4 = reinterpret_cast<uint4*>(st);
 #pragma unroll
@@ -350,11 +366,11 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       __syncwarp();
       if (lane == 0) mbar_arrive(zeroed + slot);
       if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
-      if (s_meta[slot]) {
+      if (s_meta[rs]) {
         // a thread takes kept columns of the tile and drops each column's values into the swizzled K-major tile
         // (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits).  All loads of a column are
         // issued before its stores: the value of row r sits popcount(mask below r) places after the first
-        const uint32_t* rec = reinterpret_cast<const uint32_t*>(st + kATileBytes + kBTileBytes);
+        const uint32_t* rec = reinterpret_cast<const uint32_t*>(recs + (size_t)rs * p.rec_stride);
         const int ncols = (int)rec[0];
         const uint32_t* cw = rec + 4;
         const uint16_t* vo = reinterpret_cast<const uint16_t*>(cw + ((ncols + 3) & ~3));
@@ -378,13 +394,28 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       }
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(ready + slot);
+      if (lane == 0) {
+        mbar_arrive(ready + slot);
+        mbar_arrive(rec_empty + rs);
+      }
+      if (wt == 0 && kt + nr < nkt) {
+        // the record slot is free once every warp of the group is done with it: request the record that uses it next
+        if (!mbar_wait(rec_empty + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort)) failed = true;
+        else {
+          const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt + nr];
+          s_meta[rs] = se.bytes;
+          mbar_arrive_expect_tx(rec_full + rs, se.bytes);
+          if (se.bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)se.off16 * 16, se.bytes, rec_full + rs);
+        }
+      }
+      if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     }
     // ------------------------------------------------------------------ epilogue
-    if (!__any_sync(0xffffffffu, failed)) {
+    const bool epilogue_warp = warp - 2 < 8;  // two warps per quarter of the tensor-memory lanes
+    if (epilogue_warp && !__any_sync(0xffffffffu, failed)) {
       if (!__all_sync(0xffffffffu, mbar_wait(acc_done, 0, p.spin_limit, s_abort))) failed = true;
     }
-    if (!__any_sync(0xffffffffu, failed)) {
+    if (epilogue_warp && !__any_sync(0xffffffffu, failed)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int quarter = warp & 3;                 // the tensor-memory lanes this warp may read
       const int trow = quarter * 32 + lane;         // row of the tile held by this thread's lane
@@ -480,12 +511,18 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-size_t tc_stage_bytes(const grim_bcr* h) { return (kATileBytes + kBTileBytes + (size_t)h->tc_max_rec + 1023) & ~size_t(1023); }
-size_t tc_smem_need(const grim_bcr* h, int stages) { return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(h); }
-int tc_stages(const grim_bcr* h) {
+size_t tc_stage_bytes(const grim_bcr*) { return kATileBytes + kBTileBytes; }
+size_t tc_rec_stride(const grim_bcr* h) { return ((size_t)h->tc_max_rec + 127) & ~size_t(127); }
+size_t tc_smem_need(const grim_bcr* h, int stages, int nrec) {
+  return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(h) + (size_t)nrec * tc_rec_stride(h);
+}
+// Ring sizes that fit: as many tile slots as possible first (they carry the bulk of the bytes in flight), then as
+// many record slots as are left, at least as many as tile slots.
+bool tc_rings(const grim_bcr* h, int* stages, int* nrec) {
   for (int s = kTcStages; s >= 2; --s)
-    if (tc_smem_need(h, s) <= 225 * 1024) return s;
-  return 0;
+    for (int r = kTcRecSlots; r >= s; --r)
+      if (tc_smem_need(h, s, r) <= 226 * 1024) { *stages = s; *nrec = r; return true; }
+  return false;
 }
 
 }  // namespace
@@ -501,7 +538,8 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
     return false;
   }
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
-  if (tc_stages(h) == 0) return false;
+  int st_ = 0, nr_ = 0;
+  if (!tc_rings(h, &st_, &nr_)) return false;
   if (h->tc_mtiles > 65535) return false;
   return encode_tiled_fn() != nullptr;
 }
@@ -514,7 +552,8 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;
   p.stage_bytes = (uint32_t)tc_stage_bytes(h);
-  p.nstages = tc_stages(h);
+  p.rec_stride = (uint32_t)tc_rec_stride(h);
+  tc_rings(h, &p.nstages, &p.nrec);
   p.spin_limit = 1u << 20;
   p.a = a;
 
@@ -523,7 +562,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   memset(&tm, 0, sizeof(tm));
   if (a.conv) {
     auto kern = h->bh == 4 ? bcr_tc_kernel<4, true> : (h->bh == 8 ? bcr_tc_kernel<8, true> : bcr_tc_kernel<16, true>);
-    const size_t smem = tc_smem_need(h, p.nstages);
+    const size_t smem = tc_smem_need(h, p.nstages, p.nrec);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
     dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)h->tc_mtiles);
     kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
@@ -538,7 +577,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
-  const size_t smem = tc_smem_need(h, p.nstages);
+  const size_t smem = tc_smem_need(h, p.nstages, p.nrec);
   auto kern = h->bh == 4 ? bcr_tc_kernel<4, false> : (h->bh == 8 ? bcr_tc_kernel<8, false> : bcr_tc_kernel<16, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
