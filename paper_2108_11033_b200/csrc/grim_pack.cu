@@ -1,6 +1,7 @@
 // Host-side BCR packer: validates the mask, derives per-block keep lists, builds the canonical
 // form and the two private device layouts, uploads them.  No device computation happens here.
 #include <algorithm>
+#include <cstdio>
 #include <cstring>
 #include <new>
 #include <numeric>
@@ -527,5 +528,5 @@ extern "C" grim_status_t grim_bcr_status(grim_bcr_t h) {
   unsigned v = 0;
   if (cudaMemcpy(&v, h->d_status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return GRIM_ERR_CUDA;
   if (v != 0) cudaMemset(h->d_status, 0, 4);
-  return (grim_status_t)v;
+  return (grim_status_t)(v & 0xFFu);  // the upper bits say which wait gave up (a debugging aid of the kernels)
 }

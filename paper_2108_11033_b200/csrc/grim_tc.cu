@@ -52,6 +52,7 @@ struct TcParams {
   unsigned* status;
   int nbr, M, K, bh, nkt;
   int bh_shift, slots_per_tile, nstages, nrec;
+  int mt, mtiles;  // row tiles (128 rows each) per thread block: 1 or 2 (they share every X tile); tiles in the matrix
   uint32_t stage_bytes, rec_stride;
   unsigned spin_limit;
   int64_t in_elems;  // convolution: elements of the input tensor
@@ -154,7 +155,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   uint64_t* built = empty + kTcStages;                         // convolution: the X tile of a stage is written
   uint64_t* acc_done = built + kTcStages;                      // all multiplies of the tile are complete
   uint64_t* rec_full = acc_done + 1;                           // a packed record has landed
-  uint64_t* rec_empty = rec_full + kTcRecSlots;                // a packed record has been expanded
+  unsigned* s_done = reinterpret_cast<unsigned*>(smem + 640);    // [record slot] warps that have finished expanding it
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 512);  // [record slot] bytes of the packed record (0: none)
@@ -166,7 +167,9 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
   const SpmmArgs& a = p.a;
   const int64_t q0 = (int64_t)blockIdx.x * kTQ;
-  const int pos0 = blockIdx.y * p.slots_per_tile;  // first band (schedule position) of this tile
+  const int pos0 = blockIdx.y * p.mt * p.slots_per_tile;  // first band (schedule position) of this thread block's rows
+  const uint32_t b_off = (uint32_t)p.mt * kATileBytes;     // the X tile follows the weight tiles in a stage
+  const uint32_t tmem_cols = kTmemCols * (uint32_t)p.mt;
   const int nkt = p.nkt, ns = p.nstages, nr = p.nrec;
 
   if (tid == 0) {
@@ -179,14 +182,14 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     }
     for (int s = 0; s < kTcRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
-      mbar_init(rec_empty + s, kTcGroupWarps);
+      s_done[s] = 0;
     }
     mbar_init(acc_done, 1);
     *s_abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   if (warp == 1) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(s_tmem)), "r"(tmem_cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -194,26 +197,39 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
 
+  // Requests the packed records of K tile k (one per row tile) into record slot rs; one thread.
+  auto request_records = [&](int k, int rs) {
+    uint32_t bytes[2] = {0u, 0u}, off[2] = {0u, 0u}, total = 0;
+    for (int m = 0; m < p.mt; ++m) {
+      const int t = (int)blockIdx.y * p.mt + m;
+      if (t < p.mtiles) {
+        const RcStage se = p.stage[(int64_t)t * nkt + k];
+        bytes[m] = se.bytes; off[m] = se.off16;
+      }
+      s_meta[rs * 2 + m] = bytes[m];
+      total += bytes[m];
+    }
+    mbar_arrive_expect_tx(rec_full + rs, total);
+    for (int m = 0; m < p.mt; ++m)
+      if (bytes[m]) bulk_load(recs + (size_t)(rs * p.mt + m) * p.rec_stride, p.blob + (size_t)off[m] * 16, bytes[m], rec_full + rs);
+  };
+
   bool failed = false;
+  int fail_site = 0;
   if (warp == 0) {
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
       // the first records (the ring of records is deeper than the ring of tiles); later ones are requested by the
       // expansion warps as they free a record slot
-      for (int rk = 0; rk < nr && rk < nkt; ++rk) {
-        const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + rk];
-        s_meta[rk] = se.bytes;
-        mbar_arrive_expect_tx(rec_full + rk, se.bytes);
-        if (se.bytes) bulk_load(recs + (size_t)rk * p.rec_stride, p.blob + (size_t)se.off16 * 16, se.bytes, rec_full + rk);
-      }
+      for (int rk = 0; rk < nr && rk < nkt; ++rk) request_records(rk, rk);
       for (int kt = 0; kt < nkt && !CONV; ++kt) {  // the convolution builds its X tiles itself
         const int slot = kt % ns;
-        if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true; break; }
+        if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true, fail_site = 1; break; }
         uint8_t* st = stages + (size_t)slot * stage_bytes;
         mbar_arrive_expect_tx(full + slot, (unsigned)kBTileBytes);
 #pragma unroll
         for (int i = 0; i < kTQ / 64; ++i)
-          tma_load_2d(st + kATileBytes + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+          tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
       }
     }
   } else if (warp == 1) {
@@ -223,17 +239,19 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         const int slot = kt % ns;
         const unsigned par = (unsigned)((kt / ns) & 1);
         if ((!CONV && !mbar_wait(full + slot, par, p.spin_limit, s_abort)) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort) ||
-            (CONV && !mbar_wait(built + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
+            (CONV && !mbar_wait(built + slot, par, p.spin_limit, s_abort))) { failed = true, fail_site = 2; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
         const uint32_t a_addr = smem_u32(stages + (size_t)slot * stage_bytes);
-        const uint32_t b_addr = a_addr + kATileBytes;
+        const uint32_t b_addr = a_addr + b_off;
+        for (int m = 0; m < p.mt; ++m) {
 #pragma unroll
-        for (int s = 0; s < kTK / 16; ++s) {
-          // A: K-major, rows 128 bytes apart, 8-row groups 1 KiB apart; 16 K-elements = 32 bytes further on
-          const uint64_t ad = smem_desc(a_addr + s * 32, 16, 1024);
-          // B: N-major, 64-column groups 8 KiB apart, 8-row K groups 1 KiB apart; 16 K-rows = 2 KiB further on
-          const uint64_t bd = smem_desc(b_addr + s * 2048, 64 * kTK * 2, 1024);
-          umma_bf16(tmem_base, ad, bd, (kt > 0 || s > 0) ? 1u : 0u);
+          for (int s = 0; s < kTK / 16; ++s) {
+            // A: K-major, rows 128 bytes apart, 8-row groups 1 KiB apart; 16 K-elements = 32 bytes further on
+            const uint64_t ad = smem_desc(a_addr + m * kATileBytes + s * 32, 16, 1024);
+            // B: N-major, 64-column groups 8 KiB apart, 8-row K groups 1 KiB apart; 16 K-rows = 2 KiB further on
+            const uint64_t bd = smem_desc(b_addr + s * 2048, 64 * kTK * 2, 1024);
+            umma_bf16(tmem_base + (uint32_t)m * kTmemCols, ad, bd, (kt > 0 || s > 0) ? 1u : 0u);
+          }
         }
         umma_commit(empty + slot);  // arrives when the multiplies above have read their operands
       }
@@ -282,8 +300,8 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
     for (int kt = bgrp; kt < nkt; kt += kTcBuildGroups) {
       const int slot = kt % ns;
-      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
-      uint8_t* bt_base = stages + (size_t)slot * stage_bytes + kATileBytes + panel_off;
+      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 3; break; }
+      uint8_t* bt_base = stages + (size_t)slot * stage_bytes + b_off + panel_off;
       // The thread's 16 rows of the stage are taken in batches: first the address arithmetic and the vector loads
       // of the whole batch (so that they are in flight together), then shifting, masking, storing.
       constexpr int kBatch = 4;
@@ -357,20 +375,21 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       const unsigned par = (unsigned)((kt / ns) & 1);
       // the weight tile of the slot is free once the multiplies of its previous use are done; the record is
       // normally long there
-      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true; break; }
-      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true; break; }
+      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 4; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
       uint4* a4 = reinterpret_cast<uint4*>(st);
-#pragma unroll
-      for (int i = 0; i < kATileBytes / 16 / kTcGroupThreads; ++i) a4[wt + i * kTcGroupThreads] = make_uint4(0u, 0u, 0u, 0u);
+      for (int i = 0; i < p.mt * (kATileBytes / 16 / kTcGroupThreads); ++i) a4[wt + i * kTcGroupThreads] = make_uint4(0u, 0u, 0u, 0u);
       __syncwarp();
       if (lane == 0) mbar_arrive(zeroed + slot);
-      if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true; break; }
-      if (s_meta[rs]) {
+      if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true, fail_site = 6; break; }
+      for (int m = 0; m < p.mt; ++m) {
+        if (s_meta[rs * 2 + m] == 0) continue;
+        uint8_t* at = st + m * kATileBytes;
         // a thread takes kept columns of the tile and drops each column's values into the swizzled K-major tile
         // (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits).  All loads of a column are
         // issued before its stores: the value of row r sits popcount(mask below r) places after the first
-        const uint32_t* rec = reinterpret_cast<const uint32_t*>(recs + (size_t)rs * p.rec_stride);
+        const uint32_t* rec = reinterpret_cast<const uint32_t*>(recs + (size_t)(rs * p.mt + m) * p.rec_stride);
         const int ncols = (int)rec[0];
         const uint32_t* cw = rec + 4;
         const uint16_t* vo = reinterpret_cast<const uint16_t*>(cw + ((ncols + 3) & ~3));
@@ -388,7 +407,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
 #pragma unroll
           for (int r = 0; r < BH; ++r) {
             const uint32_t row = rowbase + r;
-            if ((rm >> r) & 1u) *reinterpret_cast<uint16_t*>(st + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = val[r];
+            if ((rm >> r) & 1u) *reinterpret_cast<uint16_t*>(at + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = val[r];
           }
         }
       }
@@ -396,16 +415,11 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       __syncwarp();
       if (lane == 0) {
         mbar_arrive(ready + slot);
-        mbar_arrive(rec_empty + rs);
-      }
-      if (wt == 0 && kt + nr < nkt) {
-        // the record slot is free once every warp of the group is done with it: request the record that uses it next
-        if (!mbar_wait(rec_empty + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort)) failed = true;
-        else {
-          const RcStage se = p.stage[(int64_t)blockIdx.y * nkt + kt + nr];
-          s_meta[rs] = se.bytes;
-          mbar_arrive_expect_tx(rec_full + rs, se.bytes);
-          if (se.bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)se.off16 * 16, se.bytes, rec_full + rs);
+        // the last warp of the group to finish with the record frees its slot: it requests the record that uses
+        // the slot next (every read of the old record precedes that warp's count)
+        if (atomicAdd(s_done + rs, 1u) == (unsigned)kTcGroupWarps - 1u) {
+          s_done[rs] = 0;
+          if (kt + nr < nkt) request_records(kt + nr, rs);
         }
       }
       if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
@@ -413,22 +427,23 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     // ------------------------------------------------------------------ epilogue
     const bool epilogue_warp = warp - 2 < 8;  // two warps per quarter of the tensor-memory lanes
     if (epilogue_warp && !__any_sync(0xffffffffu, failed)) {
-      if (!__all_sync(0xffffffffu, mbar_wait(acc_done, 0, p.spin_limit, s_abort))) failed = true;
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_done, 0, p.spin_limit, s_abort))) failed = true, fail_site = 8;
     }
     if (epilogue_warp && !__any_sync(0xffffffffu, failed)) {
       asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
       const int quarter = warp & 3;                 // the tensor-memory lanes this warp may read
       const int trow = quarter * 32 + lane;         // row of the tile held by this thread's lane
-      const int pos = pos0 + (trow >> p.bh_shift);
       const int r = trow & (BH - 1);
+      const int cb0 = ((warp - 2) >> 2) * (kTQ / 64), cb1 = cb0 + kTQ / 64;  // warps 2-5: columns 0-127, warps 6-9: 128-255
+      for (int m = 0; m < p.mt; ++m) {
+      const int pos = pos0 + m * p.slots_per_tile + (trow >> p.bh_shift);
       int64_t row = -1;
-      if (pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + r;
+      if (pos < p.nbr && (int)blockIdx.y * p.mt + m < p.mtiles) row = (int64_t)p.band_order[pos] * p.bh + r;
       const bool row_ok = row >= 0 && row < p.M;
       const float bias = (row_ok && a.bias) ? __ldg(a.bias + row) : 0.f;
-      const int cb0 = ((warp - 2) >> 2) * (kTQ / 64), cb1 = cb0 + kTQ / 64;  // warps 2-5: columns 0-127, warps 6-9: 128-255
       for (int cb = cb0; cb < cb1; ++cb) {
         uint32_t v[32];
-        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(cb * 32), v);
+        tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(m * (int)kTmemCols + cb * 32), v);
         const int64_t q = q0 + cb * 32;
         if (!row_ok || q >= a.ncols) continue;
         float t[32];
@@ -479,18 +494,19 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
           }
         }
       }
+      }  // row tiles
     }
   }
 
   if (__any_sync(0xffffffffu, failed)) {
     *s_abort = 1;
-    if (lane == 0) atomicExch(p.status, (unsigned)GRIM_ERR_TIMEOUT);
+    if (fail_site) atomicOr(p.status, (unsigned)GRIM_ERR_TIMEOUT | (1u << (8 + fail_site)));
   }
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
   __syncthreads();
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(kTmemCols) : "memory");
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
   }
 }
 
@@ -511,18 +527,27 @@ EncodeTiledFn encode_tiled_fn() {
   return fn;
 }
 
-size_t tc_stage_bytes(const grim_bcr*) { return kATileBytes + kBTileBytes; }
+size_t tc_stage_bytes(int mt) { return (size_t)mt * kATileBytes + kBTileBytes; }
 size_t tc_rec_stride(const grim_bcr* h) { return ((size_t)h->tc_max_rec + 127) & ~size_t(127); }
-size_t tc_smem_need(const grim_bcr* h, int stages, int nrec) {
-  return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(h) + (size_t)nrec * tc_rec_stride(h);
+size_t tc_smem_need(const grim_bcr* h, int mt, int stages, int nrec) {
+  return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(mt) + (size_t)nrec * mt * tc_rec_stride(h);
 }
 // Ring sizes that fit: as many tile slots as possible first (they carry the bulk of the bytes in flight), then as
 // many record slots as are left, at least as many as tile slots.
-bool tc_rings(const grim_bcr* h, int* stages, int* nrec) {
-  for (int s = kTcStages; s >= 2; --s)
+// At least as many tile slots as expansion groups: a group then never waits on a barrier that is more than one
+// phase behind it (parity waits cannot tell phases two apart).
+bool tc_rings(const grim_bcr* h, int mt, int* stages, int* nrec) {
+  for (int s = kTcStages; s >= kTcGroups; --s)
     for (int r = kTcRecSlots; r >= s; --r)
-      if (tc_smem_need(h, s, r) <= 226 * 1024) { *stages = s; *nrec = r; return true; }
+      if (tc_smem_need(h, mt, s, r) <= 226 * 1024) { *stages = s; *nrec = r; return true; }
   return false;
+}
+// Row tiles per thread block: two share every X tile (half the L2 traffic per flop, which is what bounds the
+// kernel) when that still leaves enough thread blocks for the GPU and three tile slots fit.
+int tc_row_tiles(const grim_bcr* h, int64_t qtiles) {
+  int s = 0, r = 0;
+  if (h->tc_mtiles >= 2 && qtiles * ((h->tc_mtiles + 1) / 2) >= 96 && tc_rings(h, 2, &s, &r) && s >= 3) return 2;
+  return 1;
 }
 
 }  // namespace
@@ -539,7 +564,7 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   }
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
   int st_ = 0, nr_ = 0;
-  if (!tc_rings(h, &st_, &nr_)) return false;
+  if (!tc_rings(h, 1, &st_, &nr_)) return false;
   if (h->tc_mtiles > 65535) return false;
   return encode_tiled_fn() != nullptr;
 }
@@ -551,9 +576,12 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.nbr = (int)h->nbr; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.nkt = (int)h->tc_ktiles;
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;
-  p.stage_bytes = (uint32_t)tc_stage_bytes(h);
+  const int64_t qtiles_ = (a.ncols + kTQ - 1) / kTQ;
+  p.mt = (a.tile_n == 1 || a.tile_n == 2) ? a.tile_n : tc_row_tiles(h, qtiles_);
+  p.mtiles = (int)h->tc_mtiles;
+  if (!tc_rings(h, p.mt, &p.nstages, &p.nrec)) { p.mt = 1; tc_rings(h, 1, &p.nstages, &p.nrec); }
+  p.stage_bytes = (uint32_t)tc_stage_bytes(p.mt);
   p.rec_stride = (uint32_t)tc_rec_stride(h);
-  tc_rings(h, &p.nstages, &p.nrec);
   p.spin_limit = 1u << 20;
   p.a = a;
 
@@ -562,9 +590,9 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   memset(&tm, 0, sizeof(tm));
   if (a.conv) {
     auto kern = h->bh == 4 ? bcr_tc_kernel<4, true> : (h->bh == 8 ? bcr_tc_kernel<8, true> : bcr_tc_kernel<16, true>);
-    const size_t smem = tc_smem_need(h, p.nstages, p.nrec);
+    const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
-    dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)h->tc_mtiles);
+    dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt));
     kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
@@ -577,12 +605,12 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
-  const size_t smem = tc_smem_need(h, p.nstages, p.nrec);
+  const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec);
   auto kern = h->bh == 4 ? bcr_tc_kernel<4, false> : (h->bh == 8 ? bcr_tc_kernel<8, false> : bcr_tc_kernel<16, false>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
-  const int64_t mtiles = h->tc_mtiles;
+  const int64_t mtiles = (h->tc_mtiles + p.mt - 1) / p.mt;
   dim3 grid((unsigned)qtiles, (unsigned)mtiles);
   kern<<<grid, kTcThreads, smem, s>>>(tm, p);
   count_launch();

@@ -136,6 +136,17 @@ def test_register_tiled_kernel_explicit(B, case, bf16):
     check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=groups, path=1, flags=1)
 
 
+@pytest.mark.parametrize("row_tiles", [1, 2])
+def test_tensor_core_row_tiles_per_block(B, row_tiles):
+    """One or two 128-row tiles per thread block (two share every X tile), on a row count that leaves the last
+    thread block with a single, partly filled tile."""
+    M, K, bh, bw, N = 328, 700, 8, 32, 520
+    W = gen.dense_weight(M, K, seed=97)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=5, dist="uniform", seed=98, empty_frac=0.1)
+    X = gen.normal_f32((K, N), 1.0, 99, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=2, tile_n=row_tiles, flags=1)
+
+
 @pytest.mark.parametrize("y_bf16", [False, True])
 @pytest.mark.parametrize("case", [(256, 512, 8, 32, 256), (200, 333, 8, 32, 328), (300, 520, 4, 16, 520), (260, 700, 16, 64, 264),
                                   (96, 153, 8, 32, 1024), (512, 2048, 16, 64, 776)])
