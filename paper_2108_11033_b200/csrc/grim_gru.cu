@@ -415,24 +415,14 @@ __global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const G
     }
     __syncthreads();
     if (gate_live) {
+      // the thread that owns a hidden unit computes it and sends it straight to the next-step buffer of every CTA
+      // of the cluster (no staging, no second block barrier)
       const float hn = gru_gate(partial, bq, gi, g_tri, g_r, 2, BH, hcur[unit]);
-      hnew[tid] = hn;
       p.out[(int64_t)t * H + unit] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
-    }
-    __syncthreads();
-    if ((U & 3) == 0) {
-      const int q = U >> 2;
-      for (int i = tid; i < CS * q; i += kRegThreads) {
-        const int dst = i / q, j = i - dst * q;
-        float4* remote = cluster.map_shared_rank(reinterpret_cast<float4*>(hnxt_local + rank * U) + j, dst);
-        *remote = reinterpret_cast<const float4*>(hnew)[j];
-      }
-    } else {
-      for (int i = tid; i < CS * U; i += kRegThreads) {
-        const int dst = i / U, j = i - dst * U;
-        *cluster.map_shared_rank(hnxt_local + rank * U + j, dst) = hnew[j];
-      }
+      float* mine = hnxt_local + unit;
+#pragma unroll 4
+      for (int dst = 0; dst < CS; ++dst) *cluster.map_shared_rank(mine, dst) = hn;
     }
 #pragma unroll
     for (int g = 0; g < 3; ++g) gi[g] = gi_next[g];
