@@ -46,6 +46,10 @@ struct grim_gru {
   std::vector<uint32_t*> d_img_col;
   std::vector<float*> d_gi;  // per layer: hoisted pre-activations, T x 3H (layers overlap in time, so each has its own)
   float* d_seq[2] = {nullptr, nullptr};
+  // unit-major copies (feature x time, row stride = T rounded up to 4): the projections then read X row-major
+  float* d_seqT[2] = {nullptr, nullptr};
+  float* d_xT = nullptr;
+  bool transposed_inputs = true;
   // layer pipelining: layer l runs on its own stream, a chunk of time steps behind layer l - 1
   std::vector<cudaStream_t> lstream;   // streams of layers 1 .. L-1 (layer 0 uses the caller's stream)
   std::vector<cudaEvent_t> ev_chunk;   // [layer][chunk]: the layer's recurrence has produced the chunk
@@ -81,6 +85,8 @@ struct GruParams {
   const float* b_ih; // 3H or null: added to gi here (not used by the register-resident kernel)
   const float* h0;   // H or null
   float* out;        // T x H
+  float* outT;       // null, or the same values unit-major: outT[unit * ldT + t] (input of the next layer's projection)
+  int64_t ldT;
   float* hT;         // H or null
   unsigned* bar;
   unsigned* status;
@@ -251,6 +257,7 @@ __global__ void __launch_bounds__(1024, 1) gru_recurrent_kernel(const GruParams 
     if (gate_live) {
       const float hn = gru_gate(partial, bq, gi, g_tri, g_r, p.ks, BH, hs[unit]);
       p.out[(int64_t)t * p.H + unit] = hn;
+      if (p.outT) p.outT[(int64_t)unit * p.ldT + t] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
     }
     if (t == p.T - 1) break;
@@ -315,6 +322,7 @@ __global__ void __launch_bounds__(1024, 1) gru_cluster_kernel(const GruParams p)
       const float hn = gru_gate(partial, bq, gi, g_tri, g_r, p.ks, BH, hcur[unit]);
       hnew[tid] = hn;
       p.out[(int64_t)t * p.H + unit] = hn;
+      if (p.outT) p.outT[(int64_t)unit * p.ldT + t] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
     }
     __syncthreads();
@@ -419,6 +427,7 @@ __global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const G
       // of the cluster (no staging, no second block barrier)
       const float hn = gru_gate(partial, bq, gi, g_tri, g_r, 2, BH, hcur[unit]);
       p.out[(int64_t)t * H + unit] = hn;
+      if (p.outT) p.outT[(int64_t)unit * p.ldT + t] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
       float* mine = hnxt_local + unit;
 #pragma unroll 4
@@ -567,6 +576,9 @@ void destroy(grim_gru* g) {
   if (g->ev_fork) cudaEventDestroy(g->ev_fork);
   cudaFree(g->d_seq[0]);
   cudaFree(g->d_seq[1]);
+  cudaFree(g->d_seqT[0]);
+  cudaFree(g->d_seqT[1]);
+  cudaFree(g->d_xT);
   cudaFree(g->d_sync);
   delete g;
 }
@@ -581,6 +593,20 @@ __global__ void fill_rows_kernel(float* __restrict__ out, const float* __restric
   const int64_t total4 = T * n / 4, n4 = n / 4;
   for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total4; i += (int64_t)gridDim.x * blockDim.x)
     reinterpret_cast<float4*>(out)[i] = __ldg(reinterpret_cast<const float4*>(bias) + i % n4);
+}
+// out[k * ld + t] = in[t * K + k]: the caller's T x K input, feature-major.
+__global__ void transpose_input_kernel(const float* __restrict__ in, float* __restrict__ out, int64_t T, int64_t K, int64_t ld) {
+  __shared__ float tile[32][33];
+  const int64_t t0 = (int64_t)blockIdx.x * 32, k0 = (int64_t)blockIdx.y * 32;
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t t = t0 + i, k = k0 + threadIdx.x;
+    tile[i][threadIdx.x] = (t < T && k < K) ? in[t * K + k] : 0.f;
+  }
+  __syncthreads();
+  for (int i = threadIdx.y; i < 32; i += blockDim.y) {
+    const int64_t k = k0 + i, t = t0 + threadIdx.x;
+    if (k < K && t < T) out[k * ld + t] = tile[threadIdx.x][i];
+  }
 }
 // Records the next timing event of the pool on stream s (profiling only).
 void profile_mark(grim_gru* g, int kind, cudaStream_t s) {
@@ -653,6 +679,10 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
       if (e == cudaSuccess) e = cudaEventCreateWithFlags(&g->ev_fork, cudaEventDisableTiming);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seq[0], (size_t)max_T * H * 4);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seq[1], (size_t)max_T * H * 4);
+      const size_t ldT_max = (size_t)((max_T + 3) / 4 * 4);
+      if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seqT[0], ldT_max * H * 4);
+      if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_seqT[1], ldT_max * H * 4);
+      if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_xT, ldT_max * (size_t)W_ih[0]->K * 4);
       if (e == cudaSuccess) e = cudaMalloc((void**)&g->d_sync, (size_t)(layers + 1) * 4);
       if (e == cudaSuccess) e = cudaMemset(g->d_sync, 0, (size_t)(layers + 1) * 4);
       if (e != cudaSuccess) st = e == cudaErrorMemoryAllocation ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;
@@ -801,7 +831,9 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
   if (g->pipeline && L > 1 && (use_reg || use_cluster))
     chunks = g->want_chunks > 0 ? (int)std::min<int64_t>(g->want_chunks, T)
                                 : (int)std::max<int64_t>(1, std::min<int64_t>(3, T / 64));
-  const int64_t clen = (T + chunks - 1) / chunks;
+  const int64_t clen = ((T + chunks - 1) / chunks + 3) / 4 * 4;  // a multiple of 4: chunk starts stay 16-byte aligned
+  const int64_t ldT = (T + 3) / 4 * 4;
+  const bool tin = g->transposed_inputs && g->d_xT != nullptr;
   auto stream_of = [&](int l) { return (chunks > 1 && l > 0) ? g->lstream[(size_t)l - 1] : s0; };
   if (chunks > 1) {
     if (cudaEventRecord(g->ev_fork, s0) != cudaSuccess) return GRIM_ERR_CUDA;
@@ -825,8 +857,15 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     const grim_bcr* wi = g->Wih[(size_t)l];
     // gi[t, :] = W_ih x_t + b_ih for the n steps from t0 (X given q-major as n x in, output n x 3H)
     SpmmArgs a;
-    a.X = seq_in + t0 * wi->K; a.Y = g->d_gi[(size_t)l] + t0 * 3 * H; a.ncols = n;
-    a.x_sk = 1; a.x_sq = wi->K; a.y_sr = 1; a.y_sq = 3 * H;
+    a.Y = g->d_gi[(size_t)l] + t0 * 3 * H; a.ncols = n;
+    a.y_sr = 1; a.y_sq = 3 * H;
+    if (tin) {  // feature-major copy: a plain row-major K x n operand (fetched by TMA)
+      a.X = (l == 0 ? g->d_xT : g->d_seqT[(l - 1) & 1]) + t0;
+      a.x_sk = ldT; a.x_sq = 1;
+    } else {
+      a.X = seq_in + t0 * wi->K;
+      a.x_sk = 1; a.x_sq = wi->K;
+    }
     a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32;
     a.bias = g->d_bih[(size_t)l];
     a.y_prefilled = 1;  // every row of the buffer already holds b_ih (below): a split multiply adds onto it and
@@ -845,6 +884,8 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
     // the state entering a later chunk is the previous chunk's last output row
     p.h0 = t0 == 0 ? (h0 ? h0 + (int64_t)l * H : nullptr) : seq_out + (t0 - 1) * H;
     p.out = seq_out + t0 * H;
+    p.outT = (tin && l < L - 1) ? g->d_seqT[l & 1] + t0 : nullptr;
+    p.ldT = ldT;
     p.hT = (hT && t0 + n == T) ? hT + (int64_t)l * H : nullptr;
     p.bar = g->d_sync + l; p.status = g->d_sync + L;
     p.H = (int)H; p.bh = g->bh; p.T = (int)n; p.tpc = m.tpc; p.ks = m.ks; p.resident = m.resident;
@@ -882,7 +923,14 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
       if (l > 0 && c == 0 && g->d_gi[(size_t)l] == g->d_gi[0] && !prefill(l, s))
         return GRIM_ERR_CUDA;  // layers share one buffer (allocation-free variant): fill it again for this layer
       if (l == 0) {
-        if (c == 0) st = launch_projection(0, x, 0, T, s);  // the first layer's input is all there: one launch
+        if (c == 0) {  // the first layer's input is all there: one launch (after turning it feature-major)
+          if (tin) {
+            const int64_t K0 = g->Wih[0]->K;
+            transpose_input_kernel<<<dim3((unsigned)((T + 31) / 32), (unsigned)((K0 + 31) / 32)), dim3(32, 8), 0, s>>>(x, g->d_xT, T, K0, ldT);
+            count_launch();
+          }
+          st = launch_projection(0, x, 0, T, s);
+        }
       } else {
         if (chunks > 1 && cudaStreamWaitEvent(s, g->ev_chunk[(size_t)(l - 1) * g->max_chunks + c], 0) != cudaSuccess) return GRIM_ERR_CUDA;
         st = launch_projection(l, seq_in, t0, n, s);
@@ -1012,7 +1060,8 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
   const std::vector<float*> saved_gi = g->d_gi;
   float* const saved_seq0 = g->d_seq[0];
   float* const saved_seq1 = g->d_seq[1];
-  const bool saved_pipeline = g->pipeline;
+  const bool saved_pipeline = g->pipeline, saved_tin = g->transposed_inputs;
+  g->transposed_inputs = false;  // the feature-major copies live in allocated buffers: not used here
   for (float*& p : g->d_gi) p = reinterpret_cast<float*>(base);
   g->d_seq[0] = reinterpret_cast<float*>(base + gi_bytes);
   g->d_seq[1] = reinterpret_cast<float*>(base + gi_bytes + seq_bytes);
@@ -1022,5 +1071,6 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
   g->d_seq[0] = saved_seq0;
   g->d_seq[1] = saved_seq1;
   g->pipeline = saved_pipeline;
+  g->transposed_inputs = saved_tin;
   return st;
 }
