@@ -33,10 +33,10 @@ METRIC = "BCR SpMM/GEMV effective GFLOP/s (2*nnz*N)"
 # DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes) of the dominant kernel per step, from one ncu
 # capture of the same command (summaries under profiles/); None where the kernel has changed since or was not captured.
 TRAFFIC = {
-    "gru_2x1024_in153_T200_bcr8x32_c10_fp32": 6 * 3.514e6,  # six launches (2 layers x 3 chunks) of 3.5 MB each
+    "gru_2x1024_in153_T200_bcr8x32_c10_fp32": 6 * 3.519e6,  # six launches (2 layers x 3 chunks) of 3.5 MB each
     "spmm_M4096_K4096_N1024_c8_8x32_uniform_fp32": 27.68e6,
     "spmm_M8192_K8192_N1_c4_8x32_uniform_fp32": 87.46e6,
-    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.70e6,
+    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.45e6,
 }
 UNIT = "GFLOP/s"
 
