@@ -420,6 +420,22 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def max_over_ranks(values, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks of the default process group (identity when there
+    is none): a multi-GPU number is the slowest rank's."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    if dist.is_available() and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def aggregate_value(flops_per_rank_step, steps, total_ms, world):
+    """Whole-job throughput in GFLOP/s: every rank (replica) does the same work; time is the slowest rank's."""
+    return world * flops_per_rank_step * steps / (total_ms * 1e-3) / 1e9
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -483,15 +499,12 @@ def run_ours(args):
     e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
     clocks = sampler.stop() if rank == 0 else None
 
-    t = torch.tensor([total_ms, e2e_ms], device="cuda", dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_ms = float(t[0]), float(t[1])
+    total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     if rank == 0:
         peaks = measured_peaks()
-        value = world * wl.flops * args.steps / (total_ms * 1e-3) / 1e9
-        e2e_value = world * wl.flops * args.steps / (e2e_ms * 1e-3) / 1e9
+        value = aggregate_value(wl.flops, args.steps, total_ms, world)
+        e2e_value = aggregate_value(wl.flops, args.steps, e2e_ms, world)
         k_ms = statistics.mean(kernel_ms)
         # binding roofline of the dominant kernel: the slower of (algorithmic bytes at the measured HBM bandwidth) and
         # (effective flops 2*nnz*N at the peak of the unit that does the arithmetic: plain fp32 FMA pipes, derived as
