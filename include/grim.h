@@ -88,7 +88,9 @@ typedef struct {
 typedef struct {
   int32_t tile_n;  /* path 4: output columns per thread block (16, 32, 64 or 128);
                       path 1: groups of 16 row bands per thread block (1, 2 or 4), plus 256 x the number of
-                      thread blocks that share a tile's block columns (split multiply, 1 - 8) */
+                      thread blocks that share a tile's block columns (split multiply, 1 - 8);
+                      path 3: 1 = values staged in registers, 2 = values streamed through shared memory by bulk
+                      asynchronous copies (persistent thread blocks), 0 = the streaming variant when it fits */
   int32_t path;    /* 0 auto; 1 register-tiled CUDA-core kernel (N > 16); 2 tcgen05 tensor-core tiles (bf16
                       handles only); 3 lane-per-column kernel (N <= 16, N = 1 is the matrix-vector product);
                       4 shared-memory slab kernel (any N; the fall-back for operands the others do not take).

@@ -40,8 +40,13 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
     if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
     return launch_spmm_tc(h, a, s);
   }
-  if (path == 3 || (path == 0 && X->cols <= kSkinnyMaxN && h->gemv_ok))
+  if (path == 3 || (path == 0 && X->cols <= kSkinnyMaxN && h->gemv_ok)) {
+    // tile_n = 1 under path 3 asks for the register-staged variant; otherwise the streaming one runs when it can
+    if (!(path == 3 && a.tile_n == 1) && stream_path_supported(h, X->cols))
+      return launch_stream(h, X->ptr, X->dtype, X->ld, X->cols, Y->ptr, Y->dtype, Y->ld, s);
+    if (path == 3 && a.tile_n == 2) return GRIM_ERR_UNSUPPORTED;
     return launch_skinny(h, X->ptr, X->dtype, X->ld, X->cols, Y->ptr, Y->dtype, Y->ld, s);
+  }
   if (path == 4) return launch_spmm(h, a, s);
   if (path == 0 && tc_path_supported(h, a) && a.ncols >= 256) return launch_spmm_tc(h, a, s);
   if (ffma_path_supported(h, a)) return launch_ffma(h, a, s);
@@ -87,7 +92,7 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   float best_t = -1.f;
   grim_tune_t cand_best{};
   // candidates: (path, tile_n); a candidate that cannot take the request is skipped
-  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {3, 0}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
+  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
   for (const auto& cd : cand) {
     grim_tune_t c{};
     c.path = cd[0];

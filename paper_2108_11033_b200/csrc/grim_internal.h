@@ -47,6 +47,15 @@ struct ChunkDesc {
   uint32_t cw_off;
   uint32_t ncols_kr;  // ncols | kr << 16
 };
+// The streaming kernel moves the chunk layout in "runs": up to kRunChunks consecutive chunks of one band whose
+// values take at most kRunValueBytes (no single chunk is larger: 16 rows x 32 columns x 4 bytes is half of it).  Run r covers chunks [runs[r].c0, runs[r + 1].c0) and values [runs[r].v0, runs[r + 1].v0); the
+// table ends with a sentinel.  run_ptr[pos] .. run_ptr[pos + 1] are the runs of the band at schedule position pos.
+constexpr int kRunChunks = 4;
+constexpr int kRunValueBytes = 4096;
+struct RunDesc {
+  uint32_t c0;  // first chunk
+  uint32_t v0;  // first value, in elements
+};
 
 // ---------------------------------------------------------------------------------------------
 // Device layout for the register-tiled N > 16 kernel and the tensor-core kernel ("row-chunk"
@@ -132,6 +141,9 @@ struct grim_bcr {
   grim::ChunkDesc* d_chunks = nullptr;
   uint32_t* d_colwords = nullptr;
   void* d_gemv_vals = nullptr;
+  uint32_t* d_run_ptr = nullptr;
+  grim::RunDesc* d_runs = nullptr;
+  int64_t nruns = 0;
   // dense bf16 copy for the tensor-core path is decompressed on the fly; nothing stored here
 };
 
@@ -159,6 +171,10 @@ grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 constexpr int kSkinnyMaxN = 16;  // widest right-hand side taken by the lane-per-column kernel
 grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
                             int64_t ldy, cudaStream_t s);
+// same product through per-warp rings filled by bulk asynchronous copies (persistent thread blocks)
+grim_status_t launch_stream(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
+                            int64_t ldy, cudaStream_t s);
+bool stream_path_supported(const grim_bcr* h, int64_t N);
 grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a);
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);

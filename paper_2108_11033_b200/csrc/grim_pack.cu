@@ -47,6 +47,8 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_chunks);
   cudaFree(h->d_colwords);
   cudaFree(h->d_gemv_vals);
+  cudaFree(h->d_run_ptr);
+  cudaFree(h->d_runs);
   cudaFree(h->d_rc_stage);
   cudaFree(h->d_rc_blob);
   cudaFree(h->d_tc_stage);
@@ -213,6 +215,8 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
     std::vector<ChunkDesc> chunks;
     std::vector<uint32_t> colwords;
     std::vector<uint8_t> gvals;
+    std::vector<uint32_t> run_ptr;
+    std::vector<RunDesc> runs;
     h->gemv_ok = K <= 65536;
     if (h->gemv_ok) {
       gvals.reserve((size_t)nnz * vsz);
@@ -271,11 +275,35 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       }
       gvals.resize(gvals.size() + 64 * vsz, 0);  // the kernels may read (and discard) up to a warp's width past a chunk
       band_ptr[(size_t)nbr] = (uint32_t)chunks.size();
+      // runs: the transfer units of the streaming kernel
+      run_ptr.assign((size_t)nbr + 1, 0);
+      for (int64_t pos = 0; pos < nbr; ++pos) {
+        run_ptr[(size_t)pos] = (uint32_t)runs.size();
+        uint32_t c = band_ptr[(size_t)pos];
+        const uint32_t ce = band_ptr[(size_t)pos + 1];
+        while (c < ce) {
+          runs.push_back(RunDesc{c, chunks[c].val_off});
+          size_t bytes = 0;
+          int n = 0;
+          while (c < ce && n < kRunChunks) {
+            const uint32_t nk = chunks[c].ncols_kr;
+            const size_t cb = (size_t)(nk & 0xFFFFu) * (nk >> 16) * vsz;
+            if (n > 0 && bytes + cb > (size_t)kRunValueBytes) break;
+            bytes += cb;
+            ++n;
+            ++c;
+          }
+        }
+      }
+      run_ptr[(size_t)nbr] = (uint32_t)runs.size();
+      runs.push_back(RunDesc{(uint32_t)chunks.size(), (uint32_t)gv_elems});
+      h->nruns = (int64_t)runs.size() - 1;
       h->nchunks = (int64_t)chunks.size();
       h->h_gemv_band_ptr = band_ptr;
       h->h_chunks = chunks;
       h->n_colwords = (int64_t)colwords.size();
-      h->index_bytes_gemv = (int64_t)colwords.size() * 4 + (int64_t)chunks.size() * (int64_t)sizeof(ChunkDesc) +
+      // what the streaming kernel reads besides the values: column words, the run table, the band tables
+      h->index_bytes_gemv = (int64_t)colwords.size() * 4 + (int64_t)runs.size() * (int64_t)sizeof(RunDesc) +
                             (nbr + 1) * 4 + nbr * 4;
     }
 
@@ -418,6 +446,8 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
         if (e == cudaSuccess) e = upload(&h->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkDesc));
         if (e == cudaSuccess) e = upload(&h->d_colwords, colwords.data(), colwords.size() * 4);
         if (e == cudaSuccess) e = upload((uint8_t**)&h->d_gemv_vals, gvals.data(), gvals.size());
+        if (e == cudaSuccess) e = upload(&h->d_run_ptr, run_ptr.data(), run_ptr.size() * 4);
+        if (e == cudaSuccess) e = upload(&h->d_runs, runs.data(), runs.size() * sizeof(RunDesc));
       }
       if (e != cudaSuccess) {
         st = (e == cudaErrorMemoryAllocation) ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;

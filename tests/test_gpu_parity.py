@@ -186,8 +186,30 @@ def test_lane_per_column_kernel_explicit(B, N):
     W = gen.dense_weight(M, K, seed=76)
     mask = gen.bcr_mask(M, K, bh, bw, compression=5, dist="uniform", seed=77)
     X = gen.normal_f32((K, N), 1.0, 78, 0)
-    check_spmm(B, W, mask, X, bh, bw, path=3)
-    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=3)
+    for variant in (0, 1, 2):  # default choice, values staged in registers, values streamed through shared memory
+        check_spmm(B, W, mask, X, bh, bw, path=3, tile_n=variant)
+        check_spmm(B, W, mask, X, bh, bw, bf16=True, path=3, tile_n=variant)
+
+
+STREAM_CASES = [
+    # M, K, bh, bw, generator kwargs: more bands than SMs, several bands per thread block, ragged edges
+    (3000, 1500, 8, 32, dict(compression=4, dist="uniform")),
+    (2500, 700, 16, 64, dict(compression=6, dist="zipf", empty_frac=0.1)),
+    (20001, 96, 4, 16, dict(compression=3, dist="uniform")),   # > 32 bands per thread block: several batches
+    (1190, 20000, 8, 32, dict(compression=16, dist="zipf")),   # vector too long for shared memory: gathered
+]
+
+
+@pytest.mark.parametrize("N", [1, 4, 9, 16])
+@pytest.mark.parametrize("case", STREAM_CASES)
+def test_streaming_kernel_explicit(B, case, N):
+    M, K, bh, bw, kw = case
+    W = gen.dense_weight(M, K, seed=170)
+    mask = gen.bcr_mask(M, K, bh, bw, seed=171, **kw)
+    mask[bh * 3:bh * 5] = 0  # two fully pruned bands
+    X = gen.normal_f32((K, N), 1.0, 172, 0)
+    check_spmm(B, W, mask, X, bh, bw, path=3, tile_n=2)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=3, tile_n=2, y_bf16=(N == 4))
 
 
 def test_spmm_strided_operands_and_errors(B):
