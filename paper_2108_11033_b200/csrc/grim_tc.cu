@@ -30,8 +30,8 @@ constexpr int kTcGroups = 3;       // the workers form groups that take K tiles 
 constexpr int kTcGroupWarps = kTcWorkers / kTcGroups;
 constexpr int kTcGroupThreads = 32 * kTcGroupWarps;
 constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
-constexpr int kTcBuilders = 8;     // convolution only: warps that build the X tile from the NCHW input
-constexpr int kTcBuildGroups = 2;
+constexpr int kTcBuilders = 12;    // convolution only: warps that build the X tile from the NCHW input
+constexpr int kTcBuildGroups = 3;  // they form groups that take K tiles in turn, like the expansion warps
 constexpr int kTcBuildGroupWarps = kTcBuilders / kTcBuildGroups;
 constexpr int kTcConvThreads = kTcThreads + 32 * kTcBuilders;
 constexpr int kTM = 128;          // rows of W per thread block
@@ -56,6 +56,9 @@ struct TcParams {
   uint32_t stage_bytes, rec_stride;
   unsigned spin_limit;
   int64_t in_elems;  // convolution: elements of the input tensor
+  int seg_off, seg_len;  // staged convolution: elements in front of the tile's first pixel / per channel segment
+  int nseg;              // staged convolution: slots of the ring of staged planes
+  uint32_t seg_bytes;    // bytes of one such slot
   SpmmArgs a;
 };
 
@@ -77,6 +80,14 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "r"(smem_u32(bar)), "r"(parity)
       : "memory");
   return ok != 0;
+}
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+  return v;
+}
+__device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v) {
+  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
 }
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
   for (unsigned i = 0; i < limit; ++i) {
@@ -143,7 +154,9 @@ __device__ __noinline__ uint4 im2col_piece_slow(const unsigned short* in1, int i
   return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
-template <int BH, bool CONV>
+// CONV: 0 = X is a matrix (TMA tiles); 1 = implicit im2col, the builders read the NCHW input from global memory;
+// 2 = implicit im2col, the input planes the tile needs are first staged in shared memory by bulk copies.
+template <int BH, int CONV>
 __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
@@ -158,10 +171,12 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   unsigned* s_done = reinterpret_cast<unsigned*>(smem + 640);    // [record slot] warps that have finished expanding it
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
+  uint64_t* seg_free = reinterpret_cast<uint64_t*>(smem + 704);  // staged convolution: the builders are done with a slot of planes
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 512);  // [record slot] bytes of the packed record (0: none)
   uint8_t* stages = smem + kTcHdrBytes;
   const uint32_t stage_bytes = p.stage_bytes;
   uint8_t* recs = stages + (size_t)p.nstages * stage_bytes;
+  uint8_t* segs = recs + (size_t)p.nrec * p.mt * p.rec_stride;  // staged convolution: ring of input planes
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
@@ -179,6 +194,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
       mbar_init(built + s, kTcBuildGroupWarps);
+      mbar_init(seg_free + s, kTcBuildGroupWarps);
     }
     for (int s = 0; s < kTcRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
@@ -230,6 +246,49 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
 #pragma unroll
         for (int i = 0; i < kTQ / 64; ++i)
           tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+      }
+    }
+    if (CONV == 2) {
+      // Staged implicit im2col: per K tile the (at most eight) input channels it touches, and of each the stretch
+      // of the plane that the tile's 256 pixels and their 3 x 3 neighbourhoods cover, one bulk copy per channel
+      // and image.  A channel's segment holds tile pixel q at element seg_off + q; where the tile runs into the
+      // next image that image's plane follows directly (taps that would cross the boundary are masked anyway).
+      const int ohw = a.OH * a.OW;
+      const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(a.X);
+      const int64_t q_end = q0 + kTQ < a.ncols ? q0 + kTQ : a.ncols;
+      const int n0 = (int)(q0 / ohw), n1 = (int)((q_end - 1) / ohw);
+      int src_lo[3], dst_idx[3];
+      unsigned nbytes[3], per_channel = 0;
+      const int nimg = n1 - n0 + 1;  // <= 3 (checked on the host)
+      for (int i = 0; i < nimg; ++i) {
+        const int64_t img0 = (int64_t)(n0 + i) * ohw;
+        const int qa = (int)((q0 > img0 ? q0 : img0) - q0);
+        const int qb = (int)((q_end < img0 + ohw ? q_end : img0 + ohw) - q0);
+        const int pa = (int)(q0 + qa - img0), pb = pa + (qb - qa);
+        const int lo = pa - p.seg_off > 0 ? pa - p.seg_off : 0;
+        const int hi = pb + p.seg_off < ohw ? pb + p.seg_off : ohw;
+        src_lo[i] = lo;
+        dst_idx[i] = lo - pa + qa + p.seg_off;
+        nbytes[i] = (unsigned)(hi - lo) * 2u;
+        per_channel += nbytes[i];
+      }
+      // the planes have a ring of their own, freed by the builders (long before the tensor core is done with
+      // the tile built from them), so their copies run several K tiles ahead
+      for (int kt = 0; kt < nkt; ++kt) {
+        const int ss = kt % p.nseg;
+        if (kt >= p.nseg && !__all_sync(0xffffffffu, mbar_wait(seg_free + ss, (unsigned)((kt / p.nseg - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 1; break; }
+        uint8_t* seg = segs + (size_t)ss * p.seg_bytes;
+        const int c_lo = kt * kTK / 9;
+        const int k_hi = (kt + 1) * kTK < p.K ? (kt + 1) * kTK - 1 : p.K - 1;
+        const int nch = k_hi / 9 - c_lo + 1;
+        if (lane == 0) mbar_arrive_expect_tx(full + ss, per_channel * (unsigned)nch);
+        __syncwarp();  // the byte count is announced before any copy can complete
+        // one copy per lane: a single thread needs several hundred cycles per copy it issues
+        for (int idx = lane; idx < nch * nimg; idx += 32) {
+          const int ci = idx / nimg, i = idx - ci * nimg;
+          bulk_load(seg + ((size_t)ci * p.seg_len + dst_idx[i]) * 2,
+                    in + ((int64_t)(n0 + i) * a.C + c_lo + ci) * ohw + src_lo[i], nbytes[i], full + ss);
+        }
       }
     }
   } else if (warp == 1) {
@@ -300,8 +359,74 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
     for (int kt = bgrp; kt < nkt; kt += kTcBuildGroups) {
       const int slot = kt % ns;
+      const int ss = CONV == 2 ? kt % p.nseg : 0;
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 3; break; }
+      // staged variant: the planes of this K tile have landed (their copies were requested several tiles ago)
+      if (CONV == 2 && !__all_sync(0xffffffffu, mbar_wait(full + ss, (unsigned)((kt / p.nseg) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 7; break; }
       uint8_t* bt_base = stages + (size_t)slot * stage_bytes + b_off + panel_off;
+      const uint4* seg16 = reinterpret_cast<const uint4*>(segs + (size_t)ss * p.seg_bytes);
+      if (CONV == 2) {
+        // Staged variant.  Row kk of the tile is k = (c, kh, kw); the warp takes rows w, w + 4, ... and keeps (c, tap)
+        // up to date without dividing.  Everything that depends on the row only is the same in all lanes: the first
+        // element of the row in the channel's segment (rb), hence the shift inside a vector; a lane adds its piece.
+        const int w0 = bt >> 5;
+        const uint32_t seg_s = smem_u32(seg16), bt_s = smem_u32(bt_base);
+        int c_rel = (kt * kTK + w0) / 9 - kt * kTK / 9;   // channel relative to the first one staged for this K tile
+        int tap = (kt * kTK + w0) % 9;
+        // rows in batches: first the shared-memory loads of the whole batch (so that their latencies overlap),
+        // then shifting, masking and storing
+        constexpr int kRows = 4;
+        for (int kk0 = w0; kk0 < kTK; kk0 += kTcBuildGroupWarps * kRows) {
+          uint4 lo[kRows], hi[kRows];
+          int rbs[kRows], taps[kRows];
+#pragma unroll
+          for (int bb = 0; bb < kRows; ++bb) {
+            const int kh = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0), kw = tap - 3 * kh;
+            const int rb = c_rel * p.seg_len + p.seg_off + (kh - 1) * a.W + (kw - 1);
+            rbs[bb] = rb;
+            taps[bb] = kh * 4 + kw;
+            lo[bb] = lds128(seg_s + (uint32_t)((rb >> 3) + cq) * 16u);
+            hi[bb] = lds128(seg_s + (uint32_t)((rb >> 3) + cq + 1) * 16u);
+            tap += kTcBuildGroupWarps;
+            if (tap >= 9) { tap -= 9; ++c_rel; }
+          }
+#pragma unroll
+          for (int bb = 0; bb < kRows; ++bb) {
+            const int kk = kk0 + bb * kTcBuildGroupWarps;
+            uint4 out = make_uint4(0u, 0u, 0u, 0u);
+            if (kt * kTK + kk < p.K) {
+              const uint4 l = lo[bb], h = hi[bb];
+              const int rb = rbs[bb], kh = taps[bb] >> 2, kw = taps[bb] & 3;
+              const int sb = (rb & 1) * 16;
+              switch ((rb >> 1) & 3) {  // 32-bit word of the vector pair at which the piece starts
+                case 0: out = make_uint4(__funnelshift_r(l.x, l.y, sb), __funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb)); break;
+                case 1: out = make_uint4(__funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb)); break;
+                case 2: out = make_uint4(__funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb)); break;
+                default: out = make_uint4(__funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb), __funnelshift_r(h.z, h.w, sb)); break;
+              }
+              const uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
+              if (bad) {  // clear the pixels whose tap lies outside the image
+                uint32_t w[4] = {out.x, out.y, out.z, out.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                  const uint32_t b2 = (bad >> (2 * i)) & 3u;
+                  w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
+                }
+                out = make_uint4(w[0], w[1], w[2], w[3]);
+              }
+            }
+            sts128(bt_s + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4), out);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(built + slot);
+          mbar_arrive(seg_free + ss);
+        }
+        continue;
+      }
+      const int c_lo = kt * kTK / 9;
       // The thread's 16 rows of the stage are taken in batches: first the address arithmetic and the vector loads
       // of the whole batch (so that they are in flight together), then shifting, masking, storing.
       constexpr int kBatch = 4;
@@ -529,25 +654,39 @@ EncodeTiledFn encode_tiled_fn() {
 
 size_t tc_stage_bytes(int mt) { return (size_t)mt * kATileBytes + kBTileBytes; }
 size_t tc_rec_stride(const grim_bcr* h) { return ((size_t)h->tc_max_rec + 127) & ~size_t(127); }
-size_t tc_smem_need(const grim_bcr* h, int mt, int stages, int nrec) {
-  return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(mt) + (size_t)nrec * mt * tc_rec_stride(h);
+// extra: bytes besides the operand tiles and the records (the ring of staged input planes of the convolution)
+size_t tc_smem_need(const grim_bcr* h, int mt, int stages, int nrec, size_t extra = 0) {
+  return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(mt) + (size_t)nrec * mt * tc_rec_stride(h) + extra;
 }
 // Ring sizes that fit: as many tile slots as possible first (they carry the bulk of the bytes in flight), then as
 // many record slots as are left, at least as many as tile slots.
 // At least as many tile slots as expansion groups: a group then never waits on a barrier that is more than one
 // phase behind it (parity waits cannot tell phases two apart).
-bool tc_rings(const grim_bcr* h, int mt, int* stages, int* nrec) {
+bool tc_rings(const grim_bcr* h, int mt, int* stages, int* nrec, size_t extra = 0) {
   for (int s = kTcStages; s >= kTcGroups; --s)
     for (int r = kTcRecSlots; r >= s; --r)
-      if (tc_smem_need(h, mt, s, r) <= 226 * 1024) { *stages = s; *nrec = r; return true; }
+      if (tc_smem_need(h, mt, s, r, extra) <= 226 * 1024) { *stages = s; *nrec = r; return true; }
   return false;
 }
 // Row tiles per thread block: two share every X tile (half the L2 traffic per flop, which is what bounds the
 // kernel) when that still leaves enough thread blocks for the GPU and three tile slots fit.
-int tc_row_tiles(const grim_bcr* h, int64_t qtiles) {
+int tc_row_tiles(const grim_bcr* h, int64_t qtiles, size_t extra = 0) {
   int s = 0, r = 0;
-  if (h->tc_mtiles >= 2 && qtiles * ((h->tc_mtiles + 1) / 2) >= 96 && tc_rings(h, 2, &s, &r) && s >= 3) return 2;
+  if (h->tc_mtiles >= 2 && qtiles * ((h->tc_mtiles + 1) / 2) >= 96 && tc_rings(h, 2, &s, &r, extra) && s >= 3) return 2;
   return 1;
+}
+// Staged implicit im2col: elements kept in front of the tile's first pixel in a channel segment (a row and a pixel,
+// rounded to vectors, plus one vector), the segment's length, and the bytes of one slot of the ring of planes (eight
+// channels at most touch a K tile of 64).  Needs planes that start and end on 16-byte boundaries and tiles that meet at most
+// three images.
+constexpr int kTcSegSlots = 4;  // slots of the ring of staged planes (its barriers share the tile ring's arrays)
+bool conv_staging(const SpmmArgs& a, int* seg_off, int* seg_len, size_t* seg_bytes) {
+  const int64_t ohw = (int64_t)a.OH * a.OW;
+  if (!a.conv || ohw % 8 != 0 || ohw < kTQ / 2) return false;
+  *seg_off = (a.W + 1 + 7) / 8 * 8 + 8;
+  *seg_len = kTQ + 2 * *seg_off;
+  *seg_bytes = ((size_t)8 * *seg_len * 2 + 16 + 127) / 128 * 128;
+  return true;
 }
 
 }  // namespace
@@ -577,9 +716,25 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;
   const int64_t qtiles_ = (a.ncols + kTQ - 1) / kTQ;
-  p.mt = (a.tile_n == 1 || a.tile_n == 2) ? a.tile_n : tc_row_tiles(h, qtiles_);
+  size_t extra = 0, seg_bytes = 0;
+  p.seg_off = p.seg_len = 0;
+  p.nseg = kTcSegSlots;
+  bool staged = conv_staging(a, &p.seg_off, &p.seg_len, &seg_bytes);
+  const int want_mt = (a.tile_n == 1 || a.tile_n == 2) ? a.tile_n : tc_row_tiles(h, qtiles_, 0);
+  if (staged) {
+    // the ring of planes is as deep as shared memory allows without giving up the second row tile (which halves the
+    // tile-building work per output); without room for even two slots the planes are read from global memory
+    staged = false;
+    for (int n = kTcSegSlots; n >= 2 && !staged; --n) {
+      int s_ = 0, r_ = 0;
+      if (tc_rings(h, want_mt, &s_, &r_, n * seg_bytes) && (want_mt == 1 || s_ >= 3)) { p.nseg = n; staged = true; }
+    }
+  }
+  extra = staged ? p.nseg * seg_bytes : 0;
+  p.seg_bytes = (uint32_t)seg_bytes;
+  p.mt = want_mt;
   p.mtiles = (int)h->tc_mtiles;
-  if (!tc_rings(h, p.mt, &p.nstages, &p.nrec)) { p.mt = 1; tc_rings(h, 1, &p.nstages, &p.nrec); }
+  if (!tc_rings(h, p.mt, &p.nstages, &p.nrec, extra)) { p.mt = 1; tc_rings(h, 1, &p.nstages, &p.nrec, extra); }
   p.stage_bytes = (uint32_t)tc_stage_bytes(p.mt);
   p.rec_stride = (uint32_t)tc_rec_stride(h);
   p.spin_limit = 1u << 20;
@@ -589,8 +744,9 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
   if (a.conv) {
-    auto kern = h->bh == 4 ? bcr_tc_kernel<4, true> : (h->bh == 8 ? bcr_tc_kernel<8, true> : bcr_tc_kernel<16, true>);
-    const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec);
+    auto kern = staged ? (h->bh == 4 ? bcr_tc_kernel<4, 2> : (h->bh == 8 ? bcr_tc_kernel<8, 2> : bcr_tc_kernel<16, 2>))
+                       : (h->bh == 4 ? bcr_tc_kernel<4, 1> : (h->bh == 8 ? bcr_tc_kernel<8, 1> : bcr_tc_kernel<16, 1>));
+    const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec, extra);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
     dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt));
     kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
@@ -606,7 +762,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
   const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec);
-  auto kern = h->bh == 4 ? bcr_tc_kernel<4, false> : (h->bh == 8 ? bcr_tc_kernel<8, false> : bcr_tc_kernel<16, false>);
+  auto kern = h->bh == 4 ? bcr_tc_kernel<4, 0> : (h->bh == 8 ? bcr_tc_kernel<8, 0> : bcr_tc_kernel<16, 0>);
   cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;

@@ -387,6 +387,24 @@ def test_conv_bf16_batch_crossing_images(B):
     check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
 
 
+@pytest.mark.parametrize("shape", [(12, 12, 7), (8, 16, 9), (16, 10, 5), (24, 16, 3)])
+@pytest.mark.parametrize("bh", [4, 8, 16])
+def test_conv_bf16_staged_planes(B, shape, bh):
+    """Tensor-core convolution on planes whose size is a multiple of 8 pixels (the variant that stages the input
+    planes in shared memory): 256-pixel tiles that meet two or three images, a ragged last tile, several K tiles,
+    all block heights."""
+    H, Wd, batch = shape
+    C, Cout, bw = 20, 136, 32
+    rng_seed = 300 + H + Wd + bh
+    W = gen.dense_weight(Cout, C * 9, seed=rng_seed)
+    mask = gen.bcr_mask(Cout, C * 9, bh, bw, compression=4, dist="uniform", seed=rng_seed + 1)
+    bias = gen.normal_f32((Cout,), 0.1, rng_seed + 2, 0)
+    x = np.maximum(gen.normal_f32((batch, C, H, Wd), 1.0, rng_seed + 3, 0), 0)
+    L = dict(W=W, mask=mask, bias=bias, bh=bh, bw=bw)
+    check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True)
+    check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
+
+
 # ---------------------------------------------------------------------------------------- GRU
 
 
