@@ -92,6 +92,7 @@ __device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v) {
 __device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
   for (unsigned i = 0; i < limit; ++i) {
     if (mbar_try_wait(bar, parity)) return true;
+    __nanosleep(100);  // most warps of the block wait at any time: polling flat out takes issue slots from the others
     if ((i & 63u) == 63u && *abort_flag) return false;
   }
   return false;
