@@ -100,6 +100,26 @@ struct GruParams {
   const uint32_t* img_col;
 };
 
+__device__ __forceinline__ void gru_mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void gru_mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool gru_mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"((uint32_t)__cvta_generic_to_shared(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
+// Stores v at the place of CTA-local shared address `local` in CTA `rank` of the cluster and counts its 4 bytes on
+// that CTA's mbarrier at CTA-local address `bar_local`.
+__device__ __forceinline__ void gru_st_async_f32(uint32_t local, uint32_t bar_local, uint32_t rank, float v) {
+  uint32_t raddr, rbar;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(raddr) : "r"(local), "r"(rank));
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(rbar) : "r"(bar_local), "r"(rank));
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.f32 [%0], %1, [%2];" ::"r"(raddr), "f"(v), "r"(rbar) : "memory");
+}
 __device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -345,8 +365,9 @@ __global__ void __launch_bounds__(1024, 1) gru_cluster_kernel(const GruParams p)
 }
 
 // ---------------------------------------------------------------------------------------------
-// cluster version with W_hh in registers.  Same exchange as gru_cluster_kernel, but every warp keeps its
-// share of the bands in registers for the whole sequence: a band is cut in two halves (work items), an
+// cluster version with W_hh in registers.  Every warp keeps its share of the bands in registers for the whole
+// sequence, and the new state travels by asynchronous shared-memory stores counted on mbarriers instead of through a
+// cluster barrier (whose release / acquire pair was the largest stall of a step): a band is cut in two halves (work items), an
 // item's kept columns are dealt to S slots x 32 lanes, and a lane holds per slot the column index and
 // the column's BH values expanded to row positions (zeros where the row is not kept).  A time step then
 // costs one shared-memory gather of h and BH FMAs per slot - no index decoding, no predicates.
@@ -397,11 +418,27 @@ __global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const G
       gi[g] = __ldg(p.gi + g * H + unit);
     }
   for (int i = tid; i < H; i += kRegThreads) hs[i] = p.h0 ? p.h0[i] : 0.f;
+  // The state exchange: the thread that owns a hidden unit sends its new value into the next-step buffer of every
+  // CTA of the cluster with asynchronous stores that count their bytes on the receiver's mbarrier; a CTA starts a
+  // step when the H values of that step have been counted.  No cluster-wide barrier and no fence per step: a
+  // buffer is written again only after every CTA has received the whole state computed from it, i.e. after every
+  // warp of the cluster is done reading it.
+  uint64_t* hbar = reinterpret_cast<uint64_t*>(partial + nb * 2 * BH);  // [2], 8-byte aligned (all counts are even)
+  if (tid == 0) {
+    gru_mbar_init(hbar, 1);
+    gru_mbar_init(hbar + 1, 1);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
   cluster.sync();
+  const uint32_t hs_local = (uint32_t)__cvta_generic_to_shared(hs), bar_local = (uint32_t)__cvta_generic_to_shared(hbar);
+  bool failed = false;
 
   for (int t = 0; t < p.T; ++t) {
-    const float* hcur = hs + (t & 1) * H;
-    float* hnxt_local = hs + ((t + 1) & 1) * H;
+    const int cur = t & 1, nxt = cur ^ 1;
+    const float* hcur = hs + cur * H;
+    // this step's outputs arrive on the next buffer's barrier: announce the byte count (fast CTAs may already be
+    // sending, which drives the count negative; the pending arrival keeps the phase open until it is announced)
+    if (tid == 0 && t + 1 < p.T) gru_mbar_arrive_expect_tx(hbar + nxt, (unsigned)H * 4u);
     // pre-activations of the next step are fetched now so that their DRAM latency hides behind this step
     float gi_next[3] = {0.f, 0.f, 0.f};
     if (gate_live && t + 1 < p.T)
@@ -422,21 +459,40 @@ __global__ void __launch_bounds__(kRegThreads, 1) gru_cluster_reg_kernel(const G
       if (item < nb * 2) partial[item * BH + warp_row<BH>(lane)] = acc[0];
     }
     __syncthreads();
+    float hnew_val = 0.f;
     if (gate_live) {
-      // the thread that owns a hidden unit computes it and sends it straight to the next-step buffer of every CTA
-      // of the cluster (no staging, no second block barrier)
+      // the thread that owns a hidden unit computes it; below it is sent straight to the next-step buffer of every CTA
       const float hn = gru_gate(partial, bq, gi, g_tri, g_r, 2, BH, hcur[unit]);
+      hnew_val = hn;
       p.out[(int64_t)t * H + unit] = hn;
       if (p.outT) p.outT[(int64_t)unit * p.ldT + t] = hn;
       if (t == p.T - 1 && p.hT) p.hT[unit] = hn;
-      float* mine = hnxt_local + unit;
+    }
+    if (gate_live && t + 1 < p.T) {
+      // one 4-byte store per destination (pooling four neighbours' values into 16-byte stores was slower: the
+      // shuffles lengthen the chain more than the fewer messages save)
+      const uint32_t dst_local = hs_local + (uint32_t)(nxt * H + unit) * 4u, bar_nxt = bar_local + (uint32_t)nxt * 8u;
 #pragma unroll 4
-      for (int dst = 0; dst < CS; ++dst) *cluster.map_shared_rank(mine, dst) = hn;
+      for (int dst = 0; dst < CS; ++dst) gru_st_async_f32(dst_local, bar_nxt, (uint32_t)dst, hnew_val);
     }
 #pragma unroll
     for (int g = 0; g < 3; ++g) gi[g] = gi_next[g];
-    cluster.sync();
+    if (t + 1 < p.T && warp == 0) {
+      // the next step's state: bounded wait on the local barrier (its (t / 2)-th use).  One thread polls for the
+      // whole block; the others sleep in the block barrier below (many pollers slow the arrival of the stores down)
+      const unsigned parity = (unsigned)((t >> 1) & 1);
+      bool ok = false;
+      if (lane == 0)
+        for (unsigned it = 0; it < p.spin_limit && !ok; ++it) ok = gru_mbar_try_wait(hbar + nxt, parity);
+      __syncwarp();
+      if (!__shfl_sync(0xffffffffu, ok, 0)) {
+        failed = true;
+        if (lane == 0) atomicExch(p.status, (unsigned)GRIM_ERR_TIMEOUT);
+      }
+    }
+    if (__syncthreads_or(failed ? 1 : 0)) break;  // the state of the next step is there (or a wait ran out)
   }
+  cluster.sync();  // no CTA leaves while another may still address its shared memory
 }
 
 size_t smem_bytes(const grim_gru* g, const ModeCfg& m, int BH, bool cluster) {
@@ -733,7 +789,7 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
         for (const auto& v : menu) {
           if (v[0] < ni_needed || v[1] < slots_needed || !reg_kernel(BHc, v[0], v[1])) continue;
           t.ctas = cs; t.ks = 2; t.threads = kRegThreads; t.resident = 1;
-          t.smem = (((size_t)2 * H + (size_t)((t.tpc * bh + 3) & ~3) + (size_t)nb * 2 * BHc) * 4 + 15) & ~size_t(15);
+          t.smem = ((((size_t)2 * H + (size_t)((t.tpc * bh + 3) & ~3) + (size_t)nb * 2 * BHc) * 4 + 15) & ~size_t(15)) + 16;  // + the two state barriers
           if (t.smem > kSmemLimit || !cluster_fits(reg_kernel(BHc, v[0], v[1]), t)) continue;
           t.ok = true;
           g->regc = t; g->reg_ni = v[0]; g->reg_s = v[1];

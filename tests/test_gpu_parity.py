@@ -200,6 +200,27 @@ STREAM_CASES = [
 ]
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+def test_small_n_edge_cases(B, bf16):
+    """Default routing for N <= 16 on degenerate shapes: nothing kept at all, a single band shorter than a block, a
+    matrix narrower than a block, one kept element, and the widest K the 16-bit column words can address."""
+    for M, K, bh, bw, kw in [
+        (40, 64, 8, 32, dict(compression=4, dist="uniform", empty_frac=1.0)),   # every block empty
+        (5, 300, 8, 32, dict(compression=2, dist="uniform")),                   # one ragged band
+        (100, 7, 4, 16, dict(compression=2, dist="uniform")),                   # K smaller than a block
+        (64, 65536, 16, 64, dict(compression=64, dist="zipf")),                 # widest K of the chunk layout
+    ]:
+        W = gen.dense_weight(M, K, seed=180)
+        mask = gen.bcr_mask(M, K, bh, bw, seed=181, **kw)
+        for N in (1, 3, 16):
+            X = gen.normal_f32((K, N), 1.0, 182, N)
+            check_spmm(B, W, mask, X, bh, bw, bf16=bf16)
+    W = gen.dense_weight(24, 96, seed=183)
+    mask = np.zeros((24, 96), np.uint8)
+    mask[9, 70] = 1  # a single kept element
+    check_spmm(B, W, mask, gen.normal_f32((96, 1), 1.0, 184, 0), 8, 32, bf16=bf16)
+
+
 @pytest.mark.parametrize("N", [1, 4, 9, 16])
 @pytest.mark.parametrize("case", STREAM_CASES)
 def test_streaming_kernel_explicit(B, case, N):
