@@ -146,7 +146,11 @@ grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);
  * after fp32 accumulation).  Y is fully overwritten (all M rows, beta = 0): rows kept by no
  * block are written as +0.  N = 1 selects the matrix-vector kernel.  X and Y must not overlap.
  * Shape mismatch -> GRIM_ERR_SHAPE, dtype mismatch -> GRIM_ERR_DTYPE, both before any launch.
- * Asynchronous on `stream`.
+ * Asynchronous on `stream`.  One exception: a bf16 handle whose tensor-core multiply has few output
+ * tiles and a long K is split over K through an fp32 scratch of M x N floats that the handle owns;
+ * the call that first needs it (or needs a larger one) allocates it with cudaMalloc, which
+ * synchronises - make that call once before capturing a stream or entering a timed region.  The
+ * same holds for grim_bcr_conv2d.  A handle is used on one stream at a time.
  */
 grim_status_t grim_bcr_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, grim_stream_t stream);
 

@@ -133,6 +133,8 @@ struct grim_bcr {
   int64_t index_bytes_tc = 0;
   grim::RcStage* d_tc_stage = nullptr;
   uint8_t* d_tc_blob = nullptr;
+  float* d_tc_acc = nullptr;  // fp32 scratch of the split tensor-core multiply (M x N), grown on first use
+  size_t tc_acc_bytes = 0;
   unsigned* d_status = nullptr;  // error word written by kernels whose bounded waits ran out
   grim::StageEntry* d_stage = nullptr;
   uint8_t* d_blob = nullptr;

@@ -47,6 +47,7 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_chunks);
   cudaFree(h->d_colwords);
   cudaFree(h->d_gemv_vals);
+  cudaFree(h->d_tc_acc);
   cudaFree(h->d_run_ptr);
   cudaFree(h->d_runs);
   cudaFree(h->d_rc_stage);

@@ -58,6 +58,8 @@ struct TcParams {
   int64_t in_elems;  // convolution: elements of the input tensor
   int seg_off, seg_len;  // staged convolution: elements in front of the tile's first pixel / per channel segment
   int nseg;              // staged convolution: slots of the ring of staged planes
+  int ksplit, kt_per;    // > 1: blockIdx.z takes kt_per K tiles and adds its partial sums into the fp32 scratch `acc`
+  float* acc;            // [M][ncols] when ksplit > 1
   uint32_t seg_bytes;    // bytes of one such slot
   SpmmArgs a;
 };
@@ -186,7 +188,10 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   const int pos0 = blockIdx.y * p.mt * p.slots_per_tile;  // first band (schedule position) of this thread block's rows
   const uint32_t b_off = (uint32_t)p.mt * kATileBytes;     // the X tile follows the weight tiles in a stage
   const uint32_t tmem_cols = kTmemCols * (uint32_t)p.mt;
-  const int nkt = p.nkt, ns = p.nstages, nr = p.nrec;
+  // K tiles of this thread block: all of them, or its share of a split multiply; kt below counts them from 0
+  const int kbase = p.ksplit > 1 ? (int)blockIdx.z * p.kt_per : 0;
+  const int nkt = p.ksplit > 1 ? (p.nkt - kbase < p.kt_per ? p.nkt - kbase : p.kt_per) : p.nkt;
+  const int ns = p.nstages, nr = p.nrec;
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
@@ -220,7 +225,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     for (int m = 0; m < p.mt; ++m) {
       const int t = (int)blockIdx.y * p.mt + m;
       if (t < p.mtiles) {
-        const RcStage se = p.stage[(int64_t)t * nkt + k];
+        const RcStage se = p.stage[(int64_t)t * p.nkt + kbase + k];
         bytes[m] = se.bytes; off[m] = se.off16;
       }
       s_meta[rs * 2 + m] = bytes[m];
@@ -246,7 +251,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         mbar_arrive_expect_tx(full + slot, (unsigned)kBTileBytes);
 #pragma unroll
         for (int i = 0; i < kTQ / 64; ++i)
-          tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, kt * kTK, full + slot);
+          tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, (kbase + kt) * kTK, full + slot);
       }
     }
     if (CONV == 2) {
@@ -279,8 +284,8 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         const int ss = kt % p.nseg;
         if (kt >= p.nseg && !__all_sync(0xffffffffu, mbar_wait(seg_free + ss, (unsigned)((kt / p.nseg - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 1; break; }
         uint8_t* seg = segs + (size_t)ss * p.seg_bytes;
-        const int c_lo = kt * kTK / 9;
-        const int k_hi = (kt + 1) * kTK < p.K ? (kt + 1) * kTK - 1 : p.K - 1;
+        const int c_lo = (kbase + kt) * kTK / 9;
+        const int k_hi = (kbase + kt + 1) * kTK < p.K ? (kbase + kt + 1) * kTK - 1 : p.K - 1;
         const int nch = k_hi / 9 - c_lo + 1;
         if (lane == 0) mbar_arrive_expect_tx(full + ss, per_channel * (unsigned)nch);
         __syncwarp();  // the byte count is announced before any copy can complete
@@ -372,8 +377,9 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         // element of the row in the channel's segment (rb), hence the shift inside a vector; a lane adds its piece.
         const int w0 = bt >> 5;
         const uint32_t seg_s = smem_u32(seg16), bt_s = smem_u32(bt_base);
-        int c_rel = (kt * kTK + w0) / 9 - kt * kTK / 9;   // channel relative to the first one staged for this K tile
-        int tap = (kt * kTK + w0) % 9;
+        const int k0 = (kbase + kt) * kTK;  // first k of this tile
+        int c_rel = (k0 + w0) / 9 - k0 / 9;   // channel relative to the first one staged for this K tile
+        int tap = (k0 + w0) % 9;
         // rows in batches: first the shared-memory loads of the whole batch (so that their latencies overlap),
         // then shifting, masking and storing
         constexpr int kRows = 4;
@@ -395,7 +401,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
           for (int bb = 0; bb < kRows; ++bb) {
             const int kk = kk0 + bb * kTcBuildGroupWarps;
             uint4 out = make_uint4(0u, 0u, 0u, 0u);
-            if (kt * kTK + kk < p.K) {
+            if (k0 + kk < p.K) {
               const uint4 l = lo[bb], h = hi[bb];
               const int rb = rbs[bb], kh = taps[bb] >> 2, kw = taps[bb] & 3;
               const int sb = (rb & 1) * 16;
@@ -427,7 +433,6 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         }
         continue;
       }
-      const int c_lo = kt * kTK / 9;
       // The thread's 16 rows of the stage are taken in batches: first the address arithmetic and the vector loads
       // of the whole batch (so that they are in flight together), then shifting, masking, storing.
       constexpr int kBatch = 4;
@@ -437,7 +442,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
 #pragma unroll
         for (int bb = 0; bb < kBatch; ++bb) {
           const int kk = kk0 + bb * kTcBuildGroupWarps;
-          const int kg = kt * kTK + kk;
+          const int kg = (kbase + kt) * kTK + kk;
           lo[bb] = make_uint4(0u, 0u, 0u, 0u);
           hi[bb] = make_uint4(0u, 0u, 0u, 0u);
           info[bb] = 0;
@@ -480,7 +485,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
               out = make_uint4(w[0], w[1], w[2], w[3]);
             }
           } else if (mode == 2u) {
-            const int kg = kt * kTK + kk;
+            const int kg = (kbase + kt) * kTK + kk;
             const int c = kg / 9, tap = kg - c * 9;
             const int kh = tap / 3, kw = tap - kh * 3;
             out = im2col_piece_slow(in1, in_elems, plane0, plane1, c * ohw, pix0, split, (kh - 1) * a.W + (kw - 1), bad);
@@ -572,6 +577,13 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(m * (int)kTmemCols + cb * 32), v);
         const int64_t q = q0 + cb * 32;
         if (!row_ok || q >= a.ncols) continue;
+        if (p.ksplit > 1) {
+          // split multiply: partial sums go to the zeroed fp32 scratch; bias, activation and the output layout are
+          // applied by a pass over the scratch when all parts are in
+          float* dst = p.acc + row * a.ncols + q;
+          for (int i = 0; i < 32 && q + i < a.ncols; ++i) atomicAdd(dst + i, __uint_as_float(v[i]));
+          continue;
+        }
         float t[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
@@ -633,6 +645,24 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   if (warp == 1) {
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(tmem_cols) : "memory");
+  }
+}
+
+// Second pass of a split multiply: scratch + bias -> activation -> Y in its layout and type.
+__global__ void tc_finalize_kernel(const float* __restrict__ acc, int64_t ncols, int M, const float* __restrict__ bias, int relu,
+                                   void* Y, int y_dtype, int64_t y_sr, int conv, int64_t ohw) {
+  const int64_t total = (int64_t)M * ncols;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t row = i / ncols, q = i - row * ncols;
+    float v = acc[i] + (bias ? __ldg(bias + row) : 0.f);
+    if (relu) v = fmaxf(v, 0.f);
+    int64_t off = row * y_sr + q;
+    if (conv) {
+      const int64_t img = q / ohw, pix = q - img * ohw;
+      off = (img * M + row) * ohw + pix;
+    }
+    if (y_dtype == GRIM_F32) static_cast<float*>(Y)[off] = v;
+    else static_cast<__nv_bfloat16*>(Y)[off] = __float2bfloat16_rn(v);
   }
 }
 
@@ -742,6 +772,42 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.a = a;
 
   p.in_elems = a.conv ? a.ncols / ((int64_t)a.OH * a.OW) * a.C * a.H * a.W : 0;
+  // Split over K when the grid would leave most of the GPU idle (small pixel or column counts): several thread
+  // blocks share an output tile, each takes a run of K tiles and adds its partial sums into an fp32 scratch that the
+  // handle owns (grown on first use), and a second pass applies bias, activation and the output layout.
+  p.ksplit = 1; p.kt_per = p.nkt; p.acc = nullptr;
+  {
+    const int64_t blocks = qtiles_ * ((h->tc_mtiles + p.mt - 1) / p.mt);
+    const int sms = 148;
+    int want = (int)std::min<int64_t>(16, sms / std::max<int64_t>(blocks, 1));
+    want = std::min(want, p.nkt / 4);  // at least four K tiles per part
+    const size_t need = (size_t)h->M * (size_t)a.ncols * 4;
+    if (want >= 2 && blocks * 2 <= sms && need <= ((size_t)1 << 30)) {
+      grim_bcr* hm = const_cast<grim_bcr*>(h);
+      if (hm->tc_acc_bytes < need) {
+        cudaFree(hm->d_tc_acc);
+        hm->d_tc_acc = nullptr; hm->tc_acc_bytes = 0;
+        if (cudaMalloc(&hm->d_tc_acc, need) == cudaSuccess) hm->tc_acc_bytes = need;
+        else cudaGetLastError();
+      }
+      if (hm->d_tc_acc) {
+        p.kt_per = (p.nkt + want - 1) / want;
+        p.ksplit = (p.nkt + p.kt_per - 1) / p.kt_per;
+        p.acc = hm->d_tc_acc;
+        if (p.ksplit < 2) { p.ksplit = 1; p.kt_per = p.nkt; p.acc = nullptr; }
+        else if (cudaMemsetAsync(p.acc, 0, need, s) != cudaSuccess) return GRIM_ERR_CUDA;
+      }
+    }
+  }
+  auto finalize = [&]() -> grim_status_t {
+    if (p.ksplit <= 1) return GRIM_OK;
+    const int64_t total = (int64_t)h->M * a.ncols;
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 8);
+    tc_finalize_kernel<<<blocks, 256, 0, s>>>(p.acc, a.ncols, (int)h->M, a.bias, a.relu, a.Y, a.y_dtype, a.y_sr, a.conv,
+                                              (int64_t)a.OH * a.OW);
+    count_launch();
+    return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+  };
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
   if (a.conv) {
@@ -749,10 +815,11 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                        : (h->bh == 4 ? bcr_tc_kernel<4, 1> : (h->bh == 8 ? bcr_tc_kernel<8, 1> : bcr_tc_kernel<16, 1>));
     const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec, extra);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
-    dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt));
+    dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt), (unsigned)p.ksplit);
     kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+    if (cudaGetLastError() != cudaSuccess) return GRIM_ERR_CUDA;
+    return finalize();
   }
   const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
   const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * 2)};
@@ -768,10 +835,11 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
   const int64_t mtiles = (h->tc_mtiles + p.mt - 1) / p.mt;
-  dim3 grid((unsigned)qtiles, (unsigned)mtiles);
+  dim3 grid((unsigned)qtiles, (unsigned)mtiles, (unsigned)p.ksplit);
   kern<<<grid, kTcThreads, smem, s>>>(tm, p);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+  if (cudaGetLastError() != cudaSuccess) return GRIM_ERR_CUDA;
+  return finalize();
 }
 
 }  // namespace grim

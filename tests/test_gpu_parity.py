@@ -426,6 +426,25 @@ def test_conv_bf16_staged_planes(B, shape, bh):
     check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
 
 
+@pytest.mark.parametrize("y_bf16", [False, True])
+def test_tensor_core_split_over_k(B, y_bf16):
+    """Few output tiles and a long K: the tensor-core multiply is split over K (partial sums through the fp32
+    scratch, second pass for the output), matrix and convolution forms, with pruned bands and a ragged last K tile."""
+    M, K, bh, bw = 300, 2100, 8, 32
+    W = gen.dense_weight(M, K, seed=310)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=311)
+    mask[16:32] = 0
+    X = gen.normal_f32((K, 304), 1.0, 312, 0)  # row stride a multiple of 16 bytes (TMA)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=2, y_bf16=y_bf16)
+    C, Cout = 72, 200
+    Wc = gen.dense_weight(Cout, C * 9, seed=313)
+    maskc = gen.bcr_mask(Cout, C * 9, 16, 64, compression=5, dist="uniform", seed=314)
+    L = dict(W=Wc, mask=maskc, bias=gen.normal_f32((Cout,), 0.1, 315, 0), bh=16, bw=64)
+    for H, Wd, batch in ((12, 12, 3), (7, 9, 2)):  # staged planes / planes read from global memory
+        x = np.maximum(gen.normal_f32((batch, C, H, Wd), 1.0, 316, H), 0)
+        check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, out_bf16=y_bf16)
+
+
 # ---------------------------------------------------------------------------------------- GRU
 
 
