@@ -430,13 +430,13 @@ def test_conv_bf16_staged_planes(B, shape, bh):
 def test_tensor_core_split_over_k(B, y_bf16):
     """Few output tiles and a long K: the tensor-core multiply is split over K (partial sums through the fp32
     scratch, second pass for the output), matrix and convolution forms, with pruned bands and a ragged last K tile."""
-    M, K, bh, bw = 300, 2100, 8, 32
+    M, K, bh, bw = 300, 3100, 8, 32
     W = gen.dense_weight(M, K, seed=310)
     mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=311)
     mask[16:32] = 0
     X = gen.normal_f32((K, 304), 1.0, 312, 0)  # row stride a multiple of 16 bytes (TMA)
     check_spmm(B, W, mask, X, bh, bw, bf16=True, path=2, y_bf16=y_bf16)
-    C, Cout = 72, 200
+    C, Cout = 176, 200
     Wc = gen.dense_weight(Cout, C * 9, seed=313)
     maskc = gen.bcr_mask(Cout, C * 9, 16, 64, compression=5, dist="uniform", seed=314)
     L = dict(W=Wc, mask=maskc, bias=gen.normal_f32((Cout,), 0.1, 315, 0), bh=16, bw=64)
