@@ -42,3 +42,16 @@ def test_single_process_reduction_is_the_identity():
     sys.path.insert(0, ROOT)
     import bench
     assert bench.max_over_ranks([1.5, 2.5]) == [1.5, 2.5]
+
+
+def test_rotation_sets_cover_l2_or_fall_back_to_flushing():
+    """Timed steps rotate through operand sets so that a set has left L2 before its next use: the sets touched in
+    between must exceed the L2 size; a working set too small for a reasonable number of copies is flushed instead."""
+    sys.path.insert(0, ROOT)
+    import bench
+    assert bench.rotation_sets(84e6) == 3            # the 8192 x 8192 4x GEMV: two other sets = 168 MB > L2
+    assert bench.rotation_sets(400e6) == 2           # larger than L2 by itself: one other set is enough
+    assert bench.rotation_sets(1e6) == 1             # would need > 12 copies: timed one launch at a time after a flush
+    for ws in (15e6, 30e6, 60e6, 100e6, 200e6):
+        n = bench.rotation_sets(ws)
+        assert n == 1 or (n - 1) * ws >= bench.L2_BYTES, (ws, n)
