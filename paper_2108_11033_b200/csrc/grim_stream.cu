@@ -169,7 +169,11 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
   const uint32_t ring_off = p.off_ring + (uint32_t)warp * p.nslots * p.stage_bytes;  // this warp's ring, from the base
   uint8_t* ring = smem + ring_off;
   uint64_t* my_full = full + warp * kSMaxSlots;
-  const int nk = (p.nbr - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;  // bands of this thread block
+  // Bands are scheduled heaviest first; thread blocks take them in rounds of gridDim.x, forwards in even rounds and
+  // backwards in odd ones, so that no block collects the heaviest band of every round.
+  const int grid = (int)gridDim.x, bid = (int)blockIdx.x;
+  const int nfull = p.nbr / grid, rem = p.nbr - nfull * grid;
+  const int nk = nfull + ((((nfull & 1) ? grid - 1 - bid : bid) < rem) ? 1 : 0);  // bands of this thread block
   const int q0 = blockIdx.y * NQ;
   const int nslots = p.nslots;
 
@@ -179,7 +183,7 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   for (int k = threadIdx.x; k < nk; k += NW * 32) {
-    const int pos = blockIdx.x + k * gridDim.x;
+    const int pos = k * grid + ((k & 1) ? grid - 1 - bid : bid);
     s_band[k] = make_uint2(p.run_ptr[pos], p.run_ptr[pos + 1]);
     s_first_row[k] = p.band_order[pos] * (uint32_t)p.bh;
   }
