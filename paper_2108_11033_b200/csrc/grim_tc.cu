@@ -788,12 +788,12 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   {
     const int64_t blocks = qtiles_ * ((h->tc_mtiles + p.mt - 1) / p.mt);
     const int sms = 148;
-    // (measured on the VGG-16 layers: worth it from about 24 K tiles per block; with fewer, clearing the scratch,
-    // the atomic adds and the second pass cost more than the shorter K loop saves)
+    // (measured on the VGG-16 layers: worth it from about 16 K tiles per block; with fewer, clearing the scratch,
+    // the reductions into it and the second pass cost more than the shorter K loop saves)
     int want = (int)std::min<int64_t>(16, sms / std::max<int64_t>(blocks, 1));
-    want = std::min(want, p.nkt / 6);  // at least six K tiles per part
+    want = std::min(want, p.nkt / 4);  // at least four K tiles per part
     const size_t need = (size_t)h->M * (size_t)a.ncols * 4;
-    if (want >= 2 && p.nkt >= 24 && blocks * 2 <= sms && need <= ((size_t)1 << 30)) {
+    if (want >= 2 && p.nkt >= 16 && blocks * 2 <= sms && need <= ((size_t)1 << 30)) {
       grim_bcr* hm = const_cast<grim_bcr*>(h);
       if (hm->tc_acc_bytes < need) {
         cudaFree(hm->d_tc_acc);
