@@ -83,6 +83,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
+__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
 __device__ __forceinline__ uint4 lds128(uint32_t saddr) {
   uint4 v;
   asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
@@ -158,7 +164,9 @@ __device__ __noinline__ uint4 im2col_piece_slow(const unsigned short* in1, int i
 }
 
 // CONV: 0 = X is a matrix (TMA tiles); 1 = implicit im2col, the builders read the NCHW input from global memory;
-// 2 = implicit im2col, the input planes the tile needs are first staged in shared memory by bulk copies.
+// 2 = implicit im2col, the input planes the tile needs are first staged in shared memory by bulk copies; 3 = the same
+// with 8-byte asynchronous copies per lane, for planes whose size is a multiple of 4 but not of 8 pixels (their starts
+// are not all 16-byte aligned).
 template <int BH, int CONV>
 __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
@@ -195,7 +203,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
-      mbar_init(full + s, 1);
+      mbar_init(full + s, CONV == 3 ? 32u : 1u);  // completed by TMA byte counts, or by the copy warp's 32 lanes
       mbar_init(zeroed + s, kTcGroupWarps);
       mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
@@ -254,7 +262,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
           tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, (kbase + kt) * kTK, full + slot);
       }
     }
-    if (CONV == 2) {
+    if (CONV >= 2) {
       // Staged implicit im2col: per K tile the (at most eight) input channels it touches, and of each the stretch
       // of the plane that the tile's 256 pixels and their 3 x 3 neighbourhoods cover, one bulk copy per channel
       // and image.  A channel's segment holds tile pixel q at element seg_off + q; where the tile runs into the
@@ -278,6 +286,20 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         nbytes[i] = (unsigned)(hi - lo) * 2u;
         per_channel += nbytes[i];
       }
+      // 8-byte variant: the pieces of a channel's segment this lane copies (pieces lane, lane + 32, ...): byte offset
+      // in the segment and element offset in the input relative to channel 0 of image 0; -1: none
+      constexpr int kPiecesPerLane = 8;
+      int piece_dst[kPiecesPerLane], piece_src[kPiecesPerLane];
+      if (CONV == 3) {
+#pragma unroll
+        for (int t = 0; t < kPiecesPerLane; ++t) {
+          int rem = lane + 32 * t, i = 0;
+          while (i + 1 < nimg && rem >= (int)(nbytes[i] >> 3)) { rem -= (int)(nbytes[i] >> 3); ++i; }
+          const bool ok = rem < (int)(nbytes[i] >> 3);
+          piece_dst[t] = ok ? dst_idx[i] * 2 + rem * 8 : -1;
+          piece_src[t] = ok ? (n0 + i) * a.C * ohw + src_lo[i] + rem * 4 : 0;
+        }
+      }
       // the planes have a ring of their own, freed by the builders (long before the tensor core is done with
       // the tile built from them), so their copies run several K tiles ahead
       for (int kt = 0; kt < nkt; ++kt) {
@@ -287,6 +309,19 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         const int c_lo = (kbase + kt) * kTK / 9;
         const int k_hi = (kbase + kt + 1) * kTK < p.K ? (kbase + kt + 1) * kTK - 1 : p.K - 1;
         const int nch = k_hi / 9 - c_lo + 1;
+        if (CONV == 3) {
+          // 8-byte pieces: a lane copies the same pieces of every channel (worked out once, above); its arrival is
+          // deferred until its copies have landed
+          for (int ci = 0; ci < nch; ++ci) {
+            uint8_t* dch = seg + (size_t)ci * p.seg_len * 2;
+            const __nv_bfloat16* sch = in + (int64_t)(c_lo + ci) * ohw;
+#pragma unroll
+            for (int t = 0; t < kPiecesPerLane; ++t)
+              if (piece_dst[t] >= 0) cp_async8(dch + piece_dst[t], sch + piece_src[t]);
+          }
+          cp_async_arrive_noinc(full + ss);
+          continue;
+        }
         if (lane == 0) mbar_arrive_expect_tx(full + ss, per_channel * (unsigned)nch);
         __syncwarp();  // the byte count is announced before any copy can complete
         // one copy per lane: a single thread needs several hundred cycles per copy it issues
@@ -365,13 +400,13 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
     for (int kt = bgrp; kt < nkt; kt += kTcBuildGroups) {
       const int slot = kt % ns;
-      const int ss = CONV == 2 ? kt % p.nseg : 0;
+      const int ss = CONV >= 2 ? kt % p.nseg : 0;
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 3; break; }
       // staged variant: the planes of this K tile have landed (their copies were requested several tiles ago)
-      if (CONV == 2 && !__all_sync(0xffffffffu, mbar_wait(full + ss, (unsigned)((kt / p.nseg) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 7; break; }
+      if (CONV >= 2 && !__all_sync(0xffffffffu, mbar_wait(full + ss, (unsigned)((kt / p.nseg) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 7; break; }
       uint8_t* bt_base = stages + (size_t)slot * stage_bytes + b_off + panel_off;
       const uint4* seg16 = reinterpret_cast<const uint4*>(segs + (size_t)ss * p.seg_bytes);
-      if (CONV == 2) {
+      if (CONV >= 2) {
         // Staged variant.  Row kk of the tile is k = (c, kh, kw); the warp takes rows w, w + 4, ... and keeps (c, tap)
         // up to date without dividing.  Everything that depends on the row only is the same in all lanes: the first
         // element of the row in the channel's segment (rb), hence the shift inside a vector; a lane adds its piece.
@@ -717,12 +752,13 @@ int tc_row_tiles(const grim_bcr* h, int64_t qtiles, size_t extra = 0) {
 }
 // Staged implicit im2col: elements kept in front of the tile's first pixel in a channel segment (a row and a pixel,
 // rounded to vectors, plus one vector), the segment's length, and the bytes of one slot of the ring of planes (eight
-// channels at most touch a K tile of 64).  Needs planes that start and end on 16-byte boundaries and tiles that meet at most
-// three images.
+// channels at most touch a K tile of 64).  Needs planes whose size is a multiple of 4 pixels (8-byte copies; multiples of 8
+// take 16-byte-aligned bulk copies) and tiles that meet at most three images.
 constexpr int kTcSegSlots = 4;  // slots of the ring of staged planes (its barriers share the tile ring's arrays)
 bool conv_staging(const SpmmArgs& a, int* seg_off, int* seg_len, size_t* seg_bytes) {
   const int64_t ohw = (int64_t)a.OH * a.OW;
-  if (!a.conv || ohw % 8 != 0 || ohw < kTQ / 2) return false;
+  if (!a.conv || ohw % 4 != 0 || ohw < kTQ / 2) return false;  // multiples of 8: bulk copies, of 4: 8-byte copies
+  if (ohw % 8 != 0 && (kTQ + 2 * ((a.W + 1 + 7) / 8 * 8 + 8)) * 2 / 8 > 8 * 32) return false;  // 8 pieces per lane at most
   *seg_off = (a.W + 1 + 7) / 8 * 8 + 8;
   *seg_len = kTQ + 2 * *seg_off;
   *seg_bytes = ((size_t)8 * *seg_len * 2 + 16 + 127) / 128 * 128;
@@ -822,7 +858,9 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
   if (a.conv) {
-    auto kern = staged ? (h->bh == 4 ? bcr_tc_kernel<4, 2> : (h->bh == 8 ? bcr_tc_kernel<8, 2> : bcr_tc_kernel<16, 2>))
+    const bool bulk = ((int64_t)a.OH * a.OW) % 8 == 0;
+    auto kern = staged ? (bulk ? (h->bh == 4 ? bcr_tc_kernel<4, 2> : (h->bh == 8 ? bcr_tc_kernel<8, 2> : bcr_tc_kernel<16, 2>))
+                               : (h->bh == 4 ? bcr_tc_kernel<4, 3> : (h->bh == 8 ? bcr_tc_kernel<8, 3> : bcr_tc_kernel<16, 3>)))
                        : (h->bh == 4 ? bcr_tc_kernel<4, 1> : (h->bh == 8 ? bcr_tc_kernel<8, 1> : bcr_tc_kernel<16, 1>));
     const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec, extra);
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;

@@ -408,12 +408,12 @@ def test_conv_bf16_batch_crossing_images(B):
     check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
 
 
-@pytest.mark.parametrize("shape", [(12, 12, 7), (8, 16, 9), (16, 10, 5), (24, 16, 3)])
+@pytest.mark.parametrize("shape", [(12, 12, 7), (8, 16, 9), (16, 10, 5), (24, 16, 3), (10, 14, 5), (14, 14, 3)])
 @pytest.mark.parametrize("bh", [4, 8, 16])
 def test_conv_bf16_staged_planes(B, shape, bh):
-    """Tensor-core convolution on planes whose size is a multiple of 8 pixels (the variant that stages the input
-    planes in shared memory): 256-pixel tiles that meet two or three images, a ragged last tile, several K tiles,
-    all block heights."""
+    """Tensor-core convolution on planes whose size is a multiple of 8 pixels, or of 4 (the variants that stage the
+    input planes in shared memory by bulk copies / by 8-byte copies): 256-pixel tiles that meet two or three images, a
+    ragged last tile, several K tiles, all block heights."""
     H, Wd, batch = shape
     C, Cout, bw = 20, 136, 32
     rng_seed = 300 + H + Wd + bh
