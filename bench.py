@@ -37,7 +37,7 @@ TRAFFIC = {
     "gru_2x1024_in153_T200_bcr8x32_c10_fp32": 6 * 3.519e6,  # six launches (2 layers x 3 chunks) of 3.5 MB each
     "spmm_M4096_K4096_N1024_c8_8x32_uniform_fp32": 27.68e6,
     "spmm_M8192_K8192_N1_c4_8x32_uniform_fp32": 85.27e6,
-    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.40e6,
+    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.60e6,
 }
 UNIT = "GFLOP/s"
 
