@@ -198,7 +198,7 @@ class SpmmWorkload:
         self.kernel_bytes = float(i.value_bytes + idx + i.k_used * self.N * esz + self.M * self.N * 4)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * 4
-        tc = self.bf16 and self.N >= 256 and self.bh in (4, 8, 16) and self.bw in (16, 32, 64)
+        tc = self.bf16 and self.N >= 128 and self.bh in (4, 8, 16) and self.bw in (16, 32, 64)
         self.kernel = "bcr_stream_kernel" if self.N <= 16 else ("bcr_tc_kernel" if tc else "bcr_ffma_kernel")
         self.peak_kind = "tensor" if tc else "alu"
         if tc:
@@ -643,7 +643,7 @@ def run_sweep(args):
                 if bf16:
                     X = X.to(torch.bfloat16)
                 Y = torch.empty(M, N, device="cuda")
-                tc = bf16 and N >= 256
+                tc = bf16 and N >= 128
                 idx = info.index_bytes_gemv if N <= 16 else (info.index_bytes_tc if tc else info.index_bytes_spmm)
                 nbytes = float(info.value_bytes + idx + info.k_used * N * esz + M * N * 4)
                 flops = 2.0 * nnz * N

@@ -48,7 +48,7 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
     return launch_skinny(h, X->ptr, X->dtype, X->ld, X->cols, Y->ptr, Y->dtype, Y->ld, s);
   }
   if (path == 4) return launch_spmm(h, a, s);
-  if (path == 0 && tc_path_supported(h, a) && a.ncols >= 256) return launch_spmm_tc(h, a, s);
+  if (path == 0 && tc_path_supported(h, a) && a.ncols >= 128) return launch_spmm_tc(h, a, s);
   if (ffma_path_supported(h, a)) return launch_ffma(h, a, s);
   if (path == 1) return GRIM_ERR_UNSUPPORTED;
   return launch_spmm(h, a, s);

@@ -256,10 +256,13 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
         const int slot = kt % ns;
         if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true, fail_site = 1; break; }
         uint8_t* st = stages + (size_t)slot * stage_bytes;
-        mbar_arrive_expect_tx(full + slot, (unsigned)kBTileBytes);
+        // 64-column boxes that lie wholly past the last column are not requested (their part of the tile keeps
+        // whatever it held; the accumulator columns computed from it are never stored)
+        const int nbox = (int)((a.ncols - q0 + 63) / 64) < kTQ / 64 ? (int)((a.ncols - q0 + 63) / 64) : kTQ / 64;
+        mbar_arrive_expect_tx(full + slot, (unsigned)(nbox * 64 * kTK * 2));
 #pragma unroll
         for (int i = 0; i < kTQ / 64; ++i)
-          tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, (kbase + kt) * kTK, full + slot);
+          if (i < nbox) tma_load_2d(st + b_off + i * (64 * kTK * 2), &tmX, (int)q0 + 64 * i, (kbase + kt) * kTK, full + slot);
       }
     }
     if (CONV >= 2) {
