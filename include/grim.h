@@ -207,7 +207,7 @@ grim_status_t grim_maxpool2x2(const void* in_dev, void* out_dev, int64_t N, int6
  *   h_t = (1 - z) * n + z * h_{t-1};   layer l > 0 takes layer l-1's h_t as its x_t.
  *
  * grim_gru_create: W_ih[l] is 3H x in_l, W_hh[l] is 3H x H (fp32 handles packed with the same
- * bh, H a multiple of bh); b_ih_host[l], b_hh_host[l]: 3H fp32 HOST values (copied).  The packed
+ * bh, H a multiple of bh and of 4, else GRIM_ERR_UNSUPPORTED); b_ih_host[l], b_hh_host[l]: 3H fp32 HOST values (copied).  The packed
  * matrices are borrowed: they must outlive the GRU handle.  max_T bounds the sequence length;
  * scratch for the hoisted input projections is allocated here.
  *
@@ -228,7 +228,7 @@ grim_status_t grim_gru_destroy(grim_gru_t g);
 /* Layer pipelining of grim_gru_seq (execution detail, Section 4.2's concern with keeping all units busy; the paper
  * has no multi-layer schedule).  With more than one layer the sequence is cut into `chunks` pieces in time and layer
  * l works on piece k while layer l - 1 works on piece k + 1, each layer on an internal stream ordered by events; the
- * caller's stream continues after the last layer.  chunks = 0 lets the library choose, 1 runs the layers one after the
+ * caller's stream continues after the last layer.  Stacks of more than three layers are not pipelined.  chunks = 0 lets the library choose, 1 runs the layers one after the
  * other on the caller's stream, at most 8.  Results do not depend on it. */
 grim_status_t grim_gru_set_pipeline(grim_gru_t g, int chunks);
 
@@ -249,7 +249,8 @@ grim_status_t grim_gru_set_pipeline(grim_gru_t g, int chunks);
  *     8 MiB - e.g. H = 1024, two layers: T <= 409.  Larger requests return GRIM_ERR_UNSUPPORTED
  *     before anything is launched; use grim_gru_seq for those.
  *   - The first call on a device looks up the array's device address (once per device, with that
- *     device current).  Make that first call during start-up, before any CUDA stream capture.
+ *     device current).  Make that first call during start-up, before any CUDA stream capture.  The
+ *     address is cached for the life of the process: it does not survive a cudaDeviceReset.
  *   - All calls in the process share the array and it keeps whatever the previous call left there.
  *     Nothing in it has to start at zero: every word the kernels read from it is written earlier in
  *     the same call.  Two calls that overlap on the GPU (different streams or handles) race on it;

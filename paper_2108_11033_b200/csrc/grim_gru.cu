@@ -44,6 +44,7 @@ struct grim_gru {
   std::vector<uint32_t*> d_pos_of_band;
   std::vector<float*> d_img_val;      // per layer: register image of the register-resident kernel (may be empty)
   std::vector<uint32_t*> d_img_col;
+  std::vector<float*> d_gi_saved;  // grim_gru_seq_static parks d_gi here while it points the pass at the static array
   std::vector<float*> d_gi;  // per layer: hoisted pre-activations, T x 3H (layers overlap in time, so each has its own)
   float* d_seq[2] = {nullptr, nullptr};
   // unit-major copies (feature x time, row stride = T rounded up to 4): the projections then read X row-major
@@ -687,6 +688,7 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
     if (l > 0 && wi->K != H) return GRIM_ERR_SHAPE;
     if (wi->dtype != GRIM_F32 || wh->dtype != GRIM_F32) return GRIM_ERR_DTYPE;
     if (wh->bh != bh || H % bh != 0 || !wh->gemv_ok) return GRIM_ERR_UNSUPPORTED;
+    if (H % 4 != 0) return GRIM_ERR_UNSUPPORTED;  // rows of 3H floats are filled and read as 16-byte vectors
   }
   grim_gru* g = new (std::nothrow) grim_gru();
   if (!g) return GRIM_ERR_ALLOC;
@@ -722,6 +724,7 @@ extern "C" grim_status_t grim_gru_create(int layers, const grim_bcr_t* W_ih, con
         e = cudaMalloc((void**)&p, (size_t)max_T * 3 * H * 4);
         if (e == cudaSuccess) g->d_gi.push_back(p);
       }
+      g->d_gi_saved.resize(g->d_gi.size());  // sized here so that grim_gru_seq_static never touches the heap
       for (int l = 1; l < layers && e == cudaSuccess; ++l) {
         cudaStream_t st = nullptr;
         e = cudaStreamCreateWithFlags(&st, cudaStreamNonBlocking);
@@ -884,7 +887,9 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
   // stream, ordered by events), so a stack of L layers takes about (1 + (L - 1) / chunks) single-layer times instead
   // of L.  The kernels with a global barrier (fall-back) and single-layer models run as one chunk on one stream.
   int chunks = 1;
-  if (g->pipeline && L > 1 && (use_reg || use_cluster))
+  // With four or more layers, layers l and l + 2 share an inter-layer buffer, and layer l reads its chunk-entering
+  // state from that buffer while layer l + 2 may already be writing it: such stacks run one layer after the other.
+  if (g->pipeline && L > 1 && L <= 3 && (use_reg || use_cluster))
     chunks = g->want_chunks > 0 ? (int)std::min<int64_t>(g->want_chunks, T)
                                 : (int)std::max<int64_t>(1, std::min<int64_t>(3, T / 64));
   const int64_t clen = ((T + chunks - 1) / chunks + 3) / 4 * 4;  // a multiple of 4: chunk starts stay 16-byte aligned
@@ -1113,7 +1118,7 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
   // Run the ordinary pass with the handle's scratch pointers pointing into the static array for the duration of
   // the call (kernel arguments are copied at launch, so the handle can be put back at once).  All layers share one
   // pre-activation buffer here, so the layers run one after the other on the caller's stream.
-  const std::vector<float*> saved_gi = g->d_gi;
+  std::copy(g->d_gi.begin(), g->d_gi.end(), g->d_gi_saved.begin());  // same size since creation: no allocation
   float* const saved_seq0 = g->d_seq[0];
   float* const saved_seq1 = g->d_seq[1];
   const bool saved_pipeline = g->pipeline, saved_tin = g->transposed_inputs;
@@ -1123,7 +1128,7 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
   g->d_seq[1] = reinterpret_cast<float*>(base + gi_bytes + seq_bytes);
   g->pipeline = false;
   const grim_status_t st = grim_gru_seq(g, x, T, h0, y, hT, stream);
-  g->d_gi = saved_gi;
+  std::copy(g->d_gi_saved.begin(), g->d_gi_saved.end(), g->d_gi.begin());
   g->d_seq[0] = saved_seq0;
   g->d_seq[1] = saved_seq1;
   g->pipeline = saved_pipeline;

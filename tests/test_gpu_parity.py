@@ -10,12 +10,10 @@ import pytest
 import torch
 
 from oracle import bcr_oracle as orc
+from parity_util import F32_TOL, assert_close, rel_fro
 from workloads import generators as gen
 
 pytestmark = pytest.mark.gpu
-
-F32_TOL = 1e-5
-BF16_TOL = 2e-2
 
 
 @pytest.fixture(scope="module")
@@ -24,11 +22,6 @@ def B():
     build_library()
     from paper_2108_11033_b200 import binding
     return binding
-
-
-def rel_fro(got, want):
-    want = np.asarray(want, dtype=np.float64)
-    return float(np.linalg.norm(np.asarray(got, dtype=np.float64) - want) / max(np.linalg.norm(want), 1e-300))
 
 
 def to_dev(a, bf16=False):
@@ -55,15 +48,9 @@ def check_spmm(B, W, mask, X, bh, bw, *, bf16=False, flags=0, tile_n=0, y_bf16=F
         want = orc.spmm(W, mask, X, dt)
         dead = np.flatnonzero(mask.sum(axis=1) == 0)
         assert np.all(got[dead] == 0.0) and not np.any(np.signbit(got[dead])), "pruned rows must be exactly +0"
-        if bf16:
-            Wm = orc.masked_weight(W, mask, dt)
-            bound = BF16_TOL * np.linalg.norm(Wm, axis=1)[:, None] * np.linalg.norm(X.astype(np.float64), axis=0)[None, :]
-            err = np.abs(got - want)
-            assert np.all(err <= bound + 1e-30), f"max excess {np.max(err - bound)}"
-            if not y_bf16:
-                assert rel_fro(got, want) < 1e-4  # fp32 accumulation of exact bf16 products
-        else:
-            assert rel_fro(got, want) <= F32_TOL, rel_fro(got, want)
+        Wm = orc.masked_weight(W, mask, dt)
+        scale = np.linalg.norm(Wm, axis=1)[:, None] * np.linalg.norm(X.astype(np.float64), axis=0)[None, :]
+        assert_close(got, want, scale, bf16_in=bf16, out_bf16=y_bf16, what=f"spmm {M}x{K}x{N}")
     finally:
         B.grim_bcr_destroy(h)
 
@@ -306,15 +293,10 @@ def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=F
         torch.cuda.synchronize()
         got = out.float().cpu().numpy().astype(np.float64)
         want = orc.conv2d(W, mask, x, bias, ksize=ksize, stride=stride, pad=pad, relu=relu, dtype=dt)
-        if bf16:
-            Wm = orc.masked_weight(W, mask, dt)
-            bound = BF16_TOL * (np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x, ksize, stride, pad)
-                                + np.abs(bias.astype(np.float64))[None, :, None, None])
-            assert np.all(np.abs(got - want) <= bound + 1e-30)
-            if not out_bf16:
-                assert rel_fro(got, want) < 1e-4
-        else:
-            assert rel_fro(got, want) <= F32_TOL, rel_fro(got, want)
+        Wm = orc.masked_weight(W, mask, dt)
+        scale = np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x, ksize, stride, pad)
+        assert_close(got, want, scale, bf16_in=bf16, out_bf16=out_bf16,
+                     bias_abs=np.abs(bias.astype(np.float64))[None, :, None, None], what="conv")
     finally:
         B.grim_bcr_destroy(h)
 
@@ -377,9 +359,9 @@ def test_vgg_stack_small_image_per_layer(B):
         x_np = cur.float().cpu().numpy()
         want = orc.conv2d(L["W"], L["mask"], x_np, L["bias"], ksize=3, stride=1, pad=1, relu=True, dtype=orc.DTYPE_BF16)
         Wm = orc.masked_weight(L["W"], L["mask"], orc.DTYPE_BF16)
-        bound = BF16_TOL * (np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x_np, 3, 1, 1)
-                            + np.abs(L["bias"].astype(np.float64))[None, :, None, None])
-        assert np.all(np.abs(out.float().cpu().numpy() - want) <= bound + 1e-30)
+        scale = np.linalg.norm(Wm, axis=1)[None, :, None, None] * conv_col_norms(x_np, 3, 1, 1)
+        assert_close(out.float().cpu().numpy(), want, scale, bf16_in=True, out_bf16=True,
+                     bias_abs=np.abs(L["bias"].astype(np.float64))[None, :, None, None], what=f"vgg layer {L['cout']}")
         B.grim_bcr_destroy(h)
         if L["pool"]:
             pooled = torch.empty(Nb, L["cout"], H // 2, Wd // 2, device="cuda", dtype=torch.bfloat16)
@@ -487,6 +469,16 @@ def test_gru_small(B, cfg):
     h0 = gen.normal_f32((L, H), 0.5, 81, 0)
     check_gru(B, m, h0=h0)
     check_gru(B, m, h0=h0, grid_kernel=True)
+
+
+def test_gru_four_layers_and_odd_hidden_size(B):
+    """Four layers (run one after the other: the wavefront schedule is kept to three) against the oracle, and a
+    hidden size that is a multiple of the block height but not of 4 is refused at creation."""
+    check_gru(B, gen.gru_model(24, 128, 4, 70, bh=8, bw=32, compression=4, seed=97))
+    m = gen.gru_model(12, 30, 1, 3, bh=6, bw=16, compression=2, seed=98)
+    with pytest.raises(B.GrimError) as e:
+        build_gru(B, m, 3)
+    assert e.value.status == B.GRIM_ERR_UNSUPPORTED
 
 
 @pytest.mark.parametrize("grid_kernel", [False, True])

@@ -207,6 +207,36 @@ def test_pack_unpack_round_trip(shape, dtype):
     assert np.array_equal(orc.masked_weight(W, mask, dtype), u["W"].astype(np.float64))
 
 
+def _golden_canonical():
+    out = {}
+    for line in open(os.path.join(GOLDEN, "canonical_4x4_blocks2x2.txt")):
+        line = line.strip()
+        if line and not line.startswith("#"):
+            name, hexs = line.split(":")
+            out[name.strip()] = bytes.fromhex(hexs.replace(" ", ""))
+    return out
+
+
+def _golden_matrix():
+    W = np.array([[1, 2, 3, 4], [5, 0, 0, 8], [-1, -2, 0.5, 0.25], [-3, -4, 1.5, -0.5]], dtype=np.float32)
+    W.view(np.uint32)[1, 1] = 0x40C08000
+    W.view(np.uint32)[1, 2] = 0x40E18000
+    mask = np.array([[0, 1, 0, 0], [0, 1, 1, 1], [0, 0, 1, 1], [0, 0, 1, 1]], dtype=np.uint8)
+    return W, mask
+
+
+def test_pack_canonical_matches_hand_written_bytes():
+    """The byte layout itself (field order, widths, value order, trailer) against a byte string typed out by hand
+    from the layout in the public header - not produced by any packer."""
+    g = _golden_canonical()
+    W, mask = _golden_matrix()
+    assert orc.pack_canonical(W, mask, 2, 2, orc.DTYPE_F32, reorder=True) == g["f32_reorder"]
+    assert orc.pack_canonical(W, mask, 2, 2, orc.DTYPE_BF16, reorder=False) == g["bf16_plain"]
+    u = orc.unpack_canonical(g["f32_reorder"])
+    assert np.array_equal(u["mask"], mask) and list(u["row_perm"]) == [1, 2, 3, 0]
+    assert np.array_equal(u["W"].view(np.uint32), np.where(mask != 0, W, np.float32(0)).view(np.uint32))
+
+
 def test_pack_lists_sorted_and_nnz_accounting():
     M, K, bh, bw = 48, 96, 8, 32
     mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=23)

@@ -11,6 +11,7 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import bcr_oracle as orc
 from workloads import generators as gen
 
 pytestmark = pytest.mark.gpu
@@ -57,6 +58,10 @@ def test_static_scratch_gru_matches_allocating_entry_point(B):
             assert torch.cuda.memory_stats().get("allocation.all.allocated", 0) == allocs_before
             assert torch.cuda.mem_get_info()[0] >= free_before
             assert _rel(y, y_ref) <= 1e-5 and _rel(hT, hT_ref) <= 1e-5
+            # and against the CPU oracle: this entry point takes its own route through the library (one shared
+            # pre-activation buffer, layers one after the other), so agreeing with the other entry point is not enough
+            want_y, want_h = orc.gru_seq(m["layers"], x.cpu().numpy(), h0=None if h is None else h.cpu().numpy())
+            assert _rel(y, torch.from_numpy(want_y)) <= 1e-5 and _rel(hT, torch.from_numpy(want_h)) <= 1e-5
         # a request that does not fit the 8 MiB array is refused on the host, before any launch
         big_T = 5000
         xb = torch.zeros(big_T, 40, device="cuda")
