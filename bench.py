@@ -31,15 +31,89 @@ if ROOT not in sys.path:
 
 METRIC = "BCR SpMM/GEMV effective GFLOP/s (2*nnz*N)"
 
-# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum, bytes) of the dominant kernel per step, from one ncu
-# capture of the same command (summaries under profiles/); None where the kernel has changed since or was not captured.
-TRAFFIC = {
-    "gru_2x1024_in153_T200_bcr8x32_c10_fp32": 6 * 3.519e6,  # six launches (2 layers x 3 chunks) of 3.5 MB each
-    "spmm_M4096_K4096_N1024_c8_8x32_uniform_fp32": 27.68e6,
-    "spmm_M8192_K8192_N1_c4_8x32_uniform_fp32": 85.27e6,
-    "spmm_M8192_K8192_N1024_c8_8x32_uniform_bf16": 47.60e6,
-}
 UNIT = "GFLOP/s"
+CSRC = os.path.join(ROOT, "paper_2108_11033_b200", "csrc")
+
+
+def profile_traffic(workload_name):
+    """DRAM traffic per launch of the dominant kernel (dram__bytes_read.sum + dram__bytes_write.sum of one ncu
+    capture), read from the summary under profiles/ whose `workload:` line names this workload.  A summary records
+    the SHA-1 of the kernel's source file at capture time (`source_sha1: <file> <hash>`); when the file has changed
+    since, the counters no longer describe the kernel and None is returned."""
+    import hashlib
+    pdir = os.path.join(ROOT, "profiles")
+    if not os.path.isdir(pdir):
+        return None
+    for fn in sorted(os.listdir(pdir)):
+        try:
+            fields = {}
+            for line in open(os.path.join(pdir, fn)):
+                if ":" in line and line.split(":", 1)[0].strip() in ("workload", "traffic_bytes_per_launch", "source_sha1"):
+                    k, v = line.split(":", 1)
+                    fields[k.strip()] = v.strip()
+            if fields.get("workload") != workload_name or "traffic_bytes_per_launch" not in fields:
+                continue
+            src, sha = fields.get("source_sha1", " ").split()
+            with open(os.path.join(CSRC, src), "rb") as f:
+                if hashlib.sha1(f.read()).hexdigest() != sha:
+                    return None
+            return float(fields["traffic_bytes_per_launch"])
+        except Exception:
+            continue
+    return None
+
+
+_SWEEP_CACHE = {}
+
+
+def sweep_inputs(M, N, c, bh, bw, dist, bf16):
+    """Same inputs as workloads.generators.sweep_case (seed 5); the weight and the mask of a (size, compression, block,
+    distribution) are generated once and shared by the records that use them."""
+    from workloads import generators as gen
+    key = (M, c, bh, bw, dist)
+    if key not in _SWEEP_CACHE:
+        if len(_SWEEP_CACHE) >= 2:
+            _SWEEP_CACHE.pop(next(iter(_SWEEP_CACHE)))
+        _SWEEP_CACHE[key] = (gen.dense_weight(M, M, 5, 31), gen.bcr_mask(M, M, bh, bw, compression=c, dist=dist, seed=5, stream=32))
+    W, mask = _SWEEP_CACHE[key]
+    X = gen.normal_f32((M, N), 1.0, 5, 33)
+    if bf16:
+        X = gen.bf16_representable(X)
+    return dict(W=W, mask=mask, X=X, bh=bh, bw=bw)
+
+
+def parity_rows(W, mask, X, got_rows, pick, bf16, out_bf16=False):
+    """Sampled output rows against the CPU oracle (outside every timed region), element by element."""
+    from oracle import bcr_oracle as orc
+    from workloads.tolerances import assert_close
+    dt = orc.DTYPE_BF16 if bf16 else orc.DTYPE_F32
+    want = orc.spmm(W[pick], mask[pick], X, dt)
+    Wm = orc.masked_weight(W[pick], mask[pick], dt)
+    scale = np.linalg.norm(Wm, axis=1)[:, None] * np.linalg.norm(X.astype(np.float64), axis=0)[None, :]
+    assert_close(got_rows, want, scale, bf16_in=bf16, out_bf16=out_bf16, what="sampled rows")
+
+
+def parity_conv(L, x_np, got, bf16, out_bf16, rows):
+    """Output channels `rows` of a 3x3 / stride 1 / pad 1 convolution with bias and ReLU against the CPU oracle;
+    x_np: the images (NCHW, the values the GPU read), got: the GPU's output [images, len(rows), H, W]."""
+    import torch
+    from oracle import bcr_oracle as orc
+    from workloads.tolerances import assert_close
+    dt = orc.DTYPE_BF16 if bf16 else orc.DTYPE_F32
+    W, mask, bias = L["W"][rows], L["mask"][rows], L["bias"][rows]
+    want = orc.conv2d(W, mask, x_np, bias, ksize=3, stride=1, pad=1, relu=True, dtype=dt)
+    Wm = orc.masked_weight(W, mask, dt)
+    xx = torch.from_numpy(np.asarray(x_np, np.float64) ** 2)
+    ones = torch.ones(1, xx.shape[1], 3, 3, dtype=torch.float64)
+    col = torch.sqrt(torch.nn.functional.conv2d(xx, ones, padding=1)).numpy()  # norm of each im2col column
+    scale = np.linalg.norm(Wm, axis=1)[None, :, None, None] * col
+    assert_close(got, want, scale, bf16_in=bf16, out_bf16=out_bf16, bias_abs=np.abs(bias.astype(np.float64))[None, :, None, None],
+                 what="sampled channels")
+
+
+def min_index_bytes(info):
+    """The smallest index a BCR matrix needs: one row bitmask and one column bitmask per non-empty block."""
+    return info.nonempty_blocks * (info.bh + info.bw) / 8.0
 
 
 L2_BYTES = 126e6
@@ -133,17 +207,22 @@ class GruWorkload:
         self.x = self.x_host.cuda()
         self.y = torch.empty(self.T, self.H, device="cuda")
         B.grim_gru_profile(self.g, True)
-        # algorithmic bytes of the recurrent kernel (dominant): per step the kept values and their index
-        # words of W_hh, the three pre-activation rows, h read and h written; summed over the layers
-        self.kernel_bytes = 0.0
-        for hh in self.hh:
-            i = B.grim_bcr_info(hh)
-            self.kernel_bytes += self.T * (i.value_bytes + i.index_bytes_gemv + 3 * self.H * 4 + 2 * self.H * 4)
+        # Bytes the pass has to move once: every layer's packed W_ih and W_hh (values + index words), the input, the
+        # hoisted pre-activations written and read back, the inter-layer and output sequences.  (W_hh stays on chip
+        # for the whole sequence, so it is NOT counted once per time step; the figure that does count it per step is
+        # reported beside this one as notional.)
+        self.kernel_bytes, self.min_bytes, self.notional_bytes = 0.0, 0.0, 0.0
+        for hi, hh in zip(self.hi, self.hh):
+            ii, ih = B.grim_bcr_info(hi), B.grim_bcr_info(hh)
+            acts = ii.K * self.T * 4 + 2 * self.T * 3 * self.H * 4 + self.T * self.H * 4
+            self.kernel_bytes += ii.value_bytes + ii.index_bytes_spmm + ih.value_bytes + ih.index_bytes_gemv + acts
+            self.min_bytes += ii.value_bytes + min_index_bytes(ii) + ih.value_bytes + min_index_bytes(ih) + acts
+            self.notional_bytes += self.T * (ih.value_bytes + ih.index_bytes_gemv + 3 * self.H * 4 + 2 * self.H * 4)
         self.h2d = self.x_host.numel() * 4
         self.d2h = self.y_host.numel() * 4
         self.kernel = "gru_cluster_reg_kernel"
         self.peak_kind = "alu"
-        self.force_bound = "hbm"  # a chain of dependent steps: reported against the streamed-bytes figure
+        self.force_bound = "hbm"  # far from any throughput roof: a chain of T dependent steps (latency-bound)
 
     def step(self):
         self.B.grim_gru_seq(self.g, self.x, self.y)
@@ -157,7 +236,19 @@ class GruWorkload:
         return self.B.grim_gru_profile_read(self.g)[1]
 
     def check(self):
-        assert self.B.grim_gru_status(self.g) == self.B.GRIM_OK
+        """Status word, then the whole output sequence of the last pass against the oracle."""
+        from oracle import bcr_oracle as orc
+        from workloads.tolerances import F32_TOL, rel_fro
+        self.torch.cuda.synchronize()
+        assert self.B.grim_gru_status(self.g) == self.B.GRIM_OK, "a bounded device wait gave up"
+        want, _ = orc.gru_seq(self.m["layers"], self.m["x"])
+        got = self.y.cpu().numpy()
+        assert np.all(np.isfinite(got)) and rel_fro(got, want) <= F32_TOL, rel_fro(got, want)
+
+    def close(self):
+        self.B.grim_gru_destroy(self.g)
+        for h in self.hi + self.hh:
+            self.B.grim_bcr_destroy(h)
 
     def oracle_sample(self):
         from oracle import bcr_oracle as orc
@@ -171,16 +262,15 @@ class GruWorkload:
 class SpmmWorkload:
     """One point of the SpMM sweep (square W).  N = 1 runs the matrix-vector kernel."""
 
-    def __init__(self, M=8192, N=1, c=8.0, bh=8, bw=32, dist="uniform", bf16=False, conv=False):
-        from workloads import generators as gen
+    def __init__(self, M=8192, N=1, c=8.0, bh=8, bw=32, dist="uniform", bf16=False, inputs=None, name=None):
         self.M, self.N, self.bf16 = M, N, bf16
-        self.s = gen.sweep_case(M, N, c, bh, bw, dist, bf16=bf16)
+        self.s = inputs if inputs is not None else sweep_inputs(M, N, c, bh, bw, dist, bf16)
         self.bh, self.bw = bh, bw
-        self.name = f"spmm_M{M}_K{M}_N{N}_c{c:g}_{bh}x{bw}_{dist}_{'bf16' if bf16 else 'fp32'}"
+        self.name = name or f"spmm_M{M}_K{M}_N{N}_c{c:g}_{bh}x{bw}_{dist}_{'bf16' if bf16 else 'fp32'}"
         self.dtype = "bf16" if bf16 else "f32"
         self.nnz = int(self.s["mask"].sum())
         self.flops = 2.0 * self.nnz * N
-        self.copies = 1
+        self.dense_elems = int(self.s["mask"].size)
 
     def setup(self, B, torch):
         self.B, self.torch = B, torch
@@ -196,6 +286,7 @@ class SpmmWorkload:
         esz = 2 if self.bf16 else 4
         idx = i.index_bytes_gemv if self.N <= 16 else i.index_bytes_spmm
         self.kernel_bytes = float(i.value_bytes + idx + i.k_used * self.N * esz + self.M * self.N * 4)
+        self.min_bytes = float(i.value_bytes + min_index_bytes(i) + i.k_used * self.N * esz + self.M * self.N * 4)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * 4
         tc = self.bf16 and self.N >= 128 and self.bh in (4, 8, 16) and self.bw in (16, 32, 64)
@@ -232,15 +323,33 @@ class SpmmWorkload:
         return self._ev[0].elapsed_time(self._ev[1])
 
     def check(self):
-        pass
+        """Status words of every handle used, then sampled output rows of the last launch against the oracle."""
+        torch = self.torch
+        torch.cuda.synchronize()
+        for h, _, _ in self.sets:
+            assert self.B.grim_bcr_status(h) == self.B.GRIM_OK, "a bounded device wait gave up"
+        _, x, y = self.sets[(self._i - 1) % len(self.sets)] if self._i else self.sets[0]
+        pick = np.sort(np.random.default_rng(1).choice(self.M, size=min(64, self.M), replace=False))
+        got = y.cpu().numpy()
+        assert np.all(np.isfinite(got))
+        parity_rows(self.s["W"], self.s["mask"], self.s["X"], got[pick], pick, self.bf16)
 
-    def oracle_sample(self):
+    def close(self):
+        for h, _, _ in self.sets:
+            self.B.grim_bcr_destroy(h)
+        self.sets = []
+
+    def oracle_sample(self, rows=None, cols=256):
+        """Times the oracle on the first `rows` rows of W (all by default) and the first `cols` columns of X."""
         from oracle import bcr_oracle as orc
-        n = min(self.N, 64)
+        n = min(self.N, cols)
+        r = self.M if rows is None else min(self.M, rows)
+        W, mask = self.s["W"][:r], self.s["mask"][:r]
         t0 = time.perf_counter()
-        orc.spmm(self.s["W"], self.s["mask"], self.s["X"][:, :n], 1 if self.bf16 else 0)
+        orc.spmm(W, mask, self.s["X"][:, :n], 1 if self.bf16 else 0)
         dt = time.perf_counter() - t0
-        return 2.0 * self.nnz * n / dt / 1e9, f"first {n} of {self.N} columns, masked dense fp64 NumPy matmul"
+        return 2.0 * float(mask.sum()) * n / dt / 1e9, \
+            f"first {r} of {self.M} rows of W, first {n} of {self.N} columns of X, masked dense fp64 NumPy matmul"
 
 
 class ConvWorkload:
@@ -252,6 +361,7 @@ class ConvWorkload:
         self.dtype = "bf16" if bf16 else "f32"
         self.nnz = int(self.L["mask"].sum())
         self.flops = 2.0 * self.nnz * batch * 28 * 28
+        self.dense_elems = int(self.L["mask"].size)
 
     def setup(self, B, torch):
         self.B, self.torch = B, torch
@@ -268,6 +378,7 @@ class ConvWorkload:
         esz = 2 if self.bf16 else 4
         idx = i.index_bytes_tc if self.bf16 else i.index_bytes_spmm
         self.kernel_bytes = float(i.value_bytes + idx + self.x.numel() * esz + self.y.numel() * esz)
+        self.min_bytes = float(i.value_bytes + min_index_bytes(i) + self.x.numel() * esz + self.y.numel() * esz)
         self.h2d = self.x_host.numel() * esz
         self.d2h = self.y_host.numel() * esz
         self.kernel = "bcr_tc_kernel (implicit im2col)" if self.bf16 else "bcr_ffma_kernel (implicit im2col)"
@@ -300,7 +411,21 @@ class ConvWorkload:
         return self._ev[0].elapsed_time(self._ev[1])
 
     def check(self):
-        pass
+        """Status words, then the first and the last image of the last launch on 64 sampled output channels."""
+        self.torch.cuda.synchronize()
+        for h, _, _ in self.sets:
+            assert self.B.grim_bcr_status(h) == self.B.GRIM_OK, "a bounded device wait gave up"
+        _, x, y = self.sets[(self._i - 1) % len(self.sets)] if self._i else self.sets[0]
+        assert bool(self.torch.isfinite(y.float()).all())
+        imgs = sorted({0, self.batch - 1})
+        rows = np.sort(np.random.default_rng(2).choice(512, size=64, replace=False))
+        got = y[imgs].float().cpu().numpy()[:, rows]
+        parity_conv(self.L, x[imgs].float().cpu().numpy(), got, self.bf16, self.bf16, rows)
+
+    def close(self):
+        for h, _, _ in self.sets:
+            self.B.grim_bcr_destroy(h)
+        self.sets = []
 
     def oracle_sample(self):
         from oracle import bcr_oracle as orc
@@ -323,6 +448,7 @@ class VggWorkload:
         self.nnz = sum(int(L["mask"].sum()) for L in self.net["layers"])
         self.flops = sum(2.0 * int(L["mask"].sum()) * batch * L["hw"] * L["hw"] for L in self.net["layers"])
         self.peak_kind = "tensor"
+        self.dense_elems = sum(int(L["mask"].size) for L in self.net["layers"])
         self.kernel = "bcr_tc_kernel (implicit im2col, per layer)"
 
     def setup(self, B, torch):
@@ -350,6 +476,8 @@ class VggWorkload:
             self.layer_bytes.append(float(i.value_bytes + i.index_bytes_tc + 2 * L["cin"] * npx + 2 * L["cout"] * npx))
             self.layer_flops.append(2.0 * i.nnz * npx)
         self.kernel_bytes = sum(self.layer_bytes)
+        self.min_bytes = sum(float(i.value_bytes + min_index_bytes(i)) + 2.0 * (L["cin"] + L["cout"]) * self.batch * L["hw"] ** 2
+                             for L, i in zip(net["layers"], self.info))
         self.h2d = self.x_host.numel() * 2
         self.d2h = self.y_host.numel() * 2
         self.layer_ms = [[] for _ in net["layers"]]
@@ -384,7 +512,24 @@ class VggWorkload:
         return sum(ms)
 
     def check(self):
-        pass
+        """Every layer of the last pass, on the last image and 32 sampled output channels, with the oracle fed the
+        values the GPU read as that layer's input."""
+        self.torch.cuda.synchronize()
+        for h in self.h:
+            assert self.B.grim_bcr_status(h) == self.B.GRIM_OK, "a bounded device wait gave up"
+        cur = self.x
+        img = [self.batch - 1]
+        for li, L in enumerate(self.net["layers"]):
+            out, pooled = self.bufs[li]
+            rows = np.sort(np.random.default_rng(3 + li).choice(L["cout"], size=min(32, L["cout"]), replace=False))
+            assert bool(self.torch.isfinite(out[img].float()).all()), f"layer {li + 1}"
+            parity_conv(L, cur[img].float().cpu().numpy(), out[img].float().cpu().numpy()[:, rows], True, True, rows)
+            cur = pooled if pooled is not None else out
+
+    def close(self):
+        for h in self.h:
+            self.B.grim_bcr_destroy(h)
+        self.h = []
 
     def extra(self, peaks):
         """Per-layer time and fraction of the binding roofline (HBM bytes vs the measured dense bf16 tensor rate)."""
@@ -414,6 +559,8 @@ class VggWorkload:
 
 def make_workload(args):
     w = args.workload
+    if w == "suite":  # the headline point of the sweep; the other configurations follow as records
+        return SpmmWorkload(M=8192, N=1024, c=8.0, bh=8, bw=32, dist="uniform", bf16=False)
     if w == "gru":
         return GruWorkload()
     if w == "gemv":
@@ -437,11 +584,23 @@ def run_reference(args):
     wl = make_workload(args)
     if isinstance(wl, GruWorkload):
         wl.sample_T = 50
+    kw = {}
+    if isinstance(wl, SpmmWorkload):
+        # size the per-step sample so that the whole run takes about two minutes: start small, time it once, grow the
+        # number of rows (then of columns) in proportion
+        budget = 120.0 / max(1, args.steps + args.warmup)
+        kw = dict(rows=min(wl.M, 256), cols=min(wl.N, 64))
+        t0 = time.perf_counter()
+        wl.oracle_sample(**kw)
+        scale = budget / max(time.perf_counter() - t0, 1e-3)
+        rows = int(min(wl.M, max(64, kw["rows"] * scale)))
+        cols = int(min(wl.N, max(kw["cols"], kw["cols"] * scale * kw["rows"] / rows)))
+        kw = dict(rows=rows, cols=cols)
     for _ in range(args.warmup):
-        wl.oracle_sample()
+        wl.oracle_sample(**kw)
     vals, t0 = [], time.perf_counter()
     for _ in range(args.steps):
-        v, what = wl.oracle_sample()
+        v, what = wl.oracle_sample(**kw)
         vals.append(v)
     total = time.perf_counter() - t0
     # harmonic mean over steps = total work / total time
@@ -487,61 +646,34 @@ def run_ours(args):
     build_library()
     from paper_2108_11033_b200 import binding as B
 
+    bench = Bench(B, torch)
+    suite = args.workload == "suite"
     wl = make_workload(args)
     wl.setup(B, torch)
-    # written before every timed iteration: evicts the working set from L2 (126 MB) and keeps the GPU busy
-    # long enough for the host to queue the step behind it, so that no host latency sits between the events
-    flush = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
-
-    def flush_l2():
-        # the write evicts the working set; the read of half the buffer behind it pushes the write's dirty lines out
-        # to HBM, so that the timed step does not pay for writing them back when its own reads evict them
-        flush.zero_()
-        flush[: 1 << 29].view(torch.int64).sum()
+    warmup = max(args.warmup, 3)
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    for _ in range(max(args.warmup, 3)):
+    for _ in range(warmup):
         wl.step()
-    wl.check()
     barrier()
 
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     B.grim_launch_count_reset()
-    kernel_ms = []
-    rotating = bool(getattr(wl, "rotating", False))
     barrier()
-    if rotating:
-        wl.per_step_events = False
-        # Inputs larger than L2: the steps rotate through operand sets, so every launch reads from HBM, and they are
-        # queued back to back behind a few flushes (which keep the GPU busy while the host queues all steps): the
-        # time between the two events is that of the launches alone, without per-launch host or event latency.
-        for _ in range(2 + args.steps // 8):
-            flush_l2()
-        ev[0][0].record()
-        for k in range(args.steps):
-            wl.step()
-        ev[0][1].record()
-        barrier()
-        total_ms = ev[0][0].elapsed_time(ev[0][1])
-        kernel_ms = [total_ms / args.steps]
-    else:
-        for k in range(args.steps):
-            flush_l2()  # evict the working set from L2 between timed iterations (not timed)
-            ev[k][0].record()
-            wl.step()
-            ev[k][1].record()
-            kernel_ms.append(wl.kernel_ms())
-        barrier()
-        total_ms = sum(a.elapsed_time(b) for a, b in ev)
+    total_ms, k_ms = bench.time_steps(wl, args.steps)
+    barrier()
     launches = B.grim_launch_count()
-    wl.check()
+    try:
+        wl.check()
+        parity = "ok"
+    except AssertionError as e:
+        parity = ("FAIL: " + str(e))[:300]
 
     # end to end: host buffers, copies inside the timed region
     for _ in range(2):
@@ -549,47 +681,37 @@ def run_ours(args):
     barrier()
     ev2 = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
     for k in range(args.steps):
-        flush_l2()
+        bench.flush_l2()
         ev2[k][0].record()
         wl.step_e2e()
         ev2[k][1].record()
     barrier()
     e2e_ms = sum(a.elapsed_time(b) for a, b in ev2)
+
+    # the other target configurations, one record each (rank 0 at N = 1 only: they are single-GPU measurements)
+    configs = None
+    if suite and rank == 0 and world == 1:
+        configs = [record_of(bench, wl, "config 5: SpMM 8192^2, N = 1024, c = 8, fp32 (headline)", k_ms, parity)]
+        only = set(args.only.split(",")) if args.only else None
+        for i, (label, make) in enumerate(suite_workloads()):
+            if only is not None and str(i) not in only:
+                continue
+            try:
+                configs.append(measure_config(bench, label, make))
+            except Exception as e:  # a record that cannot be measured is reported, not dropped
+                configs.append(dict(config=label, parity="FAIL: " + repr(e)[:300]))
     clocks = sampler.stop() if rank == 0 else None
 
     total_ms, e2e_ms = max_over_ranks([total_ms, e2e_ms], device="cuda")
 
     if rank == 0:
-        peaks = measured_peaks()
         value = aggregate_value(wl.flops, args.steps, total_ms, world)
         e2e_value = aggregate_value(wl.flops, args.steps, e2e_ms, world)
-        k_ms = statistics.mean(kernel_ms)
-        # binding roofline of the dominant kernel: the slower of (algorithmic bytes at the measured HBM bandwidth) and
-        # (effective flops 2*nnz*N at the peak of the unit that does the arithmetic: plain fp32 FMA pipes, derived as
-        # 148 SMs x 128 lanes x 2 flop x 1.965 GHz, or the measured dense bf16 tensor rate for the tcgen05 kernel)
-        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
-        flop_peak = peaks["bf16_tflops_burst"] if wl.peak_kind == "tensor" else alu_peak
-        t_hbm = wl.kernel_bytes / (peaks["hbm_gbs"] * 1e9)
-        t_flop = wl.flops / (flop_peak * 1e12)
-        bound = getattr(wl, "force_bound", None) or ("hbm" if t_hbm >= t_flop else wl.peak_kind)
-        if bound == "hbm":
-            achieved = wl.kernel_bytes / (k_ms * 1e-3) / 1e9
-            roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
-                        traffic=None, kernel=wl.kernel, kernel_ms=k_ms, algorithmic_bytes=wl.kernel_bytes,
-                        peak_source=peaks["source"])
-        else:
-            achieved = wl.flops / (k_ms * 1e-3) / 1e12
-            roof = dict(bound=bound, achieved=achieved, peak=flop_peak, unit="TFLOP/s", frac=achieved / flop_peak, traffic=None,
-                        kernel=wl.kernel, kernel_ms=k_ms,
-                        peak_source=("measured dense bf16 (burst)" if bound == "tensor"
-                                     else "derived: 148 SM x 128 FMA lanes x 2 x 1.965 GHz"))
-        roof["traffic"] = TRAFFIC.get(wl.name)
-        roof["t_hbm_us"] = t_hbm * 1e6
-        roof["t_flop_us"] = t_flop * 1e6
-        if hasattr(wl, "extra"):
-            roof.update(wl.extra(peaks))
+        roof = bench.roofline(wl, k_ms)
+        roof["parity"] = parity
         cpu_v, cpu_what = wl.oracle_sample()
-        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=max(args.warmup, 3),
+        rotating = bool(getattr(wl, "rotating", False))
+        line = dict(metric=METRIC, value=value, unit=UNIT, n_gpus=world, steps=args.steps, warmup=warmup,
                     ms_per_step=total_ms / args.steps, higher_is_better=True, scaling="weak", vs_baseline=None,
                     dtype=wl.dtype, data="synthetic",
                     config=dict(workload=wl.name, nnz=wl.nnz,
@@ -603,9 +725,183 @@ def run_ours(args):
                     gpu_launches=int(launches), roofline=roof,
                     cpu_baseline=dict(value=cpu_v, unit=UNIT, cores=len(os.sched_getaffinity(0)), kind="oracle",
                                       sample=cpu_what))
+        if configs is not None:
+            line["configs"] = configs
+            line["ffma_peak_tflops_measured"] = bench.ffma_tflops
         print(json.dumps(line))
     if world > 1:
         dist.destroy_process_group()
+
+
+class Bench:
+    """What every measurement needs: the binding, torch, the L2 flush, the peaks."""
+
+    def __init__(self, B, torch):
+        self.B, self.torch = B, torch
+        # written before timed iterations: evicts the working set from L2 (126 MB) and keeps the GPU busy long enough for
+        # the host to queue the step behind it, so that no host latency sits between the events
+        self.flush = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+        self.peaks = measured_peaks()
+        # fp32 FMA ceiling: measured with a register-only micro-kernel at run time (it follows the clock the GPU
+        # sustains); the figure derived from unit counts and the maximum clock is kept beside it for context
+        self.ffma_tflops = B.grim_measure_ffma_peak()
+        self.ffma_derived = 148 * 128 * 2 * 1.965e9 / 1e12
+
+    def flush_l2(self):
+        # the write evicts the working set; the read of half the buffer behind it pushes the write's dirty lines out
+        # to HBM, so that the timed step does not pay for writing them back when its own reads evict them
+        self.flush.zero_()
+        self.flush[: 1 << 29].view(self.torch.int64).sum()
+
+    def time_steps(self, wl, steps):
+        """Times exactly `steps` steps of a workload; returns (total ms over the steps, mean ms of the dominant kernel).
+        Workloads whose operands exceed L2 rotate through operand sets and are queued back to back behind a few
+        flushes (the time between the two events is that of the launches alone); the others are timed one step at a
+        time with an L2 flush before each."""
+        torch = self.torch
+        if bool(getattr(wl, "rotating", False)):
+            wl.per_step_events = False
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            for _ in range(2 + min(steps, 400) // 8):
+                self.flush_l2()
+            e0.record()
+            for _ in range(steps):
+                wl.step()
+            e1.record()
+            e1.synchronize()
+            wl.per_step_events = True
+            total = e0.elapsed_time(e1)
+            return total, total / steps
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(steps)]
+        kernel_ms = []
+        for k in range(steps):
+            self.flush_l2()
+            ev[k][0].record()
+            wl.step()
+            ev[k][1].record()
+            kernel_ms.append(wl.kernel_ms())
+        torch.cuda.synchronize()
+        return sum(a.elapsed_time(b) for a, b in ev), statistics.mean(kernel_ms)
+
+    def roofline(self, wl, k_ms):
+        """Binding bound of the dominant kernel: the slower of (algorithmic bytes at the measured HBM bandwidth) and
+        (effective flops 2*nnz*N at the peak of the unit that does the arithmetic: the measured fp32 FMA rate, or the
+        measured dense bf16 tensor rate for the tcgen05 kernel)."""
+        peaks = self.peaks
+        flop_peak = peaks["bf16_tflops_burst"] if wl.peak_kind == "tensor" else self.ffma_tflops
+        t_hbm = wl.kernel_bytes / (peaks["hbm_gbs"] * 1e9)
+        t_min = getattr(wl, "min_bytes", wl.kernel_bytes) / (peaks["hbm_gbs"] * 1e9)
+        t_flop = wl.flops / (flop_peak * 1e12)
+        bound = getattr(wl, "force_bound", None) or ("hbm" if t_hbm >= t_flop else wl.peak_kind)
+        t = k_ms * 1e-3
+        if bound == "hbm":
+            achieved = wl.kernel_bytes / t / 1e9
+            roof = dict(bound="hbm", achieved=achieved, peak=peaks["hbm_gbs"], unit="GB/s", frac=achieved / peaks["hbm_gbs"],
+                        frac_min_index=t_min / t, traffic=None, kernel=wl.kernel, kernel_ms=k_ms,
+                        algorithmic_bytes=wl.kernel_bytes, min_index_bytes_total=getattr(wl, "min_bytes", None),
+                        peak_source=peaks["source"] + " HBM copy bandwidth")
+        else:
+            achieved = wl.flops / t / 1e12
+            roof = dict(bound=bound, achieved=achieved, peak=flop_peak, unit="TFLOP/s", frac=achieved / flop_peak, traffic=None,
+                        kernel=wl.kernel, kernel_ms=k_ms,
+                        peak_source=("measured dense bf16 (burst)" if bound == "tensor" else
+                                     f"measured fp32 FMA micro-kernel at run time (derived from unit counts at the maximum "
+                                     f"clock: {self.ffma_derived:.1f})"))
+        roof["traffic"] = profile_traffic(wl.name)
+        roof["t_hbm_us"] = t_hbm * 1e6
+        roof["t_flop_us"] = t_flop * 1e6
+        if hasattr(wl, "extra"):
+            roof.update(wl.extra(peaks))
+        return roof
+
+
+def suite_workloads():
+    """The five target configurations as (label, constructor) pairs, in an order that lets consecutive records share
+    generated weights.  The headline point (8192^2, N = 1024, c = 8, fp32) is measured by the main timed region."""
+    from workloads import generators as gen
+
+    def config1():
+        c = gen.config1_spmm()
+        return SpmmWorkload(M=256, N=64, c=4.0, bh=16, bw=16, inputs=c, name="config1_spmm_M256_K256_N64_16x16_keep8x8_fp32")
+
+    S = SpmmWorkload
+    return [
+        ("config 1: SpMM 256^2, N = 64, fp32", config1),
+        ("config 2: GRU 2 x 1024, T = 200, fp32", GruWorkload),
+        ("config 3: conv 512->512 28^2, batch 1, fp32", lambda: ConvWorkload(1, False)),
+        ("config 3: conv 512->512 28^2, batch 1, bf16", lambda: ConvWorkload(1, True)),
+        ("config 3: conv 512->512 28^2, batch 32, fp32", lambda: ConvWorkload(32, False)),
+        ("config 3: conv 512->512 28^2, batch 32, bf16", lambda: ConvWorkload(32, True)),
+        ("config 4: VGG-16 conv stack, batch 1, bf16", lambda: VggWorkload(1)),
+        ("config 4: VGG-16 conv stack, batch 16, bf16", lambda: VggWorkload(16)),
+        ("config 5: GEMV 4096^2, c = 4, fp32", lambda: S(4096, 1, 4.0)),
+        ("config 5: GEMV 8192^2, c = 4, fp32", lambda: S(8192, 1, 4.0)),
+        ("config 5: GEMV 8192^2, c = 4, bf16", lambda: S(8192, 1, 4.0, bf16=True)),
+        ("config 5: SpMM 8192^2, N = 16, c = 4, fp32", lambda: S(8192, 16, 4.0)),
+        ("config 5: SpMM 8192^2, N = 16, c = 4, bf16", lambda: S(8192, 16, 4.0, bf16=True)),
+        ("config 5: SpMM 8192^2, N = 128, c = 8, fp32", lambda: S(8192, 128, 8.0)),
+        ("config 5: SpMM 8192^2, N = 128, c = 8, bf16", lambda: S(8192, 128, 8.0, bf16=True)),
+        ("config 5: SpMM 8192^2, N = 1024, c = 8, bf16", lambda: S(8192, 1024, 8.0, bf16=True)),
+    ]
+
+
+def record_of(bench, wl, label, ms, parity):
+    """One entry of the `configs` array."""
+    roof = bench.roofline(wl, ms)
+    rec = dict(config=label, workload=wl.name, dtype=wl.dtype, nnz=wl.nnz, ms=ms, gflops=wl.flops / (ms * 1e-3) / 1e9,
+               bound=roof["bound"], frac=roof["frac"], frac_min_index=roof.get("frac_min_index"), kernel=wl.kernel,
+               t_hbm_us=roof["t_hbm_us"], t_flop_us=roof["t_flop_us"], parity=parity)
+    if "layers" in roof:
+        rec["layers"] = roof["layers"]
+    if isinstance(wl, GruWorkload):
+        rec["bound"] = "latency (hbm figure: bytes moved once)"
+        rec["us_per_time_step"] = ms * 1e3 / wl.T
+        rec["notional_frac_if_W_hh_were_streamed_every_step"] = wl.notional_bytes / (bench.peaks["hbm_gbs"] * 1e9) / (ms * 1e-3)
+    if wl.peak_kind == "tensor":
+        # the tensor-core kernel multiplies zero-filled tiles: at best the dense rate divided by the compression
+        rec["structural_ceiling_gflops"] = bench.peaks["bf16_tflops_burst"] * 1e3 * wl.nnz / getattr(wl, "dense_elems", wl.nnz)
+    return rec
+
+
+def measure_config(bench, label, make, min_s=0.5):
+    """Sets a workload up, times it for at least `min_s` seconds (so that the clock sampler sees it), checks the last
+    output against the oracle and the handles' status words, and releases it."""
+    torch = bench.torch
+    wl = make()
+    wl.setup(bench.B, torch)
+    for _ in range(3):
+        wl.step()
+    torch.cuda.synchronize()
+    if bool(getattr(wl, "rotating", False)):
+        _, est = bench.time_steps(wl, 20)
+        n = int(min(20000, max(20, math.ceil(min_s * 1e3 / max(est, 1e-4)))))
+        _, ms = bench.time_steps(wl, n)
+    else:
+        # one launch at a time behind an L2 flush; the flushes count towards the duration (the GPU is busy throughout)
+        samples, t0 = [], time.perf_counter()
+        while len(samples) < 20 or (time.perf_counter() - t0 < min_s and len(samples) < 2000):
+            bench.flush_l2()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            wl.step()
+            e1.record()
+            e1.synchronize()
+            # the stack and the GRU report the whole pass (their latency is the figure of merit); single kernels too
+            samples.append(e0.elapsed_time(e1))
+            if hasattr(wl, "layer_ms"):
+                wl.kernel_ms()
+        ms = statistics.median(samples)
+    try:
+        wl.check()
+        parity = "ok"
+    except AssertionError as e:
+        parity = ("FAIL: " + str(e))[:300]
+    rec = record_of(bench, wl, label, ms, parity)
+    wl.close()
+    del wl
+    torch.cuda.empty_cache()
+    return rec
+
 
 def run_sweep(args):
     """The SpMM sweep: square W with M = K in {1024, 4096, 8192}, N in {1, 16, 128, 1024}, compression in {4, 8, 16},
@@ -678,10 +974,11 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="gru", choices=["gru", "gemv", "spmm", "conv", "vgg"])
+    ap.add_argument("--workload", default="suite", choices=["suite", "gru", "gemv", "spmm", "conv", "vgg"])
+    ap.add_argument("--only", default="", help="suite: comma-separated indices of the extra records to measure (default: all)")
     ap.add_argument("--image", type=int, default=224)
     ap.add_argument("--size", type=int, default=8192)
     ap.add_argument("--ncols", type=int, default=128)

@@ -272,6 +272,12 @@ grim_status_t grim_gru_debug_barrier(grim_gru_t g, int skip_cta, unsigned spin_l
 grim_status_t grim_gru_profile(grim_gru_t g, int enable);
 grim_status_t grim_gru_profile_read(grim_gru_t g, float* projection_ms, float* recurrent_ms);
 
+/* Measures the fp32 fused-multiply-add rate of the current device with a register-only micro-kernel (16 independent
+ * chains per thread, full occupancy) and returns it in TFLOP/s: the ceiling against which the CUDA-core multiply is
+ * reported (measurement aid for Section 6 style reporting; no counterpart in the paper).  Allocates and frees a
+ * small device buffer and synchronises `stream`. */
+grim_status_t grim_measure_ffma_peak(double* tflops, grim_stream_t stream);
+
 /* Counts kernel launches issued by this library since load (or since the last reset). */
 int64_t grim_launch_count(void);
 void grim_launch_count_reset(void);

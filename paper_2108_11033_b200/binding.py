@@ -33,7 +33,7 @@ EXPORTED = [
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
-    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version",
+    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak",
 ]
 
 
@@ -89,6 +89,7 @@ lib.grim_gru_debug_barrier.argtypes = [_vp, C.c_int, C.c_uint]
 lib.grim_gru_profile.argtypes = [_vp, C.c_int]
 lib.grim_gru_set_pipeline.argtypes = [_vp, C.c_int]
 lib.grim_gru_profile_read.argtypes = [_vp, C.POINTER(C.c_float), C.POINTER(C.c_float)]
+lib.grim_measure_ffma_peak.argtypes = [C.POINTER(C.c_double), _vp]
 lib.grim_launch_count.restype = C.c_int64
 lib.grim_launch_count_reset.restype = None
 lib.grim_status_string.argtypes = [C.c_int]
@@ -268,6 +269,12 @@ def grim_gru_profile_read(g: int):
 
 def grim_gru_destroy(g: int):
     _check(lib.grim_gru_destroy(g), "grim_gru_destroy")
+
+
+def grim_measure_ffma_peak(stream=None) -> float:
+    v = C.c_double(0.0)
+    _check(lib.grim_measure_ffma_peak(C.byref(v), _stream_ptr(stream)), "grim_measure_ffma_peak")
+    return float(v.value)
 
 
 def grim_launch_count() -> int:

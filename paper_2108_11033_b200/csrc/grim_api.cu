@@ -54,6 +54,28 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
   return launch_spmm(h, a, s);
 }
 
+int dev_sms() {
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) dev = 0;
+  return sm_count(dev);
+}
+
+// 16 independent chains of dependent fused multiply-adds per thread: enough independent work per warp to keep
+// the fp32 pipes full at full occupancy.  The result is stored so that nothing is optimised away.
+__global__ void __launch_bounds__(512) ffma_peak_kernel(float* __restrict__ out, int iters, float a, float b) {
+  float acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = (float)(threadIdx.x + i);
+  for (int it = 0; it < iters; ++it) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) acc[i] = fmaf(acc[i], a, b);
+  }
+  float sum = 0.f;
+#pragma unroll
+  for (int i = 0; i < 16; ++i) sum += acc[i];
+  out[blockIdx.x * (int64_t)blockDim.x + threadIdx.x] = sum;
+}
+
 template <typename T>
 __global__ void maxpool2x2_kernel(const T* __restrict__ in, T* __restrict__ out, int64_t planes, int H, int W) {
   const int OH = H / 2, OW = W / 2;
@@ -153,7 +175,7 @@ extern "C" grim_status_t grim_maxpool2x2(const void* in, void* out, int64_t N, i
   if (dtype != GRIM_F32 && dtype != GRIM_BF16) return GRIM_ERR_DTYPE;
   const int64_t total = N * C * (H / 2) * (W / 2);
   const int threads = 256;
-  const int blocks = (int)std::min<int64_t>((total + threads - 1) / threads, 148 * 16);
+  const int blocks = (int)std::min<int64_t>((total + threads - 1) / threads, (int64_t)dev_sms() * 16);
   cudaStream_t s = (cudaStream_t)stream;
   if (dtype == GRIM_F32)
     maxpool2x2_kernel<float><<<blocks, threads, 0, s>>>((const float*)in, (float*)out, N * C, (int)H, (int)W);
@@ -162,6 +184,34 @@ extern "C" grim_status_t grim_maxpool2x2(const void* in, void* out, int64_t N, i
                                                                 (int)H, (int)W);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
+}
+
+extern "C" grim_status_t grim_measure_ffma_peak(double* tflops, grim_stream_t stream) {
+  if (!tflops) return GRIM_ERR_INVALID_ARG;
+  cudaStream_t s = (cudaStream_t)stream;
+  const int blocks = dev_sms() * 4, threads = 512, iters = 4096;
+  float* out = nullptr;
+  if (cudaMalloc((void**)&out, (size_t)blocks * threads * 4) != cudaSuccess) { cudaGetLastError(); return GRIM_ERR_ALLOC; }
+  cudaEvent_t e0 = nullptr, e1 = nullptr;
+  grim_status_t st = GRIM_OK;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) st = GRIM_ERR_CUDA;
+  float best = -1.f;
+  for (int rep = 0; rep < 6 && st == GRIM_OK; ++rep) {  // the first repetition is a warm-up
+    cudaEventRecord(e0, s);
+    ffma_peak_kernel<<<blocks, threads, 0, s>>>(out, iters, 0.999f, 0.001f);
+    cudaEventRecord(e1, s);
+    count_launch();
+    if (cudaEventSynchronize(e1) != cudaSuccess) { st = GRIM_ERR_CUDA; break; }
+    float ms = 0.f;
+    cudaEventElapsedTime(&ms, e0, e1);
+    if (rep > 0 && (best < 0.f || ms < best)) best = ms;
+  }
+  if (e0) cudaEventDestroy(e0);
+  if (e1) cudaEventDestroy(e1);
+  cudaFree(out);
+  if (st != GRIM_OK || best <= 0.f) return st == GRIM_OK ? GRIM_ERR_CUDA : st;
+  *tflops = 2.0 * 16.0 * iters * (double)blocks * threads / (best * 1e-3) / 1e12;
+  return GRIM_OK;
 }
 
 extern "C" const char* grim_status_string(grim_status_t s) {

@@ -546,7 +546,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   const int64_t qtiles = (a.ncols + kTN - 1) / kTN;
   // band groups per thread block: as many as the accumulators allow, fewer when the grid would not fill the GPU
   int bpw = BHc == 4 ? 4 : (BHc == 8 ? 2 : 1);
-  while (bpw > 1 && (smem_need(h, bpw, esz) > kSmemBudget || qtiles * ((h->rc_groups + bpw - 1) / bpw) < 148)) bpw >>= 1;
+  while (bpw > 1 && (smem_need(h, bpw, esz) > kSmemBudget || qtiles * ((h->rc_groups + bpw - 1) / bpw) < sm_count(h->device))) bpw >>= 1;
   const int tn = a.tile_n % 256;
   if (tn == 1 || tn == 2 || tn == 4) bpw = std::min(tn, BHc == 4 ? 4 : (BHc == 8 ? 2 : 1));
   if (smem_need(h, bpw, esz) > kSmemBudget) return GRIM_ERR_UNSUPPORTED;
@@ -555,8 +555,8 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   // too few tiles for the GPU: split the block columns over several thread blocks (fp32 output only)
   int ksplit = 1;
   const bool split_ok = a.y_dtype == GRIM_F32 && (a.conv || a.y_sq == 1 || a.y_sr == 1);
-  if (split_ok && qtiles * gy * 2 <= 148) {
-    ksplit = (int)std::min<int64_t>(std::min<int64_t>(8, 148 / (qtiles * gy)), std::max<int64_t>(1, h->nbc / 4));
+  if (split_ok && qtiles * gy * 2 <= sm_count(h->device)) {
+    ksplit = (int)std::min<int64_t>(std::min<int64_t>(8, sm_count(h->device) / (qtiles * gy)), std::max<int64_t>(1, h->nbc / 4));
     if (ksplit < 1) ksplit = 1;
   }
   if (a.tile_n >= 256) ksplit = split_ok ? std::max(1, std::min(8, a.tile_n / 256)) : 1;  // test / tuning override
@@ -603,7 +603,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   count_launch();
   if (e == cudaSuccess && ksplit > 1 && (a.bias || a.relu) && !(a.y_prefilled && !a.relu)) {
     const int64_t total = h->M * a.ncols;
-    bcr_finalize_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, 148 * 8), 256, 0, s>>>(a, (int)h->M);
+    bcr_finalize_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, (int64_t)sm_count(h->device) * 8), 256, 0, s>>>(a, (int)h->M);
     count_launch();
     e = cudaGetLastError();
   }

@@ -905,7 +905,7 @@ extern "C" grim_status_t grim_gru_seq(grim_gru_t g, const float* x, int64_t T, c
   // every row of a pre-activation buffer starts as b_ih: the projections may add partial sums onto it
   auto prefill = [&](int l, cudaStream_t s) {
     const int64_t total = T * 3 * H;
-    fill_rows_kernel<<<(unsigned)std::min<int64_t>((total / 4 + 255) / 256, 148 * 8), 256, 0, s>>>(g->d_gi[(size_t)l], g->d_bih[(size_t)l], T, 3 * H);
+    fill_rows_kernel<<<(unsigned)std::min<int64_t>((total / 4 + 255) / 256, (int64_t)sm_count(g->device) * 8), 256, 0, s>>>(g->d_gi[(size_t)l], g->d_bih[(size_t)l], T, 3 * H);
     count_launch();
     return cudaGetLastError() == cudaSuccess;
   };

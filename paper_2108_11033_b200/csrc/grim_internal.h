@@ -182,5 +182,7 @@ bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a);
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a);
 void count_launch(int n = 1);
+// streaming multiprocessors of a device (read once per device through the runtime)
+int sm_count(int device);
 
 }  // namespace grim

@@ -23,6 +23,21 @@ namespace grim {
 
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+int sm_count(int device) {
+  constexpr int kFallback = 148;  // B200; used only when the attribute cannot be read
+  static int cached[64] = {0};
+  if (device < 0 || device >= 64) return kFallback;
+  if (!cached[device]) {
+    int n = 0;
+    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) {
+      cudaGetLastError();
+      n = kFallback;
+    }
+    cached[device] = n;
+  }
+  return cached[device];
+}
 long long launches() { return g_launches.load(std::memory_order_relaxed); }
 void launches_reset() { g_launches.store(0, std::memory_order_relaxed); }
 
@@ -558,7 +573,7 @@ grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64
   const int passes = (int)((N + nq - 1) / nq);
   // enough warps to keep every SM's memory pipeline busy: split a band over several warps when bands are few
   int wpb = 1;
-  const int64_t want_warps = 148 * 20;
+  const int64_t want_warps = (int64_t)sm_count(h->device) * 20;
   while (wpb < 8 && (int64_t)nbr * passes * wpb < want_warps && (int64_t)nbr * wpb * 8 <= h->nchunks) wpb *= 2;
   const int bpc = kWarps / wpb;
   SkinnyParams p;

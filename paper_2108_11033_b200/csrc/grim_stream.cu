@@ -363,17 +363,6 @@ struct StreamPlan {
   size_t smem;
 };
 
-int sm_count(int device) {
-  static int cached[64] = {0};
-  if (device < 0 || device >= 64) return 148;
-  if (!cached[device]) {
-    int n = 0;
-    if (cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, device) != cudaSuccess || n <= 0) n = 148;
-    cached[device] = n;
-  }
-  return cached[device];
-}
-
 bool make_plan(const grim_bcr* h, int64_t N, StreamPlan& pl) {
   if (h->device < 0 || !h->gemv_ok || !h->d_status || !h->d_runs || N < 1 || N > kSkinnyMaxN || h->nchunks == 0) return false;
   const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);

@@ -826,7 +826,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   p.ksplit = 1; p.kt_per = p.nkt; p.acc = nullptr;
   {
     const int64_t blocks = qtiles_ * ((h->tc_mtiles + p.mt - 1) / p.mt);
-    const int sms = 148;
+    const int sms = sm_count(h->device);
     // (measured on the VGG-16 layers: worth it from about 16 K tiles per block; with fewer, clearing the scratch,
     // the reductions into it and the second pass cost more than the shorter K loop saves)
     int want = (int)std::min<int64_t>(16, sms / std::max<int64_t>(blocks, 1));
@@ -852,7 +852,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   auto finalize = [&]() -> grim_status_t {
     if (p.ksplit <= 1) return GRIM_OK;
     const int64_t total = (int64_t)h->M * a.ncols;
-    const int blocks = (int)std::min<int64_t>((total + 255) / 256, 148 * 8);
+    const int blocks = (int)std::min<int64_t>((total + 255) / 256, (int64_t)sm_count(h->device) * 8);
     tc_finalize_kernel<<<blocks, 256, 0, s>>>(p.acc, a.ncols, (int)h->M, a.bias, a.relu, a.Y, a.y_dtype, a.y_sr, a.conv,
                                               (int64_t)a.OH * a.OW);
     count_launch();

@@ -1,6 +1,6 @@
 """GPU parity: every CUDA entry point against the fp64 CPU oracle, element by element, through the C ABI.
 
-Tolerances (fixed by the benchmark spec): fp32 results  ||Y - Y*||_F / ||Y*||_F <= 1e-5;
+Tolerances (fixed requirements of this library): fp32 results  ||Y - Y*||_F / ||Y*||_F <= 1e-5;
 bf16 inputs with fp32 accumulation  max |err| <= 2e-2 * ||W row||_2 * ||X col||_2 (plus |bias| where
 a bias is added); packing is bit-exact (tests/test_packer_host.py).  Rows kept by no block must be
 exactly +0.
