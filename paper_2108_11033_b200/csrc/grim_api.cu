@@ -32,13 +32,17 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
   grim_status_t st = check_mats(h, X, Y);
   if (st != GRIM_OK) return st;
   int path = tune ? tune->path : 0;
-  if (path < 0 || path > 4) return GRIM_ERR_INVALID_ARG;
+  if (path < 0 || path > 5) return GRIM_ERR_INVALID_ARG;
   if (path == 0 && tune && tune->tile_n >= 16) path = 4;  // a column-tile width only means something to the slab kernel
   SpmmArgs a = mat_args(X, Y);
   a.tile_n = tune ? tune->tile_n : 0;
   if (path == 2) {
     if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
     return launch_spmm_tc(h, a, s);
+  }
+  if (path == 5) {
+    if (!tc2_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
+    return launch_spmm_tc2(h, a, s);
   }
   if (path == 3 || (path == 0 && X->cols <= kSkinnyMaxN && h->gemv_ok)) {
     // tile_n = 1 under path 3 asks for the register-staged variant; otherwise the streaming one runs when it can

@@ -88,6 +88,21 @@ struct RcStage {
 constexpr int kTcRows = 128;
 constexpr int kTcK = 64;
 
+// ---------------------------------------------------------------------------------------------
+// Tile-descriptor layout of the paired tensor-core kernel: the same 128 x 64 tiles, but a record is a fixed-size
+// table of block descriptors followed by the kept values in canonical order (per block kr x kc, row-major; blocks
+// by band, then by block column).  One descriptor covers one band and kTdSeg columns of the tile (a whole block for
+// bw <= 32, half a block for bw = 64; both halves then carry the block's first value).  Descriptor d of a tile is
+// band_in_tile * (64 / seg) + segment, seg = min(bw, 32).  This is what lets a thread own a 16-byte piece of the
+// expanded tile: everything it needs is one descriptor and a run of consecutive values.
+// ---------------------------------------------------------------------------------------------
+constexpr int kTdSeg = 32;
+struct TdDesc {
+  uint32_t colmask;  // kept columns of the segment (bit c: segment-local column c)
+  uint16_t rowmask;  // kept rows of the band (bit r: band-local row r)
+  uint16_t val_off;  // first value of the block, in elements from the start of the record's values
+};
+
 struct HostBlock {
   uint64_t colmask = 0;
   uint32_t rowmask = 0;
@@ -133,6 +148,10 @@ struct grim_bcr {
   int64_t index_bytes_tc = 0;
   grim::RcStage* d_tc_stage = nullptr;
   uint8_t* d_tc_blob = nullptr;
+  uint32_t td_max_rec = 0;
+  int64_t index_bytes_td = 0;
+  grim::RcStage* d_td_stage = nullptr;
+  uint8_t* d_td_blob = nullptr;
   float* d_tc_acc = nullptr;  // fp32 scratch of the split tensor-core multiply (M x N), grown on first use
   size_t tc_acc_bytes = 0;
   unsigned* d_status = nullptr;  // error word written by kernels whose bounded waits ran out
@@ -181,6 +200,9 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 bool ffma_path_supported(const grim_bcr* h, const SpmmArgs& a);
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a);
+// the paired (two thread blocks per tile pair) tensor-core kernel: matrices, bf16 handles
+grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s);
+bool tc2_path_supported(const grim_bcr* h, const SpmmArgs& a);
 void count_launch(int n = 1);
 // streaming multiprocessors of a device (read once per device through the runtime)
 int sm_count(int device);

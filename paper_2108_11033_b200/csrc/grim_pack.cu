@@ -52,6 +52,8 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_runs);
   cudaFree(h->d_rc_stage);
   cudaFree(h->d_rc_blob);
+  cudaFree(h->d_td_stage);
+  cudaFree(h->d_td_blob);
   cudaFree(h->d_tc_stage);
   cudaFree(h->d_tc_blob);
   cudaFree(h->d_status);
@@ -428,6 +430,60 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       h->index_bytes_tc = (int64_t)tc_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)tc_blob.size() - (int64_t)nnz * 2 + nbr * 4;
     }
 
+    // ---- tile-descriptor layout of the paired tensor-core kernel (same shapes and tiles as above)
+    std::vector<RcStage> td_stage;
+    std::vector<uint8_t> td_blob;
+    if (tc_shape) {
+      const int S = kTcRows / bh, J = kTcK / bw;
+      const int seg = bw < kTdSeg ? bw : kTdSeg;       // columns per descriptor
+      const int nseg = kTcK / seg;                      // descriptors per band of a tile
+      const size_t table_bytes = (size_t)S * nseg * sizeof(TdDesc);
+      td_stage.resize((size_t)(h->tc_mtiles * h->tc_ktiles));
+      uint32_t td_max = 0;
+      std::vector<TdDesc> table((size_t)S * nseg);
+      std::vector<uint16_t> tv;
+      for (int64_t t = 0; t < h->tc_mtiles && st == GRIM_OK; ++t)
+        for (int64_t kt = 0; kt < h->tc_ktiles; ++kt) {
+          std::fill(table.begin(), table.end(), TdDesc{0u, 0u, 0u});
+          tv.clear();
+          for (int ts = 0; ts < S; ++ts) {
+            const int64_t pos = t * S + ts;
+            if (pos >= nbr) break;
+            for (int jj = 0; jj < J; ++jj) {
+              const int64_t j = kt * J + jj;
+              if (j >= nbc) break;
+              const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
+              if (!(hb.kr && hb.kc)) continue;
+              const size_t first = tv.size();
+              for (size_t v = 0; v < (size_t)hb.kr * hb.kc; ++v) tv.push_back(bf16_bits(h->vals[(size_t)hb.val_off + v]));
+              for (int c0 = 0; c0 < bw; c0 += seg) {  // one descriptor per segment of the block
+                TdDesc& dsc = table[(size_t)ts * nseg + (size_t)(jj * bw + c0) / seg];
+                dsc.colmask = (uint32_t)((hb.colmask >> c0) & (seg == 32 ? 0xFFFFFFFFull : ((1ull << seg) - 1)));
+                dsc.rowmask = (uint16_t)hb.rowmask;
+                dsc.val_off = (uint16_t)first;
+              }
+            }
+          }
+          RcStage& se = td_stage[(size_t)(t * h->tc_ktiles + kt)];
+          se.off16 = (uint32_t)(td_blob.size() / 16);
+          se.bytes = 0;
+          if (tv.empty()) continue;
+          if (td_blob.size() / 16 >= (uint64_t(1) << 32) || tv.size() > 0xFFFFu) { st = GRIM_ERR_UNSUPPORTED; break; }
+          const size_t start = td_blob.size();
+          // one spare vector of values behind the last: the kernel's loads are predicated, the padding only keeps
+          // records 16-byte sized
+          const size_t vbytes = (tv.size() * 2 + 15) / 16 * 16;
+          td_blob.resize(start + table_bytes + vbytes, 0);
+          std::memcpy(&td_blob[start], table.data(), table_bytes);
+          std::memcpy(&td_blob[start + table_bytes], tv.data(), tv.size() * 2);
+          se.bytes = (uint32_t)(td_blob.size() - start);
+          td_max = std::max(td_max, se.bytes);
+        }
+      if (st != GRIM_OK) { delete h; return st; }
+      h->td_max_rec = td_max;
+      h->index_bytes_td = (int64_t)td_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)td_blob.size() - (int64_t)nnz * 2 + nbr * 4;
+    }
+
     // ---- upload
     if (!(flags & GRIM_PACK_HOST_ONLY)) {
       cudaError_t e = cudaGetDevice(&h->device);
@@ -439,6 +495,8 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       if (e == cudaSuccess && tc_shape) {
         e = upload(&h->d_tc_stage, tc_stage.data(), tc_stage.size() * sizeof(RcStage));
         if (e == cudaSuccess) e = upload(&h->d_tc_blob, tc_blob.data(), tc_blob.size());
+        if (e == cudaSuccess) e = upload(&h->d_td_stage, td_stage.data(), td_stage.size() * sizeof(RcStage));
+        if (e == cudaSuccess) e = upload(&h->d_td_blob, td_blob.data(), td_blob.size());
       }
       const unsigned zero = 0;
       if (e == cudaSuccess) e = upload(&h->d_status, &zero, 4);

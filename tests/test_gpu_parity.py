@@ -148,6 +148,22 @@ def test_tensor_core_kernel_explicit(B, case, y_bf16):
     check_spmm(B, W, mask, X, bh, bw, bf16=True, path=2, flags=1, y_bf16=y_bf16)
 
 
+@pytest.mark.parametrize("y_bf16", [False, True])
+@pytest.mark.parametrize("case", [(256, 512, 8, 32, 512), (328, 700, 8, 32, 520), (300, 520, 4, 16, 1032), (260, 700, 16, 64, 264),
+                                  (96, 153, 8, 32, 1024), (512, 2048, 16, 64, 776), (640, 320, 4, 32, 600), (400, 256, 8, 16, 520),
+                                  (384, 448, 16, 16, 512), (384, 448, 16, 32, 136), (200, 333, 4, 64, 328), (1100, 900, 8, 64, 1544)])
+def test_paired_tensor_core_kernel_explicit(B, case, y_bf16):
+    """The paired tcgen05 kernel asked for by name (path 5): two thread blocks multiply 256 rows x 512 columns
+    together.  Ragged M, K and N, an odd number of 128-row tiles (the last pair has one empty partner), a single
+    tile, empty blocks, pruned bands, every supported block shape."""
+    M, K, bh, bw, N = case
+    W = gen.dense_weight(M, K, seed=187)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=188, empty_frac=0.1)
+    mask[: 2 * bh] = 0
+    X = gen.normal_f32((K, N), 1.0, 189, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=True, path=5, flags=1, y_bf16=y_bf16)
+
+
 @pytest.mark.parametrize("split", [2, 5, 8])
 def test_split_multiply(B, split):
     """Few output tiles: several thread blocks share a tile's block columns and add their partial sums into a
