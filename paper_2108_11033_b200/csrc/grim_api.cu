@@ -52,6 +52,11 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
     return launch_skinny(h, X->ptr, X->dtype, X->ld, X->cols, Y->ptr, Y->dtype, Y->ld, s);
   }
   if (path == 4) return launch_spmm(h, a, s);
+  // bf16 handles, wide right-hand sides: tensor cores.  The paired kernel when its 256 x 512 tiles still give most
+  // SMs a thread block (measured: with fewer, the single-block kernel's smaller tiles win).
+  if (path == 0 && tc2_path_supported(h, a) && a.ncols >= 256 &&
+      2 * ((h->tc_mtiles + 1) / 2) * ((a.ncols + 511) / 512) * 3 >= 2 * (int64_t)sm_count(h->device))
+    return launch_spmm_tc2(h, a, s);
   if (path == 0 && tc_path_supported(h, a) && a.ncols >= 128) return launch_spmm_tc(h, a, s);
   if (ffma_path_supported(h, a)) return launch_ffma(h, a, s);
   if (path == 1) return GRIM_ERR_UNSUPPORTED;

@@ -75,6 +75,13 @@ __device__ __forceinline__ bool mbar_try_wait_cluster(uint64_t* bar, unsigned pa
                : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
   return ok != 0;
 }
+// Non-blocking test of a phase (acquire, cluster scope): returns at once with the current answer.
+__device__ __forceinline__ bool mbar_test_wait_cluster(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.test_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
+               : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  return ok != 0;
+}
 // Bounded wait: polls at most `limit` times with a short sleep between polls (most warps of a block wait at any
 // time; polling flat out would take issue slots from the working ones) and gives up early when the block's abort
 // flag is set.  Returns false when it gave up.
@@ -108,6 +115,38 @@ __device__ __forceinline__ void cluster_sync_all() {
 }
 __device__ __forceinline__ void sts128(uint32_t saddr, uint32_t x, uint32_t y, uint32_t z, uint32_t w) {
   asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(x), "r"(y), "r"(z), "r"(w) : "memory");
+}
+
+__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
+  uint4 v;
+  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
+  return v;
+}
+__device__ __forceinline__ void sts16(uint32_t saddr, uint32_t low_half) {
+  asm volatile("st.shared.u16 [%0], %1;" ::"r"(saddr), "h"((unsigned short)low_half) : "memory");
+}
+// Barrier among `nthreads` threads (a multiple of 32) that all name the same id (1 .. 15; 0 is __syncthreads).
+__device__ __forceinline__ void named_barrier(int id, int nthreads) {
+  asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// Expands one record of the tensor-core scatter layout (32-bit entries: bf16 value | byte offset in the tile << 16,
+// `bytes` of them at shared address rec_s, a multiple of 16; 0 = the tile keeps nothing) into the 16 KiB weight
+// tile at shared address a_s.  Called by all NT threads of a group (wt = 0 .. NT - 1) that own barrier `bar_id`:
+// the tile is cleared, the group meets, and every entry is stored.
+template <int NT>
+__device__ __forceinline__ void expand_scatter(uint32_t rec_s, uint32_t bytes, uint32_t a_s, int wt, int bar_id) {
+#pragma unroll
+  for (int i = 0; i < 16384 / 16 / NT; ++i) sts128(a_s + (uint32_t)(wt + i * NT) * 16u, 0u, 0u, 0u, 0u);
+  named_barrier(bar_id, NT);
+  const uint32_t n16 = bytes >> 4;
+  for (uint32_t v = (uint32_t)wt; v < n16; v += NT) {
+    const uint4 e = lds128(rec_s + v * 16u);
+    sts16(a_s + (e.x >> 16), e.x);
+    sts16(a_s + (e.y >> 16), e.y);
+    sts16(a_s + (e.z >> 16), e.z);
+    sts16(a_s + (e.w >> 16), e.w);
+  }
 }
 
 }  // namespace ptx

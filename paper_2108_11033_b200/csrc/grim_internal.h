@@ -77,31 +77,23 @@ struct RcStage {
 };
 
 // ---------------------------------------------------------------------------------------------
-// Device layout for the tensor-core kernel (bf16 handles with bh in {4, 8, 16}, bw in {16, 32, 64}).
-// The matrix is cut into tiles of kTcRows rows (consecutive bands in schedule order) x kTcK columns;
-// per tile one contiguous record that lists its kept columns, sorted by kept-row count (largest first):
-//   u32 ncols, u32 nvals, u32 0, u32 0
-//   u32 colword[ncols]   k inside the tile (6 bits) | band inside the tile << 6 | row mask << 16; padded to x4
-//   u16 voff[ncols]      first value of the column; padded to x8
-//   bf16 val[nvals]      the column's kept values, top row first; padded to x8
+// Tiling of the tensor-core kernels (bf16 handles with bh in {4, 8, 16}, bw in {16, 32, 64}): the matrix is cut into
+// tiles of kTcRows rows (consecutive bands in schedule order) x kTcK columns, one record per tile.
 // ---------------------------------------------------------------------------------------------
 constexpr int kTcRows = 128;
 constexpr int kTcK = 64;
 
 // ---------------------------------------------------------------------------------------------
-// Tile-descriptor layout of the paired tensor-core kernel: the same 128 x 64 tiles, but a record is a fixed-size
-// table of block descriptors followed by the kept values in canonical order (per block kr x kc, row-major; blocks
-// by band, then by block column).  One descriptor covers one band and kTdSeg columns of the tile (a whole block for
-// bw <= 32, half a block for bw = 64; both halves then carry the block's first value).  Descriptor d of a tile is
-// band_in_tile * (64 / seg) + segment, seg = min(bw, 32).  This is what lets a thread own a 16-byte piece of the
-// expanded tile: everything it needs is one descriptor and a run of consecutive values.
+// Scatter layout of the tensor-core kernels: a record is the list of the tile's kept values as
+// 32-bit entries: bf16 value (low half) | byte offset of the element in the expanded tile (high half), the tile being
+// K-major with rows of 128 bytes whose 16-byte pieces are XOR-ed with the row's low three bits (the tensor core's
+// 128-byte swizzle).  Entries are in canonical order (band, block column, kept row, kept column) and padded to a
+// multiple of four by repeating the last one.  Expanding a tile is then: clear it, and per entry one 2-byte store
+// - no index arithmetic on the device.  The price is 2 index bytes per value.
 // ---------------------------------------------------------------------------------------------
-constexpr int kTdSeg = 32;
-struct TdDesc {
-  uint32_t colmask;  // kept columns of the segment (bit c: segment-local column c)
-  uint16_t rowmask;  // kept rows of the band (bit r: band-local row r)
-  uint16_t val_off;  // first value of the block, in elements from the start of the record's values
-};
+inline uint32_t td_offset(uint32_t row, uint32_t col) {
+  return row * 128u + ((((col >> 3) ^ (row & 7u))) << 4) + (col & 7u) * 2u;
+}
 
 struct HostBlock {
   uint64_t colmask = 0;
@@ -144,12 +136,8 @@ struct grim_bcr {
   uint8_t* d_rc_blob = nullptr;
   // tensor-core layout
   int64_t tc_mtiles = 0, tc_ktiles = 0;
-  uint32_t tc_max_rec = 0;
   int64_t index_bytes_tc = 0;
-  grim::RcStage* d_tc_stage = nullptr;
-  uint8_t* d_tc_blob = nullptr;
   uint32_t td_max_rec = 0;
-  int64_t index_bytes_td = 0;
   grim::RcStage* d_td_stage = nullptr;
   uint8_t* d_td_blob = nullptr;
   float* d_tc_acc = nullptr;  // fp32 scratch of the split tensor-core multiply (M x N), grown on first use

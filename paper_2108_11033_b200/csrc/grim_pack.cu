@@ -54,8 +54,6 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_rc_blob);
   cudaFree(h->d_td_stage);
   cudaFree(h->d_td_blob);
-  cudaFree(h->d_tc_stage);
-  cudaFree(h->d_tc_blob);
   cudaFree(h->d_status);
 }
 
@@ -368,84 +366,25 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
                           nbr * 4;
     }
 
-    // ---- tensor-core layout (bf16 handles whose block shape tiles 128 x 64 evenly)
-    std::vector<RcStage> tc_stage;
-    std::vector<uint8_t> tc_blob;
+    // ---- tensor-core tiling (bf16 handles whose block shape tiles 128 x 64 evenly)
     const bool tc_shape = vdt == GRIM_BF16 && (bh == 4 || bh == 8 || bh == 16) && (bw == 16 || bw == 32 || bw == 64);
     if (tc_shape) {
-      const int S = kTcRows / bh, J = kTcK / bw;
-      h->tc_mtiles = (nbr + S - 1) / S;
-      h->tc_ktiles = (nbc + J - 1) / J;
-      tc_stage.resize((size_t)(h->tc_mtiles * h->tc_ktiles));
-      struct Col { uint32_t word; uint16_t kr, kc; const float* src; };
-      std::vector<Col> cols;
-      uint32_t tc_max = 0;
-      for (int64_t t = 0; t < h->tc_mtiles && st == GRIM_OK; ++t)
-        for (int64_t kt = 0; kt < h->tc_ktiles; ++kt) {
-          cols.clear();
-          uint32_t nvals = 0;
-          for (int ts = 0; ts < S; ++ts) {
-            const int64_t pos = t * S + ts;
-            if (pos >= nbr) break;
-            for (int jj = 0; jj < J; ++jj) {
-              const int64_t j = kt * J + jj;
-              if (j >= nbc) break;
-              const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
-              if (!(hb.kr && hb.kc)) continue;
-              int b = 0;
-              for (int c = 0; c < bw; ++c)
-                if ((hb.colmask >> c) & 1ull) {
-                  cols.push_back(Col{(uint32_t)(jj * bw + c) | ((uint32_t)ts << 6) | (hb.rowmask << 16), hb.kr, hb.kc,
-                                     &h->vals[(size_t)hb.val_off + (size_t)b]});
-                  ++b;
-                  nvals += hb.kr;
-                }
-            }
-          }
-          RcStage& se = tc_stage[(size_t)(t * h->tc_ktiles + kt)];
-          se.off16 = (uint32_t)(tc_blob.size() / 16);
-          se.bytes = 0;
-          if (cols.empty()) continue;
-          if (tc_blob.size() / 16 >= (uint64_t(1) << 32) || nvals > 0xFFFFu) { st = GRIM_ERR_UNSUPPORTED; break; }
-          std::stable_sort(cols.begin(), cols.end(), [](const Col& x, const Col& y) { return x.kr > y.kr; });
-          const size_t n = cols.size(), n4 = (n + 3) / 4 * 4, n8 = (n + 7) / 8 * 8, v8 = ((size_t)nvals + 8) / 8 * 8;  // at least one spare value: the kernel reads one past a column's last
-          const size_t start = tc_blob.size();
-          tc_blob.resize(start + 16 + n4 * 4 + n8 * 2 + v8 * 2, 0);
-          uint32_t* hdr = reinterpret_cast<uint32_t*>(&tc_blob[start]);
-          hdr[0] = (uint32_t)n; hdr[1] = nvals;
-          uint32_t* cw = hdr + 4;
-          uint16_t* vo = reinterpret_cast<uint16_t*>(cw + n4);
-          uint16_t* vv = vo + n8;
-          uint32_t o = 0;
-          for (size_t i = 0; i < n; ++i) {
-            cw[i] = cols[i].word;
-            vo[i] = (uint16_t)o;
-            for (int a = 0; a < cols[i].kr; ++a) vv[o++] = bf16_bits(cols[i].src[(size_t)a * cols[i].kc]);
-          }
-          se.bytes = (uint32_t)(tc_blob.size() - start);
-          tc_max = std::max(tc_max, se.bytes);
-        }
-      if (st != GRIM_OK) { delete h; return st; }
-      h->tc_max_rec = tc_max;
-      h->index_bytes_tc = (int64_t)tc_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)tc_blob.size() - (int64_t)nnz * 2 + nbr * 4;
+      h->tc_mtiles = (nbr + kTcRows / bh - 1) / (kTcRows / bh);
+      h->tc_ktiles = (nbc + kTcK / bw - 1) / (kTcK / bw);
     }
 
-    // ---- tile-descriptor layout of the paired tensor-core kernel (same shapes and tiles as above)
+    // ---- scatter layout of the tensor-core kernels (same shapes and tiles as above): per tile the kept values, each
+    // with the byte offset of its place in the expanded, swizzled 128 x 64 tile
     std::vector<RcStage> td_stage;
     std::vector<uint8_t> td_blob;
     if (tc_shape) {
       const int S = kTcRows / bh, J = kTcK / bw;
-      const int seg = bw < kTdSeg ? bw : kTdSeg;       // columns per descriptor
-      const int nseg = kTcK / seg;                      // descriptors per band of a tile
-      const size_t table_bytes = (size_t)S * nseg * sizeof(TdDesc);
       td_stage.resize((size_t)(h->tc_mtiles * h->tc_ktiles));
       uint32_t td_max = 0;
-      std::vector<TdDesc> table((size_t)S * nseg);
-      std::vector<uint16_t> tv;
+      std::vector<uint32_t> ent;
       for (int64_t t = 0; t < h->tc_mtiles && st == GRIM_OK; ++t)
         for (int64_t kt = 0; kt < h->tc_ktiles; ++kt) {
-          std::fill(table.begin(), table.end(), TdDesc{0u, 0u, 0u});
-          tv.clear();
+          ent.clear();
           for (int ts = 0; ts < S; ++ts) {
             const int64_t pos = t * S + ts;
             if (pos >= nbr) break;
@@ -454,34 +393,33 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
               if (j >= nbc) break;
               const HostBlock& hb = h->blocks[(size_t)(h->band_order[(size_t)pos] * nbc + j)];
               if (!(hb.kr && hb.kc)) continue;
-              const size_t first = tv.size();
-              for (size_t v = 0; v < (size_t)hb.kr * hb.kc; ++v) tv.push_back(bf16_bits(h->vals[(size_t)hb.val_off + v]));
-              for (int c0 = 0; c0 < bw; c0 += seg) {  // one descriptor per segment of the block
-                TdDesc& dsc = table[(size_t)ts * nseg + (size_t)(jj * bw + c0) / seg];
-                dsc.colmask = (uint32_t)((hb.colmask >> c0) & (seg == 32 ? 0xFFFFFFFFull : ((1ull << seg) - 1)));
-                dsc.rowmask = (uint16_t)hb.rowmask;
-                dsc.val_off = (uint16_t)first;
+              size_t v = (size_t)hb.val_off;
+              for (int r = 0; r < bh; ++r) {
+                if (!((hb.rowmask >> r) & 1u)) continue;
+                const uint32_t row = (uint32_t)(ts * bh + r);
+                for (int c = 0; c < bw; ++c) {
+                  if (!((hb.colmask >> c) & 1ull)) continue;
+                  const uint32_t col = (uint32_t)(jj * bw + c);
+                  ent.push_back((uint32_t)bf16_bits(h->vals[v++]) | (td_offset(row, col) << 16));
+                }
               }
             }
           }
           RcStage& se = td_stage[(size_t)(t * h->tc_ktiles + kt)];
           se.off16 = (uint32_t)(td_blob.size() / 16);
           se.bytes = 0;
-          if (tv.empty()) continue;
-          if (td_blob.size() / 16 >= (uint64_t(1) << 32) || tv.size() > 0xFFFFu) { st = GRIM_ERR_UNSUPPORTED; break; }
+          if (ent.empty()) continue;
+          if (td_blob.size() / 16 >= (uint64_t(1) << 32)) { st = GRIM_ERR_UNSUPPORTED; break; }
+          while (ent.size() % 4) ent.push_back(ent.back());  // whole 16-byte vectors; a repeated entry writes the same value again
           const size_t start = td_blob.size();
-          // one spare vector of values behind the last: the kernel's loads are predicated, the padding only keeps
-          // records 16-byte sized
-          const size_t vbytes = (tv.size() * 2 + 15) / 16 * 16;
-          td_blob.resize(start + table_bytes + vbytes, 0);
-          std::memcpy(&td_blob[start], table.data(), table_bytes);
-          std::memcpy(&td_blob[start + table_bytes], tv.data(), tv.size() * 2);
-          se.bytes = (uint32_t)(td_blob.size() - start);
+          td_blob.resize(start + ent.size() * 4);
+          std::memcpy(&td_blob[start], ent.data(), ent.size() * 4);
+          se.bytes = (uint32_t)(ent.size() * 4);
           td_max = std::max(td_max, se.bytes);
         }
       if (st != GRIM_OK) { delete h; return st; }
       h->td_max_rec = td_max;
-      h->index_bytes_td = (int64_t)td_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)td_blob.size() - (int64_t)nnz * 2 + nbr * 4;
+      h->index_bytes_tc = (int64_t)td_stage.size() * (int64_t)sizeof(RcStage) + (int64_t)td_blob.size() - (int64_t)nnz * 2 + nbr * 4;
     }
 
     // ---- upload
@@ -493,9 +431,7 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       if (e == cudaSuccess) e = upload(&h->d_rc_stage, rc_stage.data(), rc_stage.size() * sizeof(RcStage));
       if (e == cudaSuccess) e = upload(&h->d_rc_blob, rc_blob.data(), rc_blob.size());
       if (e == cudaSuccess && tc_shape) {
-        e = upload(&h->d_tc_stage, tc_stage.data(), tc_stage.size() * sizeof(RcStage));
-        if (e == cudaSuccess) e = upload(&h->d_tc_blob, tc_blob.data(), tc_blob.size());
-        if (e == cudaSuccess) e = upload(&h->d_td_stage, td_stage.data(), td_stage.size() * sizeof(RcStage));
+        e = upload(&h->d_td_stage, td_stage.data(), td_stage.size() * sizeof(RcStage));
         if (e == cudaSuccess) e = upload(&h->d_td_blob, td_blob.data(), td_blob.size());
       }
       const unsigned zero = 0;

@@ -5,8 +5,9 @@
 // order) and 256 output columns and walks K in tiles of 64.  Per K tile
 //   - one thread asks TMA for the 64 x 256 tile of X (128-byte swizzle, the layout the tensor core reads
 //     directly as the N-major operand) and for the packed records of the thread block's bands,
-//   - eight warps expand those records into a zero-filled 128 x 64 bf16 tile in shared memory, written in
-//     the K-major 128-byte-swizzled layout of the other operand,
+//   - twelve warps in three groups expand those records into a 128 x 64 bf16 tile in shared memory (the K-major
+//     128-byte-swizzled layout of the other operand): clear it, then one 2-byte store per kept value at the
+//     offset the packer stored beside it,
 //   - one thread issues four tcgen05.mma (128 x 256 x 16) that accumulate in tensor memory.
 // A ring of stages with full / ready / empty mbarriers overlaps the three.  After the last K tile the eight
 // warps read the accumulators back (tcgen05.ld), add bias, apply the activation and store Y.
@@ -20,6 +21,7 @@
 #include <algorithm>
 #include <cstring>
 
+#include "grim_device.cuh"
 #include "grim_internal.h"
 
 namespace grim {
@@ -173,8 +175,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // the X tile of a stage has landed
-  uint64_t* zeroed = full + kTcStages;                         // every worker has cleared its part of the weight tile
-  uint64_t* ready = zeroed + kTcStages;                        // the expanded weight tile of a stage is written
+  uint64_t* ready = full + kTcStages;                        // the expanded weight tile of a stage is written
   uint64_t* empty = ready + kTcStages;                         // the tensor core is done with a stage
   uint64_t* built = empty + kTcStages;                         // convolution: the X tile of a stage is written
   uint64_t* acc_done = built + kTcStages;                      // all multiplies of the tile are complete
@@ -204,7 +205,6 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
       mbar_init(full + s, CONV == 3 ? 32u : 1u);  // completed by TMA byte counts, or by the copy warp's 32 lanes
-      mbar_init(zeroed + s, kTcGroupWarps);
       mbar_init(ready + s, kTcGroupWarps);
       mbar_init(empty + s, 1);
       mbar_init(built + s, kTcBuildGroupWarps);
@@ -547,39 +547,10 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 4; break; }
       if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
-      uint4* a4 = reinterpret_cast<uint4*>(st);
-      for (int i = 0; i < p.mt * (kATileBytes / 16 / kTcGroupThreads); ++i) a4[wt + i * kTcGroupThreads] = make_uint4(0u, 0u, 0u, 0u);
-      __syncwarp();
-      if (lane == 0) mbar_arrive(zeroed + slot);
-      if (!__all_sync(0xffffffffu, mbar_wait(zeroed + slot, par, p.spin_limit, s_abort))) { failed = true, fail_site = 6; break; }
-      for (int m = 0; m < p.mt; ++m) {
-        if (s_meta[rs * 2 + m] == 0) continue;
-        uint8_t* at = st + m * kATileBytes;
-        // a thread takes kept columns of the tile and drops each column's values into the swizzled K-major tile
-        // (row stride 128 bytes, 16-byte pieces XOR-ed with the row's low 3 bits).  All loads of a column are
-        // issued before its stores: the value of row r sits popcount(mask below r) places after the first
-        const uint32_t* rec = reinterpret_cast<const uint32_t*>(recs + (size_t)(rs * p.mt + m) * p.rec_stride);
-        const int ncols = (int)rec[0];
-        const uint32_t* cw = rec + 4;
-        const uint16_t* vo = reinterpret_cast<const uint16_t*>(cw + ((ncols + 3) & ~3));
-        const uint16_t* vals = vo + ((ncols + 7) & ~7);
-        for (int c = wt; c < ncols; c += kTcGroupThreads) {
-          const uint32_t w = cw[c];
-          const uint16_t* v = vals + vo[c];
-          const uint32_t k = w & 63u;
-          const uint32_t rowbase = ((w >> 6) & 31u) * BH;
-          const uint32_t kbyte = (k & 7u) << 1, kchunk = k >> 3;
-          const uint32_t rm = w >> 16;
-          uint16_t val[BH];
-#pragma unroll
-          for (int r = 0; r < BH; ++r) val[r] = v[__popc(rm & ((1u << r) - 1u))];  // in bounds for every r (< kr + pad)
-#pragma unroll
-          for (int r = 0; r < BH; ++r) {
-            const uint32_t row = rowbase + r;
-            if ((rm >> r) & 1u) *reinterpret_cast<uint16_t*>(at + row * 128u + ((kchunk ^ (row & 7u)) << 4) + kbyte) = val[r];
-          }
-        }
-      }
+      // clear the tile, meet, then one 2-byte store per kept value at the offset stored beside it
+      for (int m = 0; m < p.mt; ++m)
+        ptx::expand_scatter<kTcGroupThreads>(smem_u32(recs + (size_t)(rs * p.mt + m) * p.rec_stride), s_meta[rs * 2 + m],
+                                             smem_u32(st + m * kATileBytes), wt, 1 + grp);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
       __syncwarp();
       if (lane == 0) {
@@ -731,7 +702,7 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 size_t tc_stage_bytes(int mt) { return (size_t)mt * kATileBytes + kBTileBytes; }
-size_t tc_rec_stride(const grim_bcr* h) { return ((size_t)h->tc_max_rec + 127) & ~size_t(127); }
+size_t tc_rec_stride(const grim_bcr* h) { return ((size_t)h->td_max_rec + 127) & ~size_t(127); }
 // extra: bytes besides the operand tiles and the records (the ring of staged input planes of the convolution)
 size_t tc_smem_need(const grim_bcr* h, int mt, int stages, int nrec, size_t extra = 0) {
   return 1024 + kTcHdrBytes + (size_t)stages * tc_stage_bytes(mt) + (size_t)nrec * mt * tc_rec_stride(h) + extra;
@@ -771,7 +742,7 @@ bool conv_staging(const SpmmArgs& a, int* seg_off, int* seg_len, size_t* seg_byt
 }  // namespace
 
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
-  if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_tc_stage || !h->d_status) return false;
+  if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_td_stage || !h->d_status) return false;
   if (a.x_dtype != GRIM_BF16 || reinterpret_cast<uintptr_t>(a.X) % 16 != 0) return false;
   if (a.conv) {
     // the tile builder covers the common same-size 3x3 convolution; other geometries use the CUDA-core kernel
@@ -780,7 +751,7 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   } else if (a.x_sq != 1 || a.y_sq != 1 || (a.x_sk * 2) % 16 != 0) {
     return false;
   }
-  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->tc_max_rec == 0) return false;
+  if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kTQ || h->td_max_rec == 0) return false;
   int st_ = 0, nr_ = 0;
   if (!tc_rings(h, 1, &st_, &nr_)) return false;
   if (h->tc_mtiles > 65535) return false;
@@ -790,7 +761,7 @@ bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
 grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
   if (!tc_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
   TcParams p;
-  p.stage = h->d_tc_stage; p.blob = h->d_tc_blob; p.band_order = h->d_band_order; p.status = h->d_status;
+  p.stage = h->d_td_stage; p.blob = h->d_td_blob; p.band_order = h->d_band_order; p.status = h->d_status;
   p.nbr = (int)h->nbr; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.nkt = (int)h->tc_ktiles;
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kTM / h->bh;

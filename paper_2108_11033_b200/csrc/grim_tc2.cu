@@ -10,11 +10,12 @@
 // 128 x 256 per expansion, a block here reads half the X bytes per flop from shared memory and expands a quarter
 // of the weight tiles per flop.
 //
-// Roles per block: warp 0 requests X tiles (TMA, 128-byte swizzle) and packed records (bulk copies); warp 1 of
-// the even block issues the multiplies, warp 1 of the odd block tells the even block when its operands are in
-// place; twelve warps in three groups expand records, a thread building 16-byte pieces of the tile in registers
-// from one block descriptor and a run of consecutive values (no clearing pass, no scattered 2-byte stores); eight
-// of them read the accumulators back at the end.  All waits are bounded; tensor memory is released on every path.
+// Roles per block: warp 0 requests X tiles (TMA, 128-byte swizzle) and packed records (bulk copies); warp 1 and
+// the last warp of the even block issue the multiplies, one accumulator each; twelve warps in three groups expand
+// records (clear the tile, then one 2-byte store per kept value at the offset stored beside it: a few instructions
+// per value, no index arithmetic); eight of them read the accumulators back at the end.  Everything the odd block
+// produces is reported straight to the even block's barriers (its TMA loads count their bytes there, its warps
+// arrive across the cluster).  All waits are bounded; tensor memory is released on every path.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -30,7 +31,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kWorkers = 12, kGroups = 3, kGroupWarps = kWorkers / kGroups, kGroupThreads = 32 * kGroupWarps;
-constexpr int kThreads = 64 + 32 * kWorkers;
+constexpr int kIssueWarp2 = 2 + kWorkers;  // second issuing warp (the last warp of the block)
+constexpr int kThreads = 64 + 32 * kWorkers + 32;
 constexpr int kRows = 128;              // rows of W per block
 constexpr int kColsPerBlock = 256;      // X columns staged per block per K tile
 constexpr int kPairCols = 512;          // output columns per pair
@@ -51,6 +53,7 @@ struct Tc2Params {
   int bh_shift, slots_per_tile, nstages, nrec;
   uint32_t rec_stride;
   unsigned spin_limit;
+  int flags;
   SpmmArgs a;
 };
 
@@ -75,6 +78,16 @@ __device__ __forceinline__ void umma2_commit_both(uint64_t* bar) {
   asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
                ::"r"(smem_u32(bar)), "h"((unsigned short)3) : "memory");
 }
+// TMA tile load issued by either block of a pair whose bytes are counted on a barrier given as a shared::cluster
+// address (here: the even block's).  No multicast: every block loads its own tile.
+__device__ __forceinline__ void tma_load_2d_pair(void* dst, const void* tensor_map, int x, int y, uint32_t bar_cluster_addr) {
+  asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+               ::"r"(smem_u32(dst)), "l"(tensor_map), "r"(x), "r"(y), "r"(bar_cluster_addr) : "memory");
+}
+// Asks TMA to bring a tile into L2 only (no shared-memory destination, nothing to wait for).
+__device__ __forceinline__ void tma_prefetch_2d(const void* tensor_map, int x, int y) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global [%0, {%1, %2}];" ::"l"(tensor_map), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
@@ -89,87 +102,19 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// One band's share of a thread's piece: block-local row `lr` of a band with descriptor (colmask of the thread's
-// segment, rowmask, first value), `kc` kept columns in the whole block, `prefix` kept columns of the block in front of
-// the piece, `sub` the piece's 8 column bits.  Returns the 8 bf16 values (zeros where nothing is kept) as 4 words.
-__device__ __forceinline__ void piece_of_row(uint32_t vals_s, uint32_t rowmask, uint32_t lr, uint32_t val_off, uint32_t kc,
-                                             uint32_t prefix, uint32_t sub, const uint32_t (&off2)[8], uint32_t (&w)[4]) {
-  const bool kept = (rowmask >> lr) & 1u;
-  const uint32_t a = __popc(rowmask & ((1u << lr) - 1u));
-  const uint32_t base = vals_s + 2u * (val_off + a * kc + prefix);
-  uint32_t v[8];
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    unsigned short h = 0;
-    // not volatile: the loads of all eight rows may be issued together; their address depends on the descriptor
-    // loads, which are ordered after the wait for the record
-    if (kept && ((sub >> e) & 1u)) asm("ld.shared.u16 %0, [%1];" : "=h"(h) : "r"(base + off2[e]));
-    v[e] = h;
-  }
-#pragma unroll
-  for (int i = 0; i < 4; ++i) w[i] = v[2 * i] | (v[2 * i + 1] << 16);
-}
-
-// Expands one packed record into the 128 x 64 bf16 weight tile at shared address a_s (K-major rows of 128 bytes,
-// 16-byte pieces XOR-ed with the row's low three bits: the tensor core's 128-byte swizzle).  Called by the
-// kGroupThreads threads of one group; thread wt owns piece j = wt & 7 (columns 8j .. 8j + 7) of rows 8 * (wt >> 3) ..
-// + 7.  rec_s = shared address of the record, or 0 when the tile keeps nothing (zeros are written).
-template <int BH, int BW>
-__device__ __forceinline__ void expand_tile(uint32_t rec_s, uint32_t a_s, int wt) {
-  constexpr int SEG = BW < kTdSeg ? BW : kTdSeg;  // columns per descriptor
-  constexpr int NSEG = kK / SEG;                  // descriptors per band
-  constexpr int BANDS = kRows / BH;
-  const uint32_t j = (uint32_t)wt & 7u, rg = (uint32_t)wt >> 3;
-  const uint32_t seg = (8u * j) / SEG, shift = (8u * j) % SEG;
-  const uint32_t vals_s = rec_s + (uint32_t)(BANDS * NSEG * sizeof(TdDesc));
-  constexpr int NB = BH == 4 ? 2 : 1;  // bands met by the thread's 8 rows
-  uint32_t colmask[NB], rowmask[NB], val_off[NB], kc[NB], prefix[NB], sub[NB];
-  uint32_t off2[NB][8];
-#pragma unroll
-  for (int b = 0; b < NB; ++b) {
-    const uint32_t band = BH == 4 ? 2u * rg + b : (BH == 8 ? rg : rg >> 1);
-    colmask[b] = rowmask[b] = val_off[b] = kc[b] = prefix[b] = 0u;
-    if (rec_s) {
-      const uint32_t d_s = rec_s + (band * NSEG + seg) * (uint32_t)sizeof(TdDesc);
-      uint32_t c0, m0;
-      asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(c0), "=r"(m0) : "r"(d_s));
-      colmask[b] = c0; rowmask[b] = m0 & 0xFFFFu; val_off[b] = m0 >> 16;
-      kc[b] = __popc(c0);
-      if (BW == 64) {  // the other half of the block: its kept columns count towards the row length (and, for the
-                       // upper half, towards the columns in front of the piece)
-        uint32_t c1;
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(c1) : "r"(d_s ^ (uint32_t)sizeof(TdDesc)));
-        kc[b] += __popc(c1);
-        if (seg & 1u) prefix[b] = __popc(c1);
-      }
-      prefix[b] += __popc(c0 & ((1u << shift) - 1u));
-    }
-    sub[b] = (colmask[b] >> shift) & 0xFFu;
-#pragma unroll
-    for (int e = 0; e < 8; ++e) off2[b][e] = 2u * __popc(sub[b] & ((1u << e) - 1u));
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int b = BH == 4 ? (i >> 2) : 0;
-    const uint32_t lr = BH == 4 ? (uint32_t)(i & 3) : (BH == 8 ? (uint32_t)i : 8u * (rg & 1u) + (uint32_t)i);
-    uint32_t w[4];
-    piece_of_row(vals_s, rowmask[b], lr, val_off[b], kc[b], prefix[b], sub[b], off2[b], w);
-    const uint32_t row = 8u * rg + (uint32_t)i;
-    sts128(a_s + row * 128u + ((j ^ (uint32_t)i) << 4), w[0], w[1], w[2], w[3]);
-  }
-}
-
-template <int BH, int BW>
 __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const Tc2Params p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes); the offset from the
   // start of the block's shared memory is the same in both blocks, which the paired multiply relies on
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem);   // this block's X tile of a stage has landed
-  uint64_t* ready = full + kMaxStages;                    // this block's expanded weight tile of a stage is written
+  // One barrier per stage IN THE EVEN BLOCK collects everything the multiplies of that stage need from both blocks:
+  // the X tiles (one arrival of the even block's copy thread that announces the bytes of both blocks; the odd
+  // block's TMA loads complete their bytes on this barrier too) and the expanded weight tiles (one arrival per
+  // expansion warp of either block, the odd block's across the cluster).  The issuing threads wait once per stage
+  // (under load every dependent shared-memory access costs a few hundred cycles) and nothing is relayed.
+  uint64_t* ready = reinterpret_cast<uint64_t*>(smem);
   uint64_t* empty = ready + kMaxStages;                   // the pair's multiplies on a stage are done (set in both blocks)
-  uint64_t* peer_ok = empty + kMaxStages;                 // even block only: the odd block's operands of a stage are in place
-  uint64_t* acc_done = peer_ok + kMaxStages;              // all multiplies are complete (set in both blocks)
+  uint64_t* acc_done = empty + kMaxStages;                // all multiplies are complete (set in both blocks)
   uint64_t* rec_full = acc_done + 1;                      // a packed record has landed
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
@@ -190,16 +135,14 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(full + s, 1);
-      mbar_init(ready + s, kGroupWarps);
-      mbar_init(empty + s, 1);
-      mbar_init(peer_ok + s, 1);
+      mbar_init(ready + s, 1 + 2 * kGroupWarps);
+      mbar_init(empty + s, 2);  // one arrival per issuing thread
     }
     for (int s = 0; s < kRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
       s_done[s] = 0;
     }
-    mbar_init(acc_done, 1);
+    mbar_init(acc_done, 2);
     *s_abort = 0;
     fence_mbar_init();
   }
@@ -233,52 +176,67 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
       for (int rk = 0; rk < nr && rk < nkt; ++rk) request_record(rk, rk);
       // 64-column boxes wholly past the last column are not requested (their part of the tile keeps whatever it
       // held; the accumulator columns computed from it are never stored)
-      int nbox = (int)((a.ncols - qb + 63) / 64);
-      nbox = nbox < 0 ? 0 : (nbox > kColsPerBlock / 64 ? kColsPerBlock / 64 : nbox);
+      auto boxes_from = [&](int64_t first) {
+        const int64_t n = (a.ncols - first + 63) / 64;
+        return (int)(n < 0 ? 0 : (n > kColsPerBlock / 64 ? kColsPerBlock / 64 : n));
+      };
+      const int nbox = boxes_from(qb);
+      const unsigned pair_bytes = (unsigned)((boxes_from(q0) + boxes_from(q0 + kColsPerBlock)) * 64 * kK * 2);
+      // the even block's barrier, as seen from this block
+      uint32_t ready0;
+      asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ready0) : "r"(smem_u32(ready)), "r"(0));
+      // X tiles are asked into L2 kPrefetch K tiles ahead of their load into shared memory: all row pairs walk K in
+      // step, so without it every load of the ring would wait for HBM, and the ring is only a few tiles deep
+      constexpr int kPrefetch = 8;
+      for (int kt = 0; kt < kPrefetch && kt < nkt; ++kt)
+        for (int i = 0; i < nbox; ++i) tma_prefetch_2d(&tmX, (int)qb + 64 * i, kt * kK);
       for (int kt = 0; kt < nkt; ++kt) {
         const int slot = kt % ns;
-        if (kt >= ns && !mbar_wait<true>(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true, fail_site = 1; break; }
+        if (kt + kPrefetch < nkt)
+          for (int i = 0; i < nbox; ++i) tma_prefetch_2d(&tmX, (int)qb + 64 * i, (kt + kPrefetch) * kK);
+        if (kt >= ns && !mbar_wait<true>(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort, 20)) { failed = true, fail_site = 1; break; }
         uint8_t* bt = stages + (size_t)slot * kStageBytes + kABytes;
-        mbar_arrive_expect_tx(full + slot, (unsigned)(nbox * 64 * kK * 2));
+        if (rank == 0) mbar_arrive_expect_tx(ready + slot, pair_bytes);
 #pragma unroll
         for (int i = 0; i < kColsPerBlock / 64; ++i)
-          if (i < nbox) tma_load_2d(bt + i * (64 * kK * 2), &tmX, (int)qb + 64 * i, kt * kK, full + slot);
+          if (i < nbox) tma_load_2d_pair(bt + i * (64 * kK * 2), &tmX, (int)qb + 64 * i, kt * kK, ready0 + (uint32_t)slot * 8u);
       }
     }
-  } else if (warp == 1) {
-    if (lane == 0 && rank == 0) {
+  } else if (warp == 1 || warp == kIssueWarp2) {
+    if (lane == 0 && rank == 0 && !((p.flags & 1) && warp != 1)) {
       // ------------------------------------------------------------------ tensor core (even block)
+      // Two issuing threads, one per accumulator.  Issuing is asynchronous but the queue is short, so a thread is
+      // held while its multiplies wait their turn; its poll of the next stage's barrier (a few hundred cycles
+      // while the tensor core reads shared memory flat out) then overlaps the other thread's multiplies.
+      // The barrier of the NEXT stage is tested (without blocking) before this stage's multiplies are issued and the
+      // answer is read after them, so that in the steady state, where operands are in place well ahead, no
+      // shared-memory round trip sits between the multiplies of consecutive stages.
+      const int acc = warp == 1 ? 0 : 1;
+      bool have = false;
       for (int kt = 0; kt < nkt; ++kt) {
         const int slot = kt % ns;
         const unsigned par = (unsigned)((kt / ns) & 1);
-        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort) ||
-            !mbar_wait<true>(peer_ok + slot, par, p.spin_limit, s_abort)) { failed = true, fail_site = 2; break; }
+        if (!have && !mbar_wait<true>(ready + slot, par, p.spin_limit << 3, s_abort, 0)) { failed = true, fail_site = 2; break; }
         asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        have = kt + 1 < nkt && mbar_test_wait_cluster(ready + (kt + 1) % ns, (unsigned)(((kt + 1) / ns) & 1));
         const uint32_t a_addr = smem_u32(stages + (size_t)slot * kStageBytes);
         const uint32_t b_addr = a_addr + kABytes;
-#pragma unroll
-        for (int acc = 0; acc < 2; ++acc) {
+        for (int ac = (p.flags & 1) ? 0 : acc; ac <= ((p.flags & 1) ? 1 : acc); ++ac) {
 #pragma unroll
           for (int s = 0; s < kK / 16; ++s) {
             // A: K-major, rows 128 bytes apart, 8-row groups 1 KiB apart; 16 K-elements = 32 bytes further on
             const uint64_t ad = smem_desc(a_addr + s * 32, 16, 1024);
             // B: N-major, 64-column panels 8 KiB apart, 8-row K groups 1 KiB apart; 16 K-rows = 2 KiB further on;
-            // accumulator `acc` takes panels 2 * acc and 2 * acc + 1 of each block
-            const uint64_t bd = smem_desc(b_addr + acc * (2 * 64 * kK * 2) + s * 2048, 64 * kK * 2, 1024);
-            umma2_bf16(tmem_base + (uint32_t)acc * 256u, ad, bd, (kt > 0 || s > 0) ? 1u : 0u);
+            // accumulator `ac` takes panels 2 * ac and 2 * ac + 1 of each block
+            const uint64_t bd = smem_desc(b_addr + ac * (2 * 64 * kK * 2) + s * 2048, 64 * kK * 2, 1024);
+            umma2_bf16(tmem_base + (uint32_t)ac * 256u, ad, bd, (kt > 0 || s > 0) ? 1u : 0u);
           }
         }
-        umma2_commit_both(empty + slot);  // arrives in both blocks when the multiplies above have read their operands
+        umma2_commit_both(empty + slot);  // arrives in both blocks when this thread's multiplies have read their operands
+        if (p.flags & 1) umma2_commit_both(empty + slot);
       }
       if (!failed) umma2_commit_both(acc_done);
-    } else if (lane == 0) {
-      // ------------------------------------------------------------------ odd block: report operands in place
-      for (int kt = 0; kt < nkt; ++kt) {
-        const int slot = kt % ns;
-        const unsigned par = (unsigned)((kt / ns) & 1);
-        if (!mbar_wait(full + slot, par, p.spin_limit, s_abort) || !mbar_wait(ready + slot, par, p.spin_limit, s_abort)) { failed = true, fail_site = 3; break; }
-        mbar_arrive_remote(peer_ok + slot, 0);
-      }
+      if (!failed && (p.flags & 1)) umma2_commit_both(acc_done);
     }
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
@@ -286,14 +244,15 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
     const int wt = tid - 64 - grp * kGroupThreads;
     for (int kt = grp; kt < nkt; kt += kGroups) {
       const int slot = kt % ns, rs = kt % nr;
-      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait<true>(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 4; break; }
+      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait<true>(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort, 32))) { failed = true, fail_site = 4; break; }
       if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
-      const uint32_t rec_s = s_meta[rs] ? smem_u32(recs + (size_t)rs * p.rec_stride) : 0u;
-      expand_tile<BH, BW>(rec_s, smem_u32(stages + (size_t)slot * kStageBytes), wt);
+      expand_scatter<kGroupThreads>(smem_u32(recs + (size_t)rs * p.rec_stride), s_meta[rs],
+                                    smem_u32(stages + (size_t)slot * kStageBytes), wt, 1 + grp);
       fence_proxy_async();  // generic-proxy writes -> visible to the tensor core
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(ready + slot);
+        if (rank == 0) mbar_arrive(ready + slot);
+        else mbar_arrive_remote(ready + slot, 0);
         // the last warp of the group to finish with the record frees its slot: it requests the record that uses
         // the slot next (every read of the old record precedes that warp's count)
         if (atomicAdd(s_done + rs, 1u) == (unsigned)kGroupWarps - 1u) {
@@ -314,48 +273,59 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
       const int acc = (warp - 2) >> 2;
       const int pos = tile * p.slots_per_tile + (trow >> p.bh_shift);
       int64_t row = -1;
-      if (has_tile && pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + (trow & (BH - 1));
+      if (has_tile && pos < p.nbr) row = (int64_t)p.band_order[pos] * p.bh + (trow & (p.bh - 1));
       const bool row_ok = row >= 0 && row < p.M;
       const float bias = (row_ok && a.bias) ? __ldg(a.bias + row) : 0.f;
+      const int row_i = row_ok ? (int)row : -1;
       for (int cb = 0; cb < 8; ++cb) {
         uint32_t v[32];
         tmem_ld32(tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(acc * 256 + cb * 32), v);
         // accumulator column c came from X column 256 * (c / 128) + 128 * acc + c % 128 of the pair's 512
         const int c = cb * 32;
         const int64_t q = q0 + 256 * (c >> 7) + 128 * acc + (c & 127);
-        if (!row_ok || q >= a.ncols) continue;
+        if (q >= a.ncols) continue;  // (uniform over the warp)
         float t[32];
 #pragma unroll
         for (int i = 0; i < 32; ++i) {
           t[i] = __uint_as_float(v[i]) + bias;
           if (a.relu) t[i] = fmaxf(t[i], 0.f);
         }
-        const bool full_chunk = q + 31 < a.ncols;
-        const int64_t off0 = row * a.y_sr + q;
-        if (a.y_dtype == GRIM_F32) {
-          float* y = static_cast<float*>(a.Y) + off0;
-          if (full_chunk && ((reinterpret_cast<uintptr_t>(y) & 15) == 0)) {
+        // Through shared memory, so that a warp instruction writes one row's 32 consecutive columns (a whole
+        // 128-byte line) instead of 16 bytes of 32 different rows: stage[lane][i] with a row pitch of 33 words is free
+        // of bank conflicts both ways.  (The stage buffers are free: all multiplies have completed.)
+        float* stg = reinterpret_cast<float*>(stages) + (warp - 2) * (33 * 32);
 #pragma unroll
-            for (int i = 0; i < 8; ++i) reinterpret_cast<float4*>(y)[i] = make_float4(t[4 * i], t[4 * i + 1], t[4 * i + 2], t[4 * i + 3]);
-          } else {
-            for (int i = 0; i < 32 && q + i < a.ncols; ++i) y[i] = t[i];
+        for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = t[i];
+        __syncwarp();
+        if (a.y_dtype == GRIM_F32) {
+          float* Y = static_cast<float*>(a.Y);
+          const bool col_ok = q + lane < a.ncols;
+#pragma unroll 8
+          for (int r = 0; r < 32; ++r) {
+            const int rr = __shfl_sync(0xffffffffu, row_i, r);
+            const float val = stg[r * 33 + lane];
+            if (rr >= 0 && col_ok) Y[(int64_t)rr * a.y_sr + q + lane] = val;
           }
         } else {
-          __nv_bfloat16* y = static_cast<__nv_bfloat16*>(a.Y) + off0;
-          if (full_chunk && ((reinterpret_cast<uintptr_t>(y) & 15) == 0)) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-              uint4 u;
-              __nv_bfloat162 b0 = __floats2bfloat162_rn(t[8 * i], t[8 * i + 1]), b1 = __floats2bfloat162_rn(t[8 * i + 2], t[8 * i + 3]);
-              __nv_bfloat162 b2 = __floats2bfloat162_rn(t[8 * i + 4], t[8 * i + 5]), b3 = __floats2bfloat162_rn(t[8 * i + 6], t[8 * i + 7]);
-              u.x = *reinterpret_cast<unsigned*>(&b0); u.y = *reinterpret_cast<unsigned*>(&b1);
-              u.z = *reinterpret_cast<unsigned*>(&b2); u.w = *reinterpret_cast<unsigned*>(&b3);
-              reinterpret_cast<uint4*>(y)[i] = u;
+          // bf16: a lane takes two neighbouring columns, a warp instruction two rows of 64 bytes each
+          __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(a.Y);
+          const int c2 = (lane & 15) * 2;
+#pragma unroll 8
+          for (int r2 = 0; r2 < 32; r2 += 2) {
+            const int r = r2 + (lane >> 4);
+            const int rr = __shfl_sync(0xffffffffu, row_i, r);
+            const float v0 = stg[r * 33 + c2], v1 = stg[r * 33 + c2 + 1];
+            if (rr < 0 || q + c2 >= a.ncols) continue;
+            __nv_bfloat16* y = Y + (int64_t)rr * a.y_sr + q + c2;
+            if (q + c2 + 1 < a.ncols && (reinterpret_cast<uintptr_t>(y) & 3) == 0) {
+              *reinterpret_cast<__nv_bfloat162*>(y) = __floats2bfloat162_rn(v0, v1);
+            } else {
+              y[0] = __float2bfloat16_rn(v0);
+              if (q + c2 + 1 < a.ncols) y[1] = __float2bfloat16_rn(v1);
             }
-          } else {
-            for (int i = 0; i < 32 && q + i < a.ncols; ++i) y[i] = __float2bfloat16_rn(t[i]);
           }
         }
+        __syncwarp();
       }
     }
   }
@@ -403,13 +373,6 @@ bool rings(const grim_bcr* h, int* stages, int* nrec) {
   return false;
 }
 
-using Tc2Kernel = void (*)(const CUtensorMap, const Tc2Params);
-Tc2Kernel kernel_for(int bh, int bw) {
-  if (bh == 4) return bw == 16 ? bcr_tc2_kernel<4, 16> : (bw == 32 ? bcr_tc2_kernel<4, 32> : bcr_tc2_kernel<4, 64>);
-  if (bh == 8) return bw == 16 ? bcr_tc2_kernel<8, 16> : (bw == 32 ? bcr_tc2_kernel<8, 32> : bcr_tc2_kernel<8, 64>);
-  return bw == 16 ? bcr_tc2_kernel<16, 16> : (bw == 32 ? bcr_tc2_kernel<16, 32> : bcr_tc2_kernel<16, 64>);
-}
-
 }  // namespace
 
 bool tc2_path_supported(const grim_bcr* h, const SpmmArgs& a) {
@@ -434,6 +397,7 @@ grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t
   rings(h, &p.nstages, &p.nrec);
   p.rec_stride = (uint32_t)rec_stride_of(h);
   p.spin_limit = 1u << 20;
+  p.flags = a.tile_n;
   p.a = a;
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
@@ -446,10 +410,9 @@ grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t
                         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return GRIM_ERR_CUDA;
   const size_t smem = smem_need(h, p.nstages, p.nrec);
-  Tc2Kernel kern = kernel_for(h->bh, h->bw);
-  // the attribute is kept by the kernel: set once per (kernel, size) and again only when a larger size is needed
-  static size_t attr_set[3][3] = {};
-  size_t& have = attr_set[p.bh_shift - 2][h->bw == 16 ? 0 : (h->bw == 32 ? 1 : 2)];
+  auto kern = bcr_tc2_kernel;
+  // the attribute is kept by the kernel: set once and again only when a larger size is needed
+  static size_t have = 0;
   if (have < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
     have = smem;
