@@ -93,7 +93,9 @@ typedef struct {
                       asynchronous copies (persistent thread blocks), 0 = the streaming variant when it fits */
   int32_t path;    /* 0 auto; 1 register-tiled CUDA-core kernel (N > 16); 2 tcgen05 tensor-core tiles (bf16
                       handles only); 3 lane-per-column kernel (N <= 16, N = 1 is the matrix-vector product);
-                      4 shared-memory slab kernel (any N; the fall-back for operands the others do not take).
+                      4 shared-memory slab kernel (any N; the fall-back for operands the others do not take);
+                      5 paired tcgen05 kernel: two thread blocks multiply 256 rows x 512 columns together
+                      (bf16 handles; the default for wide right-hand sides on matrices of 256 rows or more).
                       A path that cannot take the request returns GRIM_ERR_UNSUPPORTED. */
   int32_t reserved[6];
 } grim_tune_t;
@@ -182,6 +184,11 @@ grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, in
  * handle's dtype; out_dtype GRIM_F32 or (bf16 handles) GRIM_BF16.  Accumulation is fp32.
  */
 #define GRIM_CONV_RELU 1u
+/* Kernel choice (Section 4.5, per-kernel tuning), normally left to the library: ask for the paired tensor-core kernel
+ * (two thread blocks multiply 256 rows x 512 pixels together) or for the single-block one; a kernel that cannot take
+ * the request returns GRIM_ERR_UNSUPPORTED.  bf16 handles, 3x3 / stride 1 / pad 1 only. */
+#define GRIM_CONV_PAIRED 2u
+#define GRIM_CONV_SINGLE 4u
 typedef struct {
   int64_t N, C, H, W;
   int32_t KH, KW, stride, pad;

@@ -26,7 +26,7 @@ GRIM_ERR_INVALID_ARG, GRIM_ERR_SHAPE, GRIM_ERR_DTYPE, GRIM_ERR_NOT_BCR = 1, 2, 3
 GRIM_ERR_ALLOC, GRIM_ERR_CUDA, GRIM_ERR_UNSUPPORTED, GRIM_ERR_TIMEOUT = 5, 6, 7, 8
 GRIM_F32, GRIM_BF16 = 0, 1
 GRIM_PACK_REORDER, GRIM_PACK_HOST_ONLY = 1, 2
-GRIM_CONV_RELU = 1
+GRIM_CONV_RELU, GRIM_CONV_PAIRED, GRIM_CONV_SINGLE = 1, 2, 4
 
 EXPORTED = [
     "grim_bcr_pack", "grim_bcr_destroy", "grim_bcr_info", "grim_bcr_export", "grim_bcr_unpack_dense",
@@ -201,10 +201,10 @@ def grim_bcr_tune(h: int, X, Y, reps: int = 5, stream=None):
 
 
 def grim_bcr_conv2d(h: int, x, out, ksize: int, stride: int = 1, pad: int = 0, bias=None, relu: bool = False,
-                    stream=None):
+                    stream=None, kernel_flags: int = 0):
     assert x.is_cuda and out.is_cuda and x.is_contiguous() and out.is_contiguous() and x.dim() == 4
     d = grim_conv_desc_t(x.shape[0], x.shape[1], x.shape[2], x.shape[3], ksize, ksize, stride, pad,
-                         bias.data_ptr() if bias is not None else None, GRIM_CONV_RELU if relu else 0,
+                         bias.data_ptr() if bias is not None else None, (GRIM_CONV_RELU if relu else 0) | kernel_flags,
                          _torch_dtype_code(x), _torch_dtype_code(out))
     _check(lib.grim_bcr_conv2d(h, C.byref(d), x.data_ptr(), out.data_ptr(), _stream_ptr(stream)), "grim_bcr_conv2d")
 

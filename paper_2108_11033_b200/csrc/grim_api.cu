@@ -54,7 +54,7 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
   if (path == 4) return launch_spmm(h, a, s);
   // bf16 handles, wide right-hand sides: tensor cores.  The paired kernel when its 256 x 512 tiles still give most
   // SMs a thread block (measured: with fewer, the single-block kernel's smaller tiles win).
-  if (path == 0 && tc2_path_supported(h, a) && a.ncols >= 256 &&
+  if (path == 0 && tc2_path_supported(h, a) && a.ncols >= 256 && h->tc_mtiles >= 2 &&
       2 * ((h->tc_mtiles + 1) / 2) * ((a.ncols + 511) / 512) * 3 >= 2 * (int64_t)sm_count(h->device))
     return launch_spmm_tc2(h, a, s);
   if (path == 0 && tc_path_supported(h, a) && a.ncols >= 128) return launch_spmm_tc(h, a, s);
@@ -158,7 +158,7 @@ extern "C" grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d
   if (h->device < 0) return GRIM_ERR_INVALID_ARG;
   if (d->N <= 0 || d->C <= 0 || d->H <= 0 || d->W <= 0 || d->KH <= 0 || d->KW <= 0 || d->stride <= 0 || d->pad < 0)
     return GRIM_ERR_INVALID_ARG;
-  if (d->flags & ~GRIM_CONV_RELU) return GRIM_ERR_INVALID_ARG;
+  if (d->flags & ~(GRIM_CONV_RELU | GRIM_CONV_PAIRED | GRIM_CONV_SINGLE)) return GRIM_ERR_INVALID_ARG;
   if (d->C * (int64_t)d->KH * d->KW != h->K) return GRIM_ERR_SHAPE;
   const int64_t OH = (d->H + 2 * d->pad - d->KH) / d->stride + 1;
   const int64_t OW = (d->W + 2 * d->pad - d->KW) / d->stride + 1;
@@ -172,7 +172,16 @@ extern "C" grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d
   a.bias = d->bias_dev; a.relu = (d->flags & GRIM_CONV_RELU) ? 1 : 0;
   a.conv = 1; a.C = (int)d->C; a.H = (int)d->H; a.W = (int)d->W; a.KH = d->KH; a.KW = d->KW;
   a.stride = d->stride; a.pad = d->pad; a.OH = (int)OH; a.OW = (int)OW;
+  if (d->flags & GRIM_CONV_PAIRED) {
+    if (!tc2_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
+    return launch_spmm_tc2(h, a, (cudaStream_t)stream);
+  }
+  // bf16 handles: tensor cores; the paired kernel when its 256 x 512 tiles still give most SMs a thread block
+  if (!(d->flags & GRIM_CONV_SINGLE) && tc2_path_supported(h, a) && h->tc_mtiles >= 2 &&
+      2 * ((h->tc_mtiles + 1) / 2) * ((a.ncols + 511) / 512) * 3 >= 2 * (int64_t)sm_count(h->device))
+    return launch_spmm_tc2(h, a, (cudaStream_t)stream);
   if (tc_path_supported(h, a) && a.ncols >= 128) return launch_spmm_tc(h, a, (cudaStream_t)stream);
+  if (d->flags & GRIM_CONV_SINGLE) return GRIM_ERR_UNSUPPORTED;
   if (ffma_path_supported(h, a)) return launch_ffma(h, a, (cudaStream_t)stream);
   return launch_spmm(h, a, (cudaStream_t)stream);
 }

@@ -411,6 +411,24 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
           if (ent.empty()) continue;
           if (td_blob.size() / 16 >= (uint64_t(1) << 32)) { st = GRIM_ERR_UNSUPPORTED; break; }
           while (ent.size() % 4) ent.push_back(ent.back());  // whole 16-byte vectors; a repeated entry writes the same value again
+          // Order for conflict-free stores: a thread reads four consecutive entries and the 32 lanes of a warp store
+          // their k-th entry together, so entries 4 * lane + k of a run of 128 should fall into 32 different
+          // shared-memory banks.  Entries are dealt from per-bank piles in turn (32 consecutive picks hit 32 banks
+          // while all piles last) and pick i of a run goes to lane i % 32, store i / 32.
+          {
+            std::vector<uint32_t> pile[32];
+            for (uint32_t e : ent) pile[((e >> 16) >> 2) & 31u].push_back(e);
+            std::vector<uint32_t> dealt;
+            dealt.reserve(ent.size());
+            for (size_t r = 0; dealt.size() < ent.size(); ++r)
+              for (int b = 0; b < 32; ++b)
+                if (pile[b].size() > r) dealt.push_back(pile[b][r]);
+            for (size_t base = 0; base < ent.size(); base += 128) {
+              const size_t n = std::min<size_t>(128, ent.size() - base);  // a multiple of 4
+              const size_t lanes = n / 4;                                   // lanes that read a whole vector of this run
+              for (size_t i = 0; i < n; ++i) ent[base + 4 * (i % lanes) + i / lanes] = dealt[base + i];
+            }
+          }
           const size_t start = td_blob.size();
           td_blob.resize(start + ent.size() * 4);
           std::memcpy(&td_blob[start], ent.data(), ent.size() * 4);

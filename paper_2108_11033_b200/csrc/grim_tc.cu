@@ -22,6 +22,7 @@
 #include <cstring>
 
 #include "grim_device.cuh"
+#include "grim_im2col.cuh"
 #include "grim_internal.h"
 
 namespace grim {
@@ -66,58 +67,7 @@ struct TcParams {
   SpmmArgs a;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-__device__ __forceinline__ void cp_async8(void* dst, const void* src) {
-  asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
-  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ uint4 lds128(uint32_t saddr) {
-  uint4 v;
-  asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(saddr));
-  return v;
-}
-__device__ __forceinline__ void sts128(uint32_t saddr, const uint4& v) {
-  asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(saddr), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
-}
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
-  for (unsigned i = 0; i < limit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    __nanosleep(100);  // most warps of the block wait at any time: polling flat out takes issue slots from the others
-    if ((i & 63u) == 63u && *abort_flag) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
+using namespace ptx;
 
 // Shared-memory matrix descriptor of the tensor core: start address, leading / stride byte offsets
 // (all without their 4 low bits), descriptor version 1, 128-byte swizzle.
@@ -149,20 +99,6 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
       : "r"(taddr)
       : "memory");
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-}
-
-// Element-wise construction of one 8-pixel piece of an im2col row (pieces that cross into the next image or touch
-// the end of the tensor).  Kept out of line so that the common vector path stays short.
-__device__ __noinline__ uint4 im2col_piece_slow(const unsigned short* in1, int in_elems, int plane0, int plane1, int c_off,
-                                                int pix0, int split, int shift, uint32_t bad) {
-  uint32_t w[4] = {0u, 0u, 0u, 0u};
-#pragma unroll
-  for (int e = 0; e < 8; ++e) {
-    const int ee = (e < split ? plane0 + pix0 + e : plane1 + e - split) + c_off + shift;
-    const uint32_t val = (!((bad >> e) & 1u) && ee >= 0 && ee < in_elems) ? in1[ee] : 0u;
-    w[e >> 1] |= val << ((e & 1) * 16);
-  }
-  return make_uint4(w[0], w[1], w[2], w[3]);
 }
 
 // CONV: 0 = X is a matrix (TMA tiles); 1 = implicit im2col, the builders read the NCHW input from global memory;
@@ -201,6 +137,14 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   const int kbase = p.ksplit > 1 ? (int)blockIdx.z * p.kt_per : 0;
   const int nkt = p.ksplit > 1 ? (p.nkt - kbase < p.kt_per ? p.nkt - kbase : p.kt_per) : p.nkt;
   const int ns = p.nstages, nr = p.nrec;
+  Im2colCtx im;
+  if (CONV) {
+    im.a = &p.a; im.K = p.K; im.in_elems = (int)p.in_elems; im.seg_off = p.seg_off; im.seg_len = p.seg_len; im.nseg = p.nseg;
+    im.seg_bytes = p.seg_bytes; im.q0 = q0; im.nkt = nkt; im.kbase = kbase; im.ns = ns; im.stages = stages;
+    im.stage_bytes = stage_bytes; im.b_off = b_off; im.segs = segs; im.empty = empty; im.seg_full = full;
+    im.seg_free = seg_free; im.built = built; im.built_rank = -1; im.cluster_waits = false; im.spin_limit = p.spin_limit;
+    im.s_abort = s_abort;
+  }
 
   if (tid == 0) {
     for (int s = 0; s < kTcStages; ++s) {
@@ -266,74 +210,8 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       }
     }
     if (CONV >= 2) {
-      // Staged implicit im2col: per K tile the (at most eight) input channels it touches, and of each the stretch
-      // of the plane that the tile's 256 pixels and their 3 x 3 neighbourhoods cover, one bulk copy per channel
-      // and image.  A channel's segment holds tile pixel q at element seg_off + q; where the tile runs into the
-      // next image that image's plane follows directly (taps that would cross the boundary are masked anyway).
-      const int ohw = a.OH * a.OW;
-      const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(a.X);
-      const int64_t q_end = q0 + kTQ < a.ncols ? q0 + kTQ : a.ncols;
-      const int n0 = (int)(q0 / ohw), n1 = (int)((q_end - 1) / ohw);
-      int src_lo[3], dst_idx[3];
-      unsigned nbytes[3], per_channel = 0;
-      const int nimg = n1 - n0 + 1;  // <= 3 (checked on the host)
-      for (int i = 0; i < nimg; ++i) {
-        const int64_t img0 = (int64_t)(n0 + i) * ohw;
-        const int qa = (int)((q0 > img0 ? q0 : img0) - q0);
-        const int qb = (int)((q_end < img0 + ohw ? q_end : img0 + ohw) - q0);
-        const int pa = (int)(q0 + qa - img0), pb = pa + (qb - qa);
-        const int lo = pa - p.seg_off > 0 ? pa - p.seg_off : 0;
-        const int hi = pb + p.seg_off < ohw ? pb + p.seg_off : ohw;
-        src_lo[i] = lo;
-        dst_idx[i] = lo - pa + qa + p.seg_off;
-        nbytes[i] = (unsigned)(hi - lo) * 2u;
-        per_channel += nbytes[i];
-      }
-      // 8-byte variant: the pieces of a channel's segment this lane copies (pieces lane, lane + 32, ...): byte offset
-      // in the segment and element offset in the input relative to channel 0 of image 0; -1: none
-      constexpr int kPiecesPerLane = 8;
-      int piece_dst[kPiecesPerLane], piece_src[kPiecesPerLane];
-      if (CONV == 3) {
-#pragma unroll
-        for (int t = 0; t < kPiecesPerLane; ++t) {
-          int rem = lane + 32 * t, i = 0;
-          while (i + 1 < nimg && rem >= (int)(nbytes[i] >> 3)) { rem -= (int)(nbytes[i] >> 3); ++i; }
-          const bool ok = rem < (int)(nbytes[i] >> 3);
-          piece_dst[t] = ok ? dst_idx[i] * 2 + rem * 8 : -1;
-          piece_src[t] = ok ? (n0 + i) * a.C * ohw + src_lo[i] + rem * 4 : 0;
-        }
-      }
-      // the planes have a ring of their own, freed by the builders (long before the tensor core is done with
-      // the tile built from them), so their copies run several K tiles ahead
-      for (int kt = 0; kt < nkt; ++kt) {
-        const int ss = kt % p.nseg;
-        if (kt >= p.nseg && !__all_sync(0xffffffffu, mbar_wait(seg_free + ss, (unsigned)((kt / p.nseg - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 1; break; }
-        uint8_t* seg = segs + (size_t)ss * p.seg_bytes;
-        const int c_lo = (kbase + kt) * kTK / 9;
-        const int k_hi = (kbase + kt + 1) * kTK < p.K ? (kbase + kt + 1) * kTK - 1 : p.K - 1;
-        const int nch = k_hi / 9 - c_lo + 1;
-        if (CONV == 3) {
-          // 8-byte pieces: a lane copies the same pieces of every channel (worked out once, above); its arrival is
-          // deferred until its copies have landed
-          for (int ci = 0; ci < nch; ++ci) {
-            uint8_t* dch = seg + (size_t)ci * p.seg_len * 2;
-            const __nv_bfloat16* sch = in + (int64_t)(c_lo + ci) * ohw;
-#pragma unroll
-            for (int t = 0; t < kPiecesPerLane; ++t)
-              if (piece_dst[t] >= 0) cp_async8(dch + piece_dst[t], sch + piece_src[t]);
-          }
-          cp_async_arrive_noinc(full + ss);
-          continue;
-        }
-        if (lane == 0) mbar_arrive_expect_tx(full + ss, per_channel * (unsigned)nch);
-        __syncwarp();  // the byte count is announced before any copy can complete
-        // one copy per lane: a single thread needs several hundred cycles per copy it issues
-        for (int idx = lane; idx < nch * nimg; idx += 32) {
-          const int ci = idx / nimg, i = idx - ci * nimg;
-          bulk_load(seg + ((size_t)ci * p.seg_len + dst_idx[i]) * 2,
-                    in + ((int64_t)(n0 + i) * a.C + c_lo + ci) * ohw + src_lo[i], nbytes[i], full + ss);
-        }
-      }
+      // staged implicit im2col: the input planes of every K tile are copied into a ring of shared-memory segments
+      if (!conv_copy_planes<CONV>(im, lane)) failed = true, fail_site = 1;
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ tensor core
@@ -362,186 +240,15 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     }
   } else if (CONV && warp >= 2 + kTcWorkers) {
     // ------------------------------------------------------------------ implicit im2col (3x3, stride 1, pad 1)
-    // With W = OW the input element of tap (kh, kw) for output pixel pix is plane[pix + (kh-1)*W + (kw-1)], so a
-    // row of the X tile (one k = (c, kh, kw), 256 consecutive pixels) is a shifted copy of the input plane with
-    // zeros where the tap leaves the image.  A thread owns one 16-byte piece (8 pixels) of the row: it reads
-    // the two aligned 16-byte vectors that cover it, shifts, clears the out-of-image pixels (four byte masks,
-    // fixed per thread: pixel on the left / right / top / bottom edge) and stores the piece where the 128-byte
-    // swizzled N-major layout wants it.
     const int bgrp = (warp - 2 - kTcWorkers) / kTcBuildGroupWarps;
     const int bt = tid - kTcThreads - bgrp * (32 * kTcBuildGroupWarps);  // 0 .. 127 inside the group
-    const int cq = bt & 31;                                               // this thread's piece of the row
-    const int64_t qc = q0 + cq * 8;
-    const int ohw = a.OH * a.OW;
-    const __nv_bfloat16* in = static_cast<const __nv_bfloat16*>(a.X);
-    const int in_elems = (int)p.in_elems;  // < 2^31 (checked on the host)
-    uint32_t m_left = 0, m_right = 0, m_top = 0, m_bottom = 0, m_off = 0;  // bit e: pixel e of the piece
-    int plane0, plane1, pix0;  // element offsets of channel 0 of the image of the first / last pixel; first pixel
-    {
-      const int64_t img = qc / ohw, img1 = (qc + 7) / ohw;
-      pix0 = (int)(qc - img * ohw);
-      plane0 = (int)(img * a.C * ohw);
-      plane1 = (int)(img1 * a.C * ohw);
-#pragma unroll
-      for (int e = 0; e < 8; ++e) {
-        const int64_t q = qc + e;
-        if (q >= a.ncols) { m_off |= 1u << e; continue; }
-        const int pe = (int)(q - (q / ohw) * ohw);
-        const int oh = pe / a.OW, ow = pe - oh * a.OW;
-        if (ow == 0) m_left |= 1u << e;
-        if (ow == a.OW - 1) m_right |= 1u << e;
-        if (oh == 0) m_top |= 1u << e;
-        if (oh == a.OH - 1) m_bottom |= 1u << e;
-      }
-      if (qc >= a.ncols) { plane0 = plane1 = 0; pix0 = 0; }
-    }
-    const int split = (plane1 != plane0) ? (ohw - pix0) : 8;  // pixels of the piece that lie in the first image
-    const uint32_t panel_off = (uint32_t)(cq >> 3) * (64 * kTK * 2);  // 64-pixel panel of the tile
-    const uint32_t piece = (uint32_t)(cq & 7);
-    const uint4* in16 = reinterpret_cast<const uint4*>(in);
-    const unsigned short* in1 = reinterpret_cast<const unsigned short*>(in);
-    const int nvec = in_elems >> 3;  // complete 16-byte vectors of the tensor
-    for (int kt = bgrp; kt < nkt; kt += kTcBuildGroups) {
-      const int slot = kt % ns;
-      const int ss = CONV >= 2 ? kt % p.nseg : 0;
-      if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 3; break; }
-      // staged variant: the planes of this K tile have landed (their copies were requested several tiles ago)
-      if (CONV >= 2 && !__all_sync(0xffffffffu, mbar_wait(full + ss, (unsigned)((kt / p.nseg) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 7; break; }
-      uint8_t* bt_base = stages + (size_t)slot * stage_bytes + b_off + panel_off;
-      const uint4* seg16 = reinterpret_cast<const uint4*>(segs + (size_t)ss * p.seg_bytes);
-      if (CONV >= 2) {
-        // Staged variant.  Row kk of the tile is k = (c, kh, kw); the warp takes rows w, w + 4, ... and keeps (c, tap)
-        // up to date without dividing.  Everything that depends on the row only is the same in all lanes: the first
-        // element of the row in the channel's segment (rb), hence the shift inside a vector; a lane adds its piece.
-        const int w0 = bt >> 5;
-        const uint32_t seg_s = smem_u32(seg16), bt_s = smem_u32(bt_base);
-        const int k0 = (kbase + kt) * kTK;  // first k of this tile
-        int c_rel = (k0 + w0) / 9 - k0 / 9;   // channel relative to the first one staged for this K tile
-        int tap = (k0 + w0) % 9;
-        // rows in batches: first the shared-memory loads of the whole batch (so that their latencies overlap),
-        // then shifting, masking and storing
-        constexpr int kRows = 4;
-        for (int kk0 = w0; kk0 < kTK; kk0 += kTcBuildGroupWarps * kRows) {
-          uint4 lo[kRows], hi[kRows];
-          int rbs[kRows], taps[kRows];
-#pragma unroll
-          for (int bb = 0; bb < kRows; ++bb) {
-            const int kh = tap >= 6 ? 2 : (tap >= 3 ? 1 : 0), kw = tap - 3 * kh;
-            const int rb = c_rel * p.seg_len + p.seg_off + (kh - 1) * a.W + (kw - 1);
-            rbs[bb] = rb;
-            taps[bb] = kh * 4 + kw;
-            lo[bb] = lds128(seg_s + (uint32_t)((rb >> 3) + cq) * 16u);
-            hi[bb] = lds128(seg_s + (uint32_t)((rb >> 3) + cq + 1) * 16u);
-            tap += kTcBuildGroupWarps;
-            if (tap >= 9) { tap -= 9; ++c_rel; }
-          }
-#pragma unroll
-          for (int bb = 0; bb < kRows; ++bb) {
-            const int kk = kk0 + bb * kTcBuildGroupWarps;
-            uint4 out = make_uint4(0u, 0u, 0u, 0u);
-            if (k0 + kk < p.K) {
-              const uint4 l = lo[bb], h = hi[bb];
-              const int rb = rbs[bb], kh = taps[bb] >> 2, kw = taps[bb] & 3;
-              const int sb = (rb & 1) * 16;
-              switch ((rb >> 1) & 3) {  // 32-bit word of the vector pair at which the piece starts
-                case 0: out = make_uint4(__funnelshift_r(l.x, l.y, sb), __funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb)); break;
-                case 1: out = make_uint4(__funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb)); break;
-                case 2: out = make_uint4(__funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb)); break;
-                default: out = make_uint4(__funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb), __funnelshift_r(h.z, h.w, sb)); break;
-              }
-              const uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
-              if (bad) {  // clear the pixels whose tap lies outside the image
-                uint32_t w[4] = {out.x, out.y, out.z, out.w};
-#pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                  const uint32_t b2 = (bad >> (2 * i)) & 3u;
-                  w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
-                }
-                out = make_uint4(w[0], w[1], w[2], w[3]);
-              }
-            }
-            sts128(bt_s + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4), out);
-          }
-        }
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        __syncwarp();
-        if (lane == 0) {
-          mbar_arrive(built + slot);
-          mbar_arrive(seg_free + ss);
-        }
-        continue;
-      }
-      // The thread's 16 rows of the stage are taken in batches: first the address arithmetic and the vector loads
-      // of the whole batch (so that they are in flight together), then shifting, masking, storing.
-      constexpr int kBatch = 4;
-      for (int kk0 = bt >> 5; kk0 < kTK; kk0 += kTcBuildGroupWarps * kBatch) {
-        uint4 lo[kBatch], hi[kBatch];
-        uint32_t info[kBatch];  // bits 0-7: pixels to clear, 8-10: shift inside the vector, 12-13: 0 zeros / 1 vectors / 2 element-wise
-#pragma unroll
-        for (int bb = 0; bb < kBatch; ++bb) {
-          const int kk = kk0 + bb * kTcBuildGroupWarps;
-          const int kg = (kbase + kt) * kTK + kk;
-          lo[bb] = make_uint4(0u, 0u, 0u, 0u);
-          hi[bb] = make_uint4(0u, 0u, 0u, 0u);
-          info[bb] = 0;
-          if (kg >= p.K || m_off == 0xFFu) continue;
-          const int c = kg / 9, tap = kg - c * 9;
-          const int kh = tap / 3, kw = tap - kh * 3;
-          const uint32_t bad = m_off | (kw == 0 ? m_left : 0u) | (kw == 2 ? m_right : 0u) | (kh == 0 ? m_top : 0u) | (kh == 2 ? m_bottom : 0u);
-          if (bad == 0xFFu) continue;
-          const int e0 = plane0 + c * ohw + pix0 + (kh - 1) * a.W + (kw - 1);
-          const int v0 = e0 >> 3;  // floor: the vector that holds the first pixel (negative at the very start)
-          const int sh = e0 & 7;
-          // pieces that cross into the next image, or whose vectors are not both complete vectors of the tensor
-          // (its very end), are built element by element
-          if (split != 8 || v0 + 1 >= nvec) { info[bb] = bad | (2u << 12); continue; }
-          if (v0 >= 0) lo[bb] = __ldg(in16 + v0);
-          if (sh != 0 && v0 + 1 >= 0) hi[bb] = __ldg(in16 + v0 + 1);
-          info[bb] = bad | ((uint32_t)sh << 8) | (1u << 12);
-        }
-#pragma unroll
-        for (int bb = 0; bb < kBatch; ++bb) {
-          const int kk = kk0 + bb * kTcBuildGroupWarps;
-          const uint32_t bad = info[bb] & 0xFFu, mode = info[bb] >> 12;
-          uint4 out = make_uint4(0u, 0u, 0u, 0u);
-          if (mode == 1u) {
-            const uint4 l = lo[bb], h = hi[bb];
-            const int sb = (int)((info[bb] >> 8) & 1u) * 16;
-            switch ((info[bb] >> 9) & 3u) {  // 32-bit word of the vector pair at which the piece starts
-              case 0: out = make_uint4(__funnelshift_r(l.x, l.y, sb), __funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb)); break;
-              case 1: out = make_uint4(__funnelshift_r(l.y, l.z, sb), __funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb)); break;
-              case 2: out = make_uint4(__funnelshift_r(l.z, l.w, sb), __funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb)); break;
-              default: out = make_uint4(__funnelshift_r(l.w, h.x, sb), __funnelshift_r(h.x, h.y, sb), __funnelshift_r(h.y, h.z, sb), __funnelshift_r(h.z, h.w, sb)); break;
-            }
-            if (bad) {  // clear the pixels whose tap lies outside the image
-              uint32_t w[4] = {out.x, out.y, out.z, out.w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                const uint32_t b2 = (bad >> (2 * i)) & 3u;
-                w[i] &= ~((b2 & 1u ? 0xFFFFu : 0u) | (b2 & 2u ? 0xFFFF0000u : 0u));
-              }
-              out = make_uint4(w[0], w[1], w[2], w[3]);
-            }
-          } else if (mode == 2u) {
-            const int kg = (kbase + kt) * kTK + kk;
-            const int c = kg / 9, tap = kg - c * 9;
-            const int kh = tap / 3, kw = tap - kh * 3;
-            out = im2col_piece_slow(in1, in_elems, plane0, plane1, c * ohw, pix0, split, (kh - 1) * a.W + (kw - 1), bad);
-          }
-          *reinterpret_cast<uint4*>(bt_base + (uint32_t)kk * 128u + ((piece ^ ((uint32_t)kk & 7u)) << 4)) = out;
-        }
-      }
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(built + slot);
-    }
+    if (!conv_build_tiles<CONV>(im, bgrp, kTcBuildGroups, bt, lane, fail_site)) failed = true;
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
     const int grp = (warp - 2) / kTcGroupWarps;               // this warp's group
     const int wt = tid - 64 - grp * kTcGroupThreads;           // 0 .. kTcGroupThreads - 1 inside the group
     for (int kt = grp; kt < nkt; kt += kTcGroups) {
       const int slot = kt % ns, rs = kt % nr;
-      const unsigned par = (unsigned)((kt / ns) & 1);
       // the weight tile of the slot is free once the multiplies of its previous use are done; the record is
       // normally long there
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 4; break; }
@@ -724,21 +431,6 @@ int tc_row_tiles(const grim_bcr* h, int64_t qtiles, size_t extra = 0) {
   if (h->tc_mtiles >= 2 && qtiles * ((h->tc_mtiles + 1) / 2) >= 96 && tc_rings(h, 2, &s, &r, extra) && s >= 3) return 2;
   return 1;
 }
-// Staged implicit im2col: elements kept in front of the tile's first pixel in a channel segment (a row and a pixel,
-// rounded to vectors, plus one vector), the segment's length, and the bytes of one slot of the ring of planes (eight
-// channels at most touch a K tile of 64).  Needs planes whose size is a multiple of 4 pixels (8-byte copies; multiples of 8
-// take 16-byte-aligned bulk copies) and tiles that meet at most three images.
-constexpr int kTcSegSlots = 4;  // slots of the ring of staged planes (its barriers share the tile ring's arrays)
-bool conv_staging(const SpmmArgs& a, int* seg_off, int* seg_len, size_t* seg_bytes) {
-  const int64_t ohw = (int64_t)a.OH * a.OW;
-  if (!a.conv || ohw % 4 != 0 || ohw < kTQ / 2) return false;  // multiples of 8: bulk copies, of 4: 8-byte copies
-  if (ohw % 8 != 0 && (kTQ + 2 * ((a.W + 1 + 7) / 8 * 8 + 8)) * 2 / 8 > 8 * 32) return false;  // 8 pieces per lane at most
-  *seg_off = (a.W + 1 + 7) / 8 * 8 + 8;
-  *seg_len = kTQ + 2 * *seg_off;
-  *seg_bytes = ((size_t)8 * *seg_len * 2 + 16 + 127) / 128 * 128;
-  return true;
-}
-
 }  // namespace
 
 bool tc_path_supported(const grim_bcr* h, const SpmmArgs& a) {
@@ -768,14 +460,14 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   const int64_t qtiles_ = (a.ncols + kTQ - 1) / kTQ;
   size_t extra = 0, seg_bytes = 0;
   p.seg_off = p.seg_len = 0;
-  p.nseg = kTcSegSlots;
+  p.nseg = kImSegSlots;
   bool staged = conv_staging(a, &p.seg_off, &p.seg_len, &seg_bytes);
   const int want_mt = (a.tile_n == 1 || a.tile_n == 2) ? a.tile_n : tc_row_tiles(h, qtiles_, 0);
   if (staged) {
     // the ring of planes is as deep as shared memory allows without giving up the second row tile (which halves the
     // tile-building work per output); without room for even two slots the planes are read from global memory
     staged = false;
-    for (int n = kTcSegSlots; n >= 2 && !staged; --n) {
+    for (int n = kImSegSlots; n >= 2 && !staged; --n) {
       int s_ = 0, r_ = 0;
       if (tc_rings(h, want_mt, &s_, &r_, n * seg_bytes) && (want_mt == 1 || s_ >= 3)) { p.nseg = n; staged = true; }
     }

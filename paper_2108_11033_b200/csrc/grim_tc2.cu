@@ -23,6 +23,7 @@
 #include <cstring>
 
 #include "grim_device.cuh"
+#include "grim_im2col.cuh"
 #include "grim_internal.h"
 
 namespace grim {
@@ -33,6 +34,8 @@ using namespace ptx;
 constexpr int kWorkers = 12, kGroups = 3, kGroupWarps = kWorkers / kGroups, kGroupThreads = 32 * kGroupWarps;
 constexpr int kIssueWarp2 = 2 + kWorkers;  // second issuing warp (the last warp of the block)
 constexpr int kThreads = 64 + 32 * kWorkers + 32;
+constexpr int kBuilders = 12, kBuildGroups = 3;  // convolution only: warps that build the X tile from the NCHW input
+constexpr int kConvThreads = kThreads + 32 * kBuilders;
 constexpr int kRows = 128;              // rows of W per block
 constexpr int kColsPerBlock = 256;      // X columns staged per block per K tile
 constexpr int kPairCols = 512;          // output columns per pair
@@ -54,6 +57,8 @@ struct Tc2Params {
   uint32_t rec_stride;
   unsigned spin_limit;
   int flags;
+  int in_elems, seg_off, seg_len, nseg;  // convolution (see grim_im2col.cuh)
+  uint32_t seg_bytes;
   SpmmArgs a;
 };
 
@@ -102,7 +107,9 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-__global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const Tc2Params p) {
+// CONV: 0 = X is a matrix (TMA tiles); 1, 2, 3 = implicit im2col, the X tiles are built on chip (grim_im2col.cuh).
+template <int CONV>
+__global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const Tc2Params p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes); the offset from the
   // start of the block's shared memory is the same in both blocks, which the paired multiply relies on
@@ -120,8 +127,11 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 512);  // [record slot] bytes of the record (0: the tile is empty)
   unsigned* s_done = reinterpret_cast<unsigned*>(smem + 640);  // [record slot] warps that have finished with it
+  uint64_t* seg_full = reinterpret_cast<uint64_t*>(smem + 704);  // staged convolution: the planes of a K tile have landed
+  uint64_t* seg_free = reinterpret_cast<uint64_t*>(smem + 768);  // ... and the builders are done with them
   uint8_t* stages = smem + kHdrBytes;
   uint8_t* recs = stages + (size_t)p.nstages * kStageBytes;
+  uint8_t* segs = recs + (size_t)p.nrec * p.rec_stride;
 
   const int tid = threadIdx.x, lane = tid & 31;
   const int warp = __shfl_sync(0xffffffffu, tid >> 5, 0);
@@ -135,8 +145,11 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
 
   if (tid == 0) {
     for (int s = 0; s < kMaxStages; ++s) {
-      mbar_init(ready + s, 1 + 2 * kGroupWarps);
+      // matrix: the copy thread + the expansion warps of both blocks; convolution: expansion and builder warps
+      mbar_init(ready + s, CONV ? 2 * kGroupWarps + 2 * kImBuildWarps : 1 + 2 * kGroupWarps);
       mbar_init(empty + s, 2);  // one arrival per issuing thread
+      mbar_init(seg_full + s, CONV == 3 ? 32u : 1u);  // completed by byte counts, or by the copy warp's 32 lanes
+      mbar_init(seg_free + s, kImBuildWarps);
     }
     for (int s = 0; s < kRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
@@ -170,9 +183,22 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
 
   bool failed = false;
   int fail_site = 0;
+  Im2colCtx im;
+  if (CONV) {
+    im.a = &p.a; im.K = p.K; im.in_elems = p.in_elems; im.seg_off = p.seg_off; im.seg_len = p.seg_len; im.nseg = p.nseg;
+    im.seg_bytes = p.seg_bytes; im.q0 = qb; im.nkt = nkt; im.kbase = 0; im.ns = ns; im.stages = stages;
+    im.stage_bytes = kStageBytes; im.b_off = kABytes; im.segs = segs; im.empty = empty; im.seg_full = seg_full;
+    im.seg_free = seg_free; im.built = ready; im.built_rank = rank == 0 ? -1 : 0; im.cluster_waits = true;
+    im.spin_limit = p.spin_limit; im.s_abort = s_abort;
+  }
   if (warp == 0) {
     // ------------------------------------------------------------------ copies
-    if (lane == 0) {
+    if (CONV) {
+      if (lane == 0)
+        for (int rk = 0; rk < nr && rk < nkt; ++rk) request_record(rk, rk);
+      __syncwarp();
+      if (CONV >= 2 && !conv_copy_planes<CONV>(im, lane)) failed = true, fail_site = 1;
+    } else if (lane == 0) {
       for (int rk = 0; rk < nr && rk < nkt; ++rk) request_record(rk, rk);
       // 64-column boxes wholly past the last column are not requested (their part of the tile keeps whatever it
       // held; the accumulator columns computed from it are never stored)
@@ -238,6 +264,11 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
       if (!failed) umma2_commit_both(acc_done);
       if (!failed && (p.flags & 1)) umma2_commit_both(acc_done);
     }
+  } else if (CONV && warp > kIssueWarp2) {
+    // ------------------------------------------------------------------ implicit im2col: this block's 256 pixels
+    const int bgrp = (warp - kIssueWarp2 - 1) / kImBuildWarps;
+    const int bt = tid - kThreads - bgrp * (32 * kImBuildWarps);
+    if (!conv_build_tiles<CONV>(im, bgrp, kBuildGroups, bt, lane, fail_site)) failed = true;
   } else {
     // ------------------------------------------------------------------ expansion of the packed weights
     const int grp = (warp - 2) / kGroupWarps;
@@ -297,31 +328,43 @@ __global__ void __launch_bounds__(kThreads, 1) bcr_tc2_kernel(const __grid_const
 #pragma unroll
         for (int i = 0; i < 32; ++i) stg[lane * 33 + i] = t[i];
         __syncwarp();
+        // element (row r, column qq) of the output: matrix Y[r * y_sr + qq]; convolution (NCHW, qq = image * OH*OW +
+        // pixel): out[(image * M + r) * OH*OW + pixel] - per column a base offset, per row a stride
+        const int64_t ohw = CONV ? (int64_t)a.OH * a.OW : 1;
+        const int64_t rstride = CONV ? ohw : a.y_sr;
+        auto col_base = [&](int64_t qq) -> int64_t {
+          if (!CONV) return qq;
+          const int64_t img = qq / ohw;
+          return img * p.M * ohw + (qq - img * ohw);
+        };
         if (a.y_dtype == GRIM_F32) {
           float* Y = static_cast<float*>(a.Y);
           const bool col_ok = q + lane < a.ncols;
+          const int64_t base = col_base(q + lane);
 #pragma unroll 8
           for (int r = 0; r < 32; ++r) {
             const int rr = __shfl_sync(0xffffffffu, row_i, r);
             const float val = stg[r * 33 + lane];
-            if (rr >= 0 && col_ok) Y[(int64_t)rr * a.y_sr + q + lane] = val;
+            if (rr >= 0 && col_ok) Y[(int64_t)rr * rstride + base] = val;
           }
         } else {
           // bf16: a lane takes two neighbouring columns, a warp instruction two rows of 64 bytes each
           __nv_bfloat16* Y = static_cast<__nv_bfloat16*>(a.Y);
           const int c2 = (lane & 15) * 2;
+          const int64_t base0 = col_base(q + c2), base1 = col_base(q + c2 + 1);
+          const bool ok0 = q + c2 < a.ncols, ok1 = q + c2 + 1 < a.ncols;
 #pragma unroll 8
           for (int r2 = 0; r2 < 32; r2 += 2) {
             const int r = r2 + (lane >> 4);
             const int rr = __shfl_sync(0xffffffffu, row_i, r);
             const float v0 = stg[r * 33 + c2], v1 = stg[r * 33 + c2 + 1];
-            if (rr < 0 || q + c2 >= a.ncols) continue;
-            __nv_bfloat16* y = Y + (int64_t)rr * a.y_sr + q + c2;
-            if (q + c2 + 1 < a.ncols && (reinterpret_cast<uintptr_t>(y) & 3) == 0) {
+            if (rr < 0 || !ok0) continue;
+            __nv_bfloat16* y = Y + (int64_t)rr * rstride + base0;
+            if (ok1 && base1 == base0 + 1 && (reinterpret_cast<uintptr_t>(y) & 3) == 0) {
               *reinterpret_cast<__nv_bfloat162*>(y) = __floats2bfloat162_rn(v0, v1);
             } else {
               y[0] = __float2bfloat16_rn(v0);
-              if (q + c2 + 1 < a.ncols) y[1] = __float2bfloat16_rn(v1);
+              if (ok1) Y[(int64_t)rr * rstride + base1] = __float2bfloat16_rn(v1);
             }
           }
         }
@@ -361,15 +404,16 @@ EncodeTiledFn encode_tiled_fn() {
 }
 
 size_t rec_stride_of(const grim_bcr* h) { return ((size_t)h->td_max_rec + 127) & ~size_t(127); }
-size_t smem_need(const grim_bcr* h, int stages, int nrec) {
-  return 1024 + kHdrBytes + (size_t)stages * kStageBytes + (size_t)nrec * rec_stride_of(h);
+// extra: bytes besides the operand tiles and the records (the ring of staged input planes of the convolution)
+size_t smem_need(const grim_bcr* h, int stages, int nrec, size_t extra = 0) {
+  return 1024 + kHdrBytes + (size_t)stages * kStageBytes + (size_t)nrec * rec_stride_of(h) + extra;
 }
 // As many tile slots as fit (at least as many as expansion groups, so that no wait is ever more than one barrier
 // phase behind), then as many record slots as are left, at least as many as tile slots.
-bool rings(const grim_bcr* h, int* stages, int* nrec) {
+bool rings(const grim_bcr* h, int* stages, int* nrec, size_t extra = 0) {
   for (int s = kMaxStages; s >= kGroups; --s)
     for (int r = kRecSlots; r >= s; --r)
-      if (smem_need(h, s, r) <= 227 * 1024) { *stages = s; *nrec = r; return true; }
+      if (smem_need(h, s, r, extra) <= 227 * 1024) { *stages = s; *nrec = r; return true; }
   return false;
 }
 
@@ -377,8 +421,12 @@ bool rings(const grim_bcr* h, int* stages, int* nrec) {
 
 bool tc2_path_supported(const grim_bcr* h, const SpmmArgs& a) {
   if (h->device < 0 || h->dtype != GRIM_BF16 || !h->d_td_stage || !h->d_status || h->td_max_rec == 0) return false;
-  if (a.conv || a.x_dtype != GRIM_BF16 || reinterpret_cast<uintptr_t>(a.X) % 16 != 0) return false;
-  if (a.x_sq != 1 || a.y_sq != 1 || (a.x_sk * 2) % 16 != 0) return false;
+  if (a.x_dtype != GRIM_BF16 || reinterpret_cast<uintptr_t>(a.X) % 16 != 0) return false;
+  if (a.conv) {
+    if (!conv_tiles_supported(a)) return false;
+  } else if (a.x_sq != 1 || a.y_sq != 1 || (a.x_sk * 2) % 16 != 0) {
+    return false;
+  }
   if (a.ncols <= 0 || a.ncols > (int64_t(1) << 31) - kPairCols) return false;
   if ((a.ncols + kPairCols - 1) / kPairCols > 65535) return false;
   int s = 0, r = 0;
@@ -394,32 +442,52 @@ grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t
   p.mtiles = (int)h->tc_mtiles;
   p.bh_shift = h->bh == 4 ? 2 : (h->bh == 8 ? 3 : 4);
   p.slots_per_tile = kRows / h->bh;
-  rings(h, &p.nstages, &p.nrec);
   p.rec_stride = (uint32_t)rec_stride_of(h);
   p.spin_limit = 1u << 20;
-  p.flags = a.tile_n;
+  p.flags = a.conv ? 0 : a.tile_n;
   p.a = a;
+  // convolution: stage the input planes in shared memory when their size allows and a ring of at least two
+  // segments fits beside three tile slots; otherwise the builders read them from global memory
+  size_t seg_bytes = 0, extra = 0;
+  int mode = 0;
+  p.in_elems = 0; p.seg_off = p.seg_len = 0; p.nseg = kImSegSlots; p.seg_bytes = 0;
+  if (a.conv) {
+    mode = 1;
+    p.in_elems = (int)(a.ncols / ((int64_t)a.OH * a.OW) * a.C * a.H * a.W);
+    if (conv_staging(a, &p.seg_off, &p.seg_len, &seg_bytes)) {
+      for (int n = kImSegSlots; n >= 2 && mode == 1; --n) {
+        int s_ = 0, r_ = 0;
+        if (rings(h, &s_, &r_, n * seg_bytes)) { p.nseg = n; mode = ((int64_t)a.OH * a.OW) % 8 == 0 ? 2 : 3; }
+      }
+    }
+    if (mode > 1) { extra = p.nseg * seg_bytes; p.seg_bytes = (uint32_t)seg_bytes; }
+  }
+  if (!rings(h, &p.nstages, &p.nrec, extra)) return GRIM_ERR_UNSUPPORTED;
   CUtensorMap tm;
   memset(&tm, 0, sizeof(tm));
-  const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
-  const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * 2)};
-  const cuuint32_t box[2] = {64, (cuuint32_t)kK};
-  const cuuint32_t estr[2] = {1, 1};
-  if (encode_tiled_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.X), dims, strides, box, estr,
-                        CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
-                        CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return GRIM_ERR_CUDA;
-  const size_t smem = smem_need(h, p.nstages, p.nrec);
-  auto kern = bcr_tc2_kernel;
+  if (!a.conv) {
+    const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
+    const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * 2)};
+    const cuuint32_t box[2] = {64, (cuuint32_t)kK};
+    const cuuint32_t estr[2] = {1, 1};
+    if (encode_tiled_fn()(&tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(a.X), dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+      return GRIM_ERR_CUDA;
+  }
+  const size_t smem = smem_need(h, p.nstages, p.nrec, extra);
+  using Kern = void (*)(const CUtensorMap, const Tc2Params);
+  const Kern kerns[4] = {bcr_tc2_kernel<0>, bcr_tc2_kernel<1>, bcr_tc2_kernel<2>, bcr_tc2_kernel<3>};
+  Kern kern = kerns[mode];
   // the attribute is kept by the kernel: set once and again only when a larger size is needed
-  static size_t have = 0;
-  if (have < smem) {
+  static size_t have[4] = {0, 0, 0, 0};
+  if (have[mode] < smem) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
-    have = smem;
+    have[mode] = smem;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * ((h->tc_mtiles + 1) / 2)), (unsigned)((a.ncols + kPairCols - 1) / kPairCols), 1);
-  cfg.blockDim = dim3(kThreads);
+  cfg.blockDim = dim3(a.conv ? kConvThreads : kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
   cudaLaunchAttribute attr[1];

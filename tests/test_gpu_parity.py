@@ -293,7 +293,7 @@ def conv_col_norms(x, ksize, stride, pad):
     return torch.sqrt(torch.nn.functional.conv2d(xx, ones, stride=stride, padding=pad)).numpy()  # N,1,OH,OW
 
 
-def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=False):
+def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=False, kernel_flags=0):
     W, mask, bias = L["W"], L["mask"], L["bias"]
     dt = B.GRIM_BF16 if bf16 else B.GRIM_F32
     x = gen.bf16_representable(batch_x) if bf16 else batch_x
@@ -305,8 +305,9 @@ def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=F
         OW = (Wd + 2 * pad - ksize) // stride + 1
         out = torch.full((Nb, W.shape[0], OH, OW), float("nan"), device="cuda",
                          dtype=torch.bfloat16 if out_bf16 else torch.float32)
-        B.grim_bcr_conv2d(h, xd, out, ksize, stride, pad, bias=to_dev(bias), relu=relu)
+        B.grim_bcr_conv2d(h, xd, out, ksize, stride, pad, bias=to_dev(bias), relu=relu, kernel_flags=kernel_flags)
         torch.cuda.synchronize()
+        assert B.grim_bcr_status(h) == B.GRIM_OK
         got = out.float().cpu().numpy().astype(np.float64)
         want = orc.conv2d(W, mask, x, bias, ksize=ksize, stride=stride, pad=pad, relu=relu, dtype=dt)
         Wm = orc.masked_weight(W, mask, dt)
@@ -422,6 +423,25 @@ def test_conv_bf16_staged_planes(B, shape, bh):
     L = dict(W=W, mask=mask, bias=bias, bh=bh, bw=bw)
     check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True)
     check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True)
+
+
+@pytest.mark.parametrize("shape", [(12, 12, 7), (8, 16, 9), (16, 10, 5), (24, 16, 3), (10, 14, 5), (14, 14, 3), (7, 9, 4), (15, 15, 5)])
+@pytest.mark.parametrize("bh,cout", [(4, 136), (8, 300), (16, 520)])
+def test_conv_bf16_paired_kernel(B, shape, bh, cout):
+    """The paired tensor-core convolution asked for by name: planes staged by bulk copies (multiples of 8 pixels), by
+    8-byte copies (multiples of 4) and read from global memory (others); tiles that meet two or three images, pixel
+    counts that leave the odd block of a pair with a partial or an empty tile, one to five row tiles (odd counts give
+    the last pair an empty partner), fp32 and bf16 outputs."""
+    H, Wd, batch = shape
+    C, bw = 20, 32
+    rng_seed = 400 + H + Wd + bh
+    W = gen.dense_weight(cout, C * 9, seed=rng_seed)
+    mask = gen.bcr_mask(cout, C * 9, bh, bw, compression=4, dist="uniform", seed=rng_seed + 1)
+    bias = gen.normal_f32((cout,), 0.1, rng_seed + 2, 0)
+    x = np.maximum(gen.normal_f32((batch, C, H, Wd), 1.0, rng_seed + 3, 0), 0)
+    L = dict(W=W, mask=mask, bias=bias, bh=bh, bw=bw)
+    check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, kernel_flags=B.GRIM_CONV_PAIRED)
+    check_conv(B, L, x, ksize=3, stride=1, pad=1, bf16=True, relu=False, out_bf16=True, kernel_flags=B.GRIM_CONV_PAIRED)
 
 
 @pytest.mark.parametrize("y_bf16", [False, True])
