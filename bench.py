@@ -276,7 +276,8 @@ class SpmmWorkload:
         self.B, self.torch = B, torch
         s = self.s
         dt = B.GRIM_BF16 if self.bf16 else B.GRIM_F32
-        self.h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, B.GRIM_PACK_REORDER)
+        self.pack_flags = B.GRIM_PACK_REORDER | (B.GRIM_PACK_NARROW_ONLY if self.N <= 16 else B.GRIM_PACK_WIDE_ONLY)
+        self.h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, self.pack_flags)
         tdt = torch.bfloat16 if self.bf16 else torch.float32
         self.x_host = torch.from_numpy(s["X"]).to(tdt).pin_memory()
         self.x = self.x_host.cuda()
@@ -298,7 +299,7 @@ class SpmmWorkload:
         # operand sets the timed steps rotate through (own copy of the packed matrix, of X and of Y each)
         self.sets = [(self.h, self.x, self.y)]
         for _ in range(rotation_sets(self.kernel_bytes) - 1):
-            h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, B.GRIM_PACK_REORDER)
+            h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, self.pack_flags)
             self.sets.append((h, self.x.clone(), torch.empty_like(self.y)))
         self.rotating = len(self.sets) > 1
         self.per_step_events = True
@@ -368,7 +369,9 @@ class ConvWorkload:
         L = self.L
         dt = B.GRIM_BF16 if self.bf16 else B.GRIM_F32
         tdt = torch.bfloat16 if self.bf16 else torch.float32
-        self.h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, dt, B.GRIM_PACK_REORDER)
+        self.h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, dt, B.GRIM_PACK_REORDER | B.GRIM_PACK_WIDE_ONLY)
+        if self.bf16:
+            B.grim_bcr_reserve(self.h, self.batch * 28 * 28)
         self.x_host = torch.from_numpy(L["x"]).to(tdt).pin_memory()
         self.x = self.x_host.cuda()
         self.bias = torch.from_numpy(L["bias"]).cuda()
@@ -386,7 +389,9 @@ class ConvWorkload:
         self._ev = (torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
         self.sets = [(self.h, self.x, self.y)]
         for _ in range(rotation_sets(self.kernel_bytes) - 1):
-            h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, dt, B.GRIM_PACK_REORDER)
+            h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, dt, B.GRIM_PACK_REORDER | B.GRIM_PACK_WIDE_ONLY)
+            if self.bf16:
+                B.grim_bcr_reserve(h, self.batch * 28 * 28)
             self.sets.append((h, self.x.clone(), torch.empty_like(self.y)))
         self.rotating = len(self.sets) > 1
         self.per_step_events = True
@@ -459,7 +464,9 @@ class VggWorkload:
         self.x = self.x_host.cuda()
         cur_hw = self.image
         for L in net["layers"]:
-            self.h.append(B.grim_bcr_pack(L["W"], L["mask"], net["bh"], net["bw"], B.GRIM_BF16, B.GRIM_PACK_REORDER))
+            self.h.append(B.grim_bcr_pack(L["W"], L["mask"], net["bh"], net["bw"], B.GRIM_BF16,
+                                          B.GRIM_PACK_REORDER | B.GRIM_PACK_WIDE_ONLY))
+            B.grim_bcr_reserve(self.h[-1], self.batch * cur_hw * cur_hw)
             self.bias.append(torch.from_numpy(L["bias"]).cuda())
             out = torch.empty(self.batch, L["cout"], cur_hw, cur_hw, device="cuda", dtype=torch.bfloat16)
             pooled = None

@@ -64,6 +64,11 @@ typedef struct {
 /* grim_bcr_pack flags */
 #define GRIM_PACK_REORDER 1u   /* schedule row bands by decreasing work; export the row permutation */
 #define GRIM_PACK_HOST_ONLY 2u /* build host-side data only (no CUDA call); compute calls then fail */
+/* A handle normally uploads one private device layout per kernel regime (3 - 4 x the compact size in device memory).
+ * A handle that will only see narrow right-hand sides (N <= 16, GRU matrices) or only wide ones can say so and keep
+ * just that regime's layouts; a multiply outside the regime then returns GRIM_ERR_UNSUPPORTED. */
+#define GRIM_PACK_NARROW_ONLY 4u
+#define GRIM_PACK_WIDE_ONLY 8u
 
 typedef struct {
   int64_t M, K;
@@ -148,13 +153,19 @@ grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);
  * after fp32 accumulation).  Y is fully overwritten (all M rows, beta = 0): rows kept by no
  * block are written as +0.  N = 1 selects the matrix-vector kernel.  X and Y must not overlap.
  * Shape mismatch -> GRIM_ERR_SHAPE, dtype mismatch -> GRIM_ERR_DTYPE, both before any launch.
- * Asynchronous on `stream`.  One exception: a bf16 handle whose tensor-core multiply has few output
- * tiles and a long K is split over K through an fp32 scratch of M x N floats that the handle owns;
- * the call that first needs it (or needs a larger one) allocates it with cudaMalloc, which
- * synchronises - make that call once before capturing a stream or entering a timed region.  The
- * same holds for grim_bcr_conv2d.  A handle is used on one stream at a time.
+ * Asynchronous on `stream`; never allocates.  A handle is used on one stream at a time.
+ * Without an explicit choice (grim_bcr_spmm_ex) the kernel and tile shape are the ones grim_bcr_tune found for
+ * this handle and this kind of request (same power-of-two bucket of N, same dtypes), else a static default.
  */
 grim_status_t grim_bcr_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, grim_stream_t stream);
+
+/* Workspace of the split tensor-core multiply (Section 4.5: the tile plan depends on the problem; bf16 handles with
+ * few output tiles and a long K - small batches of the deeper convolution layers - are split over K through an fp32
+ * scratch of M x N floats).  Compute calls never allocate: grim_bcr_reserve allocates that scratch for right-hand
+ * sides of up to max_ncols columns (for a convolution: images x OH x OW), once, at set-up time; it synchronises the
+ * device.  Without it (or beyond max_ncols) such multiplies simply run unsplit, slower.  max_ncols = 0 frees it.
+ * More than 2^30 bytes -> GRIM_ERR_UNSUPPORTED. */
+grim_status_t grim_bcr_reserve(grim_bcr_t h, int64_t max_ncols);
 
 /* The multiply kernels bound every device-side wait (on a shared-memory barrier that an asynchronous copy
  * completes).  If one ever gives up, the kernel leaves, Y is invalid and an error word in the handle is set.
@@ -168,7 +179,9 @@ grim_status_t grim_bcr_spmm_ex(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y,
 
 /* Times the candidate tile shapes for (handle, X/Y shapes and dtypes) on `stream` (synchronises)
  * and returns the fastest in *best (Section 4.5: per-kernel tuning of tile shape; the paper's
- * genetic search is replaced by a small fixed candidate set).  Y is overwritten. */
+ * genetic search is replaced by a small fixed candidate set).  Y is overwritten.  The answer is also
+ * stored in the handle: later grim_bcr_spmm calls with N in the same power-of-two bucket and the same
+ * dtypes use it. */
 grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, int reps, grim_tune_t* best,
                             float* best_ms, grim_stream_t stream);
 

@@ -25,7 +25,7 @@ GRIM_OK = 0
 GRIM_ERR_INVALID_ARG, GRIM_ERR_SHAPE, GRIM_ERR_DTYPE, GRIM_ERR_NOT_BCR = 1, 2, 3, 4
 GRIM_ERR_ALLOC, GRIM_ERR_CUDA, GRIM_ERR_UNSUPPORTED, GRIM_ERR_TIMEOUT = 5, 6, 7, 8
 GRIM_F32, GRIM_BF16 = 0, 1
-GRIM_PACK_REORDER, GRIM_PACK_HOST_ONLY = 1, 2
+GRIM_PACK_REORDER, GRIM_PACK_HOST_ONLY, GRIM_PACK_NARROW_ONLY, GRIM_PACK_WIDE_ONLY = 1, 2, 4, 8
 GRIM_CONV_RELU, GRIM_CONV_PAIRED, GRIM_CONV_SINGLE = 1, 2, 4
 
 EXPORTED = [
@@ -33,7 +33,7 @@ EXPORTED = [
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
-    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak",
+    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve",
 ]
 
 
@@ -70,6 +70,7 @@ lib.grim_bcr_pack.argtypes = [_vp, C.c_int64, _vp, C.c_int64, C.c_int64, C.c_int
                               C.c_uint32, C.POINTER(_vp)]
 lib.grim_bcr_destroy.argtypes = [_vp]
 lib.grim_bcr_status.argtypes = [_vp]
+lib.grim_bcr_reserve.argtypes = [_vp, C.c_int64]
 lib.grim_bcr_info.argtypes = [_vp, C.POINTER(grim_bcr_info_t)]
 lib.grim_bcr_export.argtypes = [_vp, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.grim_bcr_unpack_dense.argtypes = [_vp, _vp, C.c_int64]
@@ -179,6 +180,10 @@ def grim_bcr_unpack_dense(h: int) -> np.ndarray:
 def grim_bcr_spmm(h: int, X, Y, stream=None):
     mx, my = _mat(X), _mat(Y)
     _check(lib.grim_bcr_spmm(h, C.byref(mx), C.byref(my), _stream_ptr(stream)), "grim_bcr_spmm")
+
+
+def grim_bcr_reserve(h: int, max_ncols: int):
+    _check(lib.grim_bcr_reserve(h, int(max_ncols)), "grim_bcr_reserve")
 
 
 def grim_bcr_status(h: int) -> int:

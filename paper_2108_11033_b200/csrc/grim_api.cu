@@ -28,9 +28,21 @@ SpmmArgs mat_args(const grim_mat_t* X, const grim_mat_t* Y) {
   return a;
 }
 
+// Slot of the tune cache for a request: right-hand sides whose widths fall into the same power-of-two bucket share
+// an answer (tile choices change with the order of magnitude of N, not with N).
+grim_tune_t* tuned_slot(grim_bcr_t h, const grim_mat_t* X, const grim_mat_t* Y) {
+  int b = 0;
+  while (b < 31 && (int64_t(1) << b) < X->cols) ++b;
+  return &h->tuned[b][X->dtype == GRIM_BF16 ? 1 : 0][Y->dtype == GRIM_BF16 ? 1 : 0];
+}
+
 grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const grim_tune_t* tune, cudaStream_t s) {
   grim_status_t st = check_mats(h, X, Y);
   if (st != GRIM_OK) return st;
+  if (!tune) {  // no explicit choice: an earlier grim_bcr_tune for this kind of request decides
+    const grim_tune_t* t = tuned_slot(h, X, Y);
+    if (t->path != 0) tune = t;
+  }
   int path = tune ? tune->path : 0;
   if (path < 0 || path > 5) return GRIM_ERR_INVALID_ARG;
   if (path == 0 && tune && tune->tile_n >= 16) path = 4;  // a column-tile width only means something to the slab kernel
@@ -123,7 +135,7 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   float best_t = -1.f;
   grim_tune_t cand_best{};
   // candidates: (path, tile_n); a candidate that cannot take the request is skipped
-  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
+  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {5, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
   for (const auto& cd : cand) {
     grim_tune_t c{};
     c.path = cd[0];
@@ -149,6 +161,23 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   if (st != GRIM_OK) return st;
   *best = cand_best;
   if (best_ms) *best_ms = best_t;
+  *tuned_slot(h, X, Y) = cand_best;  // grim_bcr_spmm takes this choice for requests of the same kind from now on
+  return GRIM_OK;
+}
+
+extern "C" grim_status_t grim_bcr_reserve(grim_bcr_t h, int64_t max_ncols) {
+  if (!h || max_ncols < 0) return GRIM_ERR_INVALID_ARG;
+  if (h->device < 0) return GRIM_ERR_INVALID_ARG;
+  const size_t need = (size_t)h->M * (size_t)max_ncols * 4;
+  if (need > ((size_t)1 << 30)) return GRIM_ERR_UNSUPPORTED;  // the split multiply is only used for small outputs
+  if (h->tc_acc_bytes >= need && need > 0) return GRIM_OK;
+  if (cudaDeviceSynchronize() != cudaSuccess) return GRIM_ERR_CUDA;  // a launch in flight may still use the old scratch
+  cudaFree(h->d_tc_acc);
+  h->d_tc_acc = nullptr;
+  h->tc_acc_bytes = 0;
+  if (need == 0) return GRIM_OK;
+  if (cudaMalloc((void**)&h->d_tc_acc, need) != cudaSuccess) { cudaGetLastError(); return GRIM_ERR_ALLOC; }
+  h->tc_acc_bytes = need;
   return GRIM_OK;
 }
 

@@ -499,7 +499,7 @@ cudaError_t zero_output(const SpmmArgs& a, int64_t M, cudaStream_t s) {
 template <int BH, int BPW, typename XT, int MODE>
 cudaError_t launch_variant(const CUtensorMap& tm, const FParams& p, size_t smem, dim3 grid, cudaStream_t s) {
   auto kern = bcr_ffma_kernel<BH, BPW, XT, MODE>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
   if (e != cudaSuccess) return e;
   kern<<<grid, kFThreads, smem, s>>>(tm, p);
   return cudaGetLastError();

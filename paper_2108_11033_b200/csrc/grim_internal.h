@@ -140,8 +140,10 @@ struct grim_bcr {
   uint32_t td_max_rec = 0;
   grim::RcStage* d_td_stage = nullptr;
   uint8_t* d_td_blob = nullptr;
-  float* d_tc_acc = nullptr;  // fp32 scratch of the split tensor-core multiply (M x N), grown on first use
+  float* d_tc_acc = nullptr;  // fp32 scratch of the split tensor-core multiply (M x N); grim_bcr_reserve allocates it
   size_t tc_acc_bytes = 0;
+  // answers of grim_bcr_tune, one per (log2 bucket of N, X dtype, Y dtype); path 0 = not tuned
+  grim_tune_t tuned[32][2][2] = {};
   unsigned* d_status = nullptr;  // error word written by kernels whose bounded waits ran out
   grim::StageEntry* d_stage = nullptr;
   uint8_t* d_blob = nullptr;
@@ -194,5 +196,8 @@ bool tc2_path_supported(const grim_bcr* h, const SpmmArgs& a);
 void count_launch(int n = 1);
 // streaming multiprocessors of a device (read once per device through the runtime)
 int sm_count(int device);
+// raises a kernel's dynamic shared-memory limit to `bytes` unless an earlier call already did (the attribute is
+// kept by the kernel, so it is set once per kernel and size, not per launch)
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
 
 }  // namespace grim

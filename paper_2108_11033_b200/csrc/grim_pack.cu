@@ -67,7 +67,8 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
   if (!W || !mask || !out) return GRIM_ERR_INVALID_ARG;
   if (M <= 0 || K <= 0 || bh <= 0 || bw <= 0 || ldw < K || ldm < K) return GRIM_ERR_INVALID_ARG;
   if (vdt != GRIM_F32 && vdt != GRIM_BF16) return GRIM_ERR_DTYPE;
-  if (flags & ~(GRIM_PACK_REORDER | GRIM_PACK_HOST_ONLY)) return GRIM_ERR_INVALID_ARG;
+  if (flags & ~(GRIM_PACK_REORDER | GRIM_PACK_HOST_ONLY | GRIM_PACK_NARROW_ONLY | GRIM_PACK_WIDE_ONLY)) return GRIM_ERR_INVALID_ARG;
+  if ((flags & GRIM_PACK_NARROW_ONLY) && (flags & GRIM_PACK_WIDE_ONLY)) return GRIM_ERR_INVALID_ARG;
   if (bh > 16 || bw > 64 || M >= (int64_t(1) << 31) || K >= (int64_t(1) << 31)) return GRIM_ERR_UNSUPPORTED;
 
   grim_bcr* h = new (std::nothrow) grim_bcr();
@@ -443,18 +444,20 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
     // ---- upload
     if (!(flags & GRIM_PACK_HOST_ONLY)) {
       cudaError_t e = cudaGetDevice(&h->device);
-      if (e == cudaSuccess) e = upload(&h->d_stage, stage.data(), stage.size() * sizeof(StageEntry));
-      if (e == cudaSuccess) e = upload(&h->d_blob, blob.data(), blob.size());
+      // a handle packed for one regime keeps only that regime's layouts in device memory
+      const bool wide = !(flags & GRIM_PACK_NARROW_ONLY), narrow = !(flags & GRIM_PACK_WIDE_ONLY);
+      if (e == cudaSuccess && wide) e = upload(&h->d_stage, stage.data(), stage.size() * sizeof(StageEntry));
+      if (e == cudaSuccess && wide) e = upload(&h->d_blob, blob.data(), blob.size());
       if (e == cudaSuccess) e = upload(&h->d_band_order, h->band_order.data(), h->band_order.size() * 4);
-      if (e == cudaSuccess) e = upload(&h->d_rc_stage, rc_stage.data(), rc_stage.size() * sizeof(RcStage));
-      if (e == cudaSuccess) e = upload(&h->d_rc_blob, rc_blob.data(), rc_blob.size());
-      if (e == cudaSuccess && tc_shape) {
+      if (e == cudaSuccess && wide) e = upload(&h->d_rc_stage, rc_stage.data(), rc_stage.size() * sizeof(RcStage));
+      if (e == cudaSuccess && wide) e = upload(&h->d_rc_blob, rc_blob.data(), rc_blob.size());
+      if (e == cudaSuccess && tc_shape && wide) {
         e = upload(&h->d_td_stage, td_stage.data(), td_stage.size() * sizeof(RcStage));
         if (e == cudaSuccess) e = upload(&h->d_td_blob, td_blob.data(), td_blob.size());
       }
       const unsigned zero = 0;
       if (e == cudaSuccess) e = upload(&h->d_status, &zero, 4);
-      if (e == cudaSuccess && h->gemv_ok) {
+      if (e == cudaSuccess && h->gemv_ok && narrow) {
         e = upload(&h->d_gemv_band_ptr, band_ptr.data(), band_ptr.size() * 4);
         if (e == cudaSuccess) e = upload(&h->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkDesc));
         if (e == cudaSuccess) e = upload(&h->d_colwords, colwords.data(), colwords.size() * 4);

@@ -17,12 +17,26 @@
 #include <atomic>
 
 #include "grim_device.cuh"
+#include <mutex>
+#include <unordered_map>
+
 #include "grim_internal.h"
 
 namespace grim {
 
 static std::atomic<long long> g_launches{0};
 void count_launch(int n) { g_launches.fetch_add(n, std::memory_order_relaxed); }
+
+cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes) {
+  static std::mutex mu;
+  static std::unordered_map<const void*, size_t> have;
+  std::lock_guard<std::mutex> lock(mu);
+  size_t& h = have[kernel];
+  if (h >= bytes) return cudaSuccess;
+  const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+  if (e == cudaSuccess) h = bytes;
+  return e;
+}
 
 int sm_count(int device) {
   constexpr int kFallback = 148;  // B200; used only when the attribute cannot be read
@@ -485,7 +499,7 @@ cudaError_t launch_one(const KParams& p, cudaStream_t s) {
   const size_t smem = (size_t)2 * p.bw * TN * 4 + (size_t)2 * q.blob_stride;
   auto kern = bcr_spmm_kernel<BH, BPW, NQL, VT, CONV>;
   if (smem > 48 * 1024) {
-    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
     if (e != cudaSuccess) return e;
   }
   const int64_t ntiles = (p.a.ncols + TN - 1) / TN;
@@ -525,6 +539,7 @@ int default_tile_n(int64_t ncols) {
 
 grim_status_t launch_spmm(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) {
   if (h->device < 0) return GRIM_ERR_INVALID_ARG;
+  if (!h->d_stage) return GRIM_ERR_UNSUPPORTED;  // packed for narrow right-hand sides only
   KParams p;
   p.stage = h->d_stage; p.blob = h->d_blob; p.band_order = h->d_band_order;
   p.nbr = (int)h->nbr; p.nbc = (int)h->nbc; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.bw = h->bw; p.G = h->G;
@@ -564,7 +579,7 @@ cudaError_t launch_skinny_bh(const SkinnyParams& p, int BHc, int nq, dim3 grid, 
 
 grim_status_t launch_skinny(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
                             int64_t ldy, cudaStream_t s) {
-  if (h->device < 0 || !h->gemv_ok || N < 1 || N > kSkinnyMaxN) return GRIM_ERR_UNSUPPORTED;
+  if (h->device < 0 || !h->gemv_ok || !h->d_chunks || N < 1 || N > kSkinnyMaxN) return GRIM_ERR_UNSUPPORTED;
   if (x_dtype != h->dtype) return GRIM_ERR_DTYPE;
   const int nbr = (int)h->nbr;
   const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);

@@ -404,7 +404,7 @@ bool make_plan(const grim_bcr* h, int64_t N, StreamPlan& pl) {
 template <int BH, int NQ, int NW, bool XS, typename VT>
 cudaError_t launch_kernel(const StreamParams& p, const StreamPlan& pl, cudaStream_t s) {
   auto kern = bcr_stream_kernel<BH, NQ, NW, XS, VT, VT>;
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)pl.smem);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), pl.smem);
   if (e != cudaSuccess) return e;
   kern<<<dim3((unsigned)pl.grid_x, (unsigned)pl.passes), NW * 32, pl.smem, s>>>(p);
   return cudaGetLastError();

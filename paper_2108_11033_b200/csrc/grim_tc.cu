@@ -496,17 +496,11 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
     want = std::min(want, p.nkt / 4);  // at least four K tiles per part
     const size_t need = (size_t)h->M * (size_t)a.ncols * 4;
     if (want >= 2 && p.nkt >= 16 && blocks * 2 <= sms && need <= ((size_t)1 << 30)) {
-      grim_bcr* hm = const_cast<grim_bcr*>(h);
-      if (hm->tc_acc_bytes < need) {
-        cudaFree(hm->d_tc_acc);
-        hm->d_tc_acc = nullptr; hm->tc_acc_bytes = 0;
-        if (cudaMalloc(&hm->d_tc_acc, need) == cudaSuccess) hm->tc_acc_bytes = need;
-        else cudaGetLastError();
-      }
-      if (hm->d_tc_acc) {
+      // the scratch is reserved ahead of time (grim_bcr_reserve); without it, or when it is too small, the multiply runs unsplit
+      if (h->d_tc_acc && h->tc_acc_bytes >= need) {
         p.kt_per = (p.nkt + want - 1) / want;
         p.ksplit = (p.nkt + p.kt_per - 1) / p.kt_per;
-        p.acc = hm->d_tc_acc;
+        p.acc = h->d_tc_acc;
         if (p.ksplit < 2) { p.ksplit = 1; p.kt_per = p.nkt; p.acc = nullptr; }
         else if (cudaMemsetAsync(p.acc, 0, need, s) != cudaSuccess) return GRIM_ERR_CUDA;
       }
@@ -529,7 +523,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
                                : (h->bh == 4 ? bcr_tc_kernel<4, 3> : (h->bh == 8 ? bcr_tc_kernel<8, 3> : bcr_tc_kernel<16, 3>)))
                        : (h->bh == 4 ? bcr_tc_kernel<4, 1> : (h->bh == 8 ? bcr_tc_kernel<8, 1> : bcr_tc_kernel<16, 1>));
     const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec, extra);
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
+    if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem) != cudaSuccess) return GRIM_ERR_CUDA;
     dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt), (unsigned)p.ksplit);
     kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
     count_launch();
@@ -546,7 +540,7 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
     return GRIM_ERR_CUDA;
   const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec);
   auto kern = h->bh == 4 ? bcr_tc_kernel<4, 0> : (h->bh == 8 ? bcr_tc_kernel<8, 0> : bcr_tc_kernel<16, 0>);
-  cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+  cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
   if (e != cudaSuccess) return GRIM_ERR_CUDA;
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
   const int64_t mtiles = (h->tc_mtiles + p.mt - 1) / p.mt;

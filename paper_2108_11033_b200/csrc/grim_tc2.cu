@@ -479,12 +479,7 @@ grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t
   using Kern = void (*)(const CUtensorMap, const Tc2Params);
   const Kern kerns[4] = {bcr_tc2_kernel<0>, bcr_tc2_kernel<1>, bcr_tc2_kernel<2>, bcr_tc2_kernel<3>};
   Kern kern = kerns[mode];
-  // the attribute is kept by the kernel: set once and again only when a larger size is needed
-  static size_t have[4] = {0, 0, 0, 0};
-  if (have[mode] < smem) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return GRIM_ERR_CUDA;
-    have[mode] = smem;
-  }
+  if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem) != cudaSuccess) return GRIM_ERR_CUDA;
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3((unsigned)(2 * ((h->tc_mtiles + 1) / 2)), (unsigned)((a.ncols + kPairCols - 1) / kPairCols), 1);
   cfg.blockDim = dim3(a.conv ? kConvThreads : kThreads);

@@ -95,6 +95,8 @@ def test_config3_conv_batch32(B, bf16):
     h = B.grim_bcr_pack(L["W"], L["mask"], 16, 64, B.GRIM_BF16 if bf16 else B.GRIM_F32, B.GRIM_PACK_REORDER)
     try:
         out = torch.full((32, 512, 28, 28), float("nan"), device="cuda", dtype=torch.bfloat16 if bf16 else torch.float32)
+        if bf16:
+            B.grim_bcr_reserve(h, 32 * 28 * 28)
         B.grim_bcr_conv2d(h, to_dev(x, bf16), out, 3, 1, 1, bias=to_dev(L["bias"]), relu=True)
         torch.cuda.synchronize()
         assert B.grim_bcr_status(h) == B.GRIM_OK
@@ -116,6 +118,7 @@ def test_config4_vgg_stack_full_size(B, batch):
         h = B.grim_bcr_pack(L["W"], L["mask"], net["bh"], net["bw"], B.GRIM_BF16, B.GRIM_PACK_REORDER)
         Nb, C, H, Wd = cur.shape
         out = torch.full((Nb, L["cout"], H, Wd), float("nan"), device="cuda", dtype=torch.bfloat16)
+        B.grim_bcr_reserve(h, Nb * H * Wd)  # as the benchmark does at set-up
         B.grim_bcr_conv2d(h, cur, out, 3, 1, 1, bias=to_dev(L["bias"]), relu=True)
         torch.cuda.synchronize()
         assert B.grim_bcr_status(h) == B.GRIM_OK

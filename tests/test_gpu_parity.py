@@ -36,6 +36,8 @@ def check_spmm(B, W, mask, X, bh, bw, *, bf16=False, flags=0, tile_n=0, y_bf16=F
     dt = B.GRIM_BF16 if bf16 else B.GRIM_F32
     h = B.grim_bcr_pack(W, mask, bh, bw, dt, flags)
     try:
+        if bf16:
+            B.grim_bcr_reserve(h, N)  # workspace of the split tensor-core multiply, where the library chooses it
         Xd = to_dev(X, bf16)
         Yd = torch.full((M, N), float("nan"), device="cuda", dtype=torch.bfloat16 if y_bf16 else torch.float32)
         if tile_n or path:
@@ -280,7 +282,41 @@ def test_tune_returns_a_valid_choice(B):
     B.grim_bcr_spmm_ex(h, X, Y, tile_n=best["tile_n"], path=best["path"])
     torch.cuda.synchronize()
     assert rel_fro(Y.cpu().numpy(), orc.spmm(s["W"], s["mask"], s["X"])) <= F32_TOL
+    # the answer is kept in the handle: the plain call now launches exactly what the explicit call launches
+    Y.fill_(float("nan"))
+    n0 = B.grim_launch_count()
+    B.grim_bcr_spmm_ex(h, X, Y, tile_n=best["tile_n"], path=best["path"])
+    n_explicit = B.grim_launch_count() - n0
+    Y2 = torch.full_like(Y, float("nan"))
+    B.grim_bcr_spmm(h, X, Y2)
+    assert B.grim_launch_count() - n0 - n_explicit == n_explicit
+    torch.cuda.synchronize()
+    assert torch.equal(Y, Y2) or rel_fro(Y2.cpu().numpy(), Y.cpu().numpy()) <= 1e-6  # (a split multiply adds in any order)
     B.grim_bcr_destroy(h)
+
+
+def test_regime_flags_keep_one_set_of_layouts(B):
+    """A handle packed for narrow right-hand sides only multiplies N <= 16, one packed for wide ones N > 16; the other
+    regime is refused before any launch, and each holds less device memory than a handle with every layout."""
+    s = gen.sweep_case(1024, 64, 8.0, 8, 32, "uniform")
+    X64, X4 = to_dev(s["X"]), to_dev(s["X"][:, :4])
+    want = orc.spmm(s["W"], s["mask"], s["X"])
+    free0 = torch.cuda.mem_get_info()[0]
+    h_all = B.grim_bcr_pack(s["W"], s["mask"], 8, 32, B.GRIM_F32, 0)
+    used_all = free0 - torch.cuda.mem_get_info()[0]
+    B.grim_bcr_destroy(h_all)
+    for flag, ok_x, bad_x in ((B.GRIM_PACK_NARROW_ONLY, X4, X64), (B.GRIM_PACK_WIDE_ONLY, X64, X4)):
+        free1 = torch.cuda.mem_get_info()[0]
+        h = B.grim_bcr_pack(s["W"], s["mask"], 8, 32, B.GRIM_F32, flag)
+        assert free1 - torch.cuda.mem_get_info()[0] <= used_all
+        Y = torch.full((1024, ok_x.shape[1]), float("nan"), device="cuda")
+        B.grim_bcr_spmm(h, ok_x, Y)
+        torch.cuda.synchronize()
+        assert rel_fro(Y.cpu().numpy(), want[:, :ok_x.shape[1]]) <= F32_TOL
+        with pytest.raises(B.GrimError) as e:
+            B.grim_bcr_spmm(h, bad_x, torch.empty(1024, bad_x.shape[1], device="cuda"))
+        assert e.value.status == B.GRIM_ERR_UNSUPPORTED
+        B.grim_bcr_destroy(h)
 
 
 # ---------------------------------------------------------------------------------------- convolution
@@ -305,6 +341,8 @@ def check_conv(B, L, batch_x, *, ksize, stride, pad, bf16, relu=True, out_bf16=F
         OW = (Wd + 2 * pad - ksize) // stride + 1
         out = torch.full((Nb, W.shape[0], OH, OW), float("nan"), device="cuda",
                          dtype=torch.bfloat16 if out_bf16 else torch.float32)
+        if bf16:
+            B.grim_bcr_reserve(h, Nb * OH * OW)
         B.grim_bcr_conv2d(h, xd, out, ksize, stride, pad, bias=to_dev(bias), relu=relu, kernel_flags=kernel_flags)
         torch.cuda.synchronize()
         assert B.grim_bcr_status(h) == B.GRIM_OK
