@@ -141,6 +141,27 @@ grim_status_t grim_bcr_info(grim_bcr_t h, grim_bcr_info_t* info);
  */
 grim_status_t grim_bcr_export(grim_bcr_t h, void* buf_host, int64_t capacity, int64_t* written);
 
+/* BCRC, the storage format of Section 4.3, written to HOST arrays.  Rows are reordered by kept-weight count (largest
+ * first), then by column list, then by row id, so that rows with the same column list are neighbours; such a run of
+ * rows is a group and its column list is stored once:
+ *   reorder[M]                 original row at each position of the reordered matrix
+ *   row_offset[M + 1]          first weight of each reordered row in `weights`
+ *   occurrence[groups + 1]     first reordered row of each group
+ *   column_stride[groups + 1]  first entry of each group's column list in compact_column
+ *   compact_column[compact_columns]   the groups' column lists (ascending column ids)
+ *   weights[nnz]               kept weights row by row of the reordered matrix, fp32 (bf16 handles: the rounded values)
+ * Call once with all six array pointers NULL to learn the sizes, then with arrays of those sizes.  (The figure that
+ * carries the paper's worked example is not part of the available text; the fragments quoted in the text are
+ * reproduced by a test.) */
+typedef struct {
+  int64_t M, K, nnz;
+  int64_t groups;           /* runs of reordered rows that share one column list */
+  int64_t compact_columns;  /* entries of compact_column */
+} grim_bcrc_sizes_t;
+grim_status_t grim_bcr_export_bcrc(grim_bcr_t h, int32_t* reorder, int64_t* row_offset, int32_t* occurrence,
+                                   int64_t* column_stride, int32_t* compact_column, float* weights,
+                                   grim_bcrc_sizes_t* sizes);
+
 /* Writes the masked weight (zeros at pruned positions; bf16 handles: the rounded values) as
  * fp32 into HOST memory W_host[M x K], row stride ldw. */
 grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);

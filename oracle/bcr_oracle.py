@@ -258,3 +258,65 @@ def unpack_canonical(buf: bytes):
     if off != len(buf):
         raise ValueError("trailing bytes")
     return dict(W=W, mask=mask, row_perm=perm, M=M, K=K, bh=bh, bw=bw, nbr=nbr, nbc=nbc, dtype=dtype, nnz=nnz)
+
+
+# ----------------------------------------------------------------------------------------------
+# BCRC, the paper's storage format (Section 4.3).  parity unpinned against the paper's own worked example: the
+# figure that carries it is not in the available text.  The fragments the text quotes (reorder 0, 3; row offset 0, 3;
+# column stride 0, 3; first column list 0, 3, 6; occurrence 0, 2) are reproduced by a test on a matrix built to have
+# them, and the arrays are pinned by what they must satisfy: they rebuild the masked weight exactly, every group's
+# rows have exactly the stored list, and with no two equal lists the column arrays reduce to CSR of the reordered
+# matrix.
+# ----------------------------------------------------------------------------------------------
+
+
+def bcrc_export(W, mask, dtype: int = DTYPE_F32):
+    """The six arrays of Section 4.3 for the masked weight.
+
+    Rows are reordered by kept-weight count (largest first), then by column list (lexicographic), then by row id: rows
+    with equal lists become neighbours and form a group whose list is stored once.  reorder[p] = original row at
+    position p; row_offset[p] = first weight of reordered row p; occurrence[g] = first reordered row of group g;
+    column_stride[g] = first entry of group g's list in compact_column; weights = kept weights row by row.
+    """
+    Wm = masked_weight(W, mask, dtype)
+    keep = np.asarray(mask) != 0
+    M = keep.shape[0]
+    lists = [tuple(int(c) for c in np.flatnonzero(keep[r])) for r in range(M)]
+    order = sorted(range(M), key=lambda r: (-len(lists[r]), lists[r], r))
+    reorder, row_offset, occurrence, column_stride, compact, weights = [], [0], [], [], [], []
+    for p, r in enumerate(order):
+        reorder.append(r)
+        if p == 0 or lists[r] != lists[order[p - 1]]:
+            occurrence.append(p)
+            column_stride.append(len(compact))
+            compact.extend(lists[r])
+        weights.extend(float(Wm[r, c]) for c in lists[r])
+        row_offset.append(len(weights))
+    occurrence.append(M)
+    column_stride.append(len(compact))
+    return dict(reorder=np.array(reorder, np.int32), row_offset=np.array(row_offset, np.int64),
+                occurrence=np.array(occurrence, np.int32), column_stride=np.array(column_stride, np.int64),
+                compact_column=np.array(compact, np.int32), weights=np.array(weights, np.float32))
+
+
+def bcrc_to_dense(b, M: int, K: int) -> np.ndarray:
+    """Rebuilds the dense fp32 matrix from the six arrays (what a kernel that walks BCRC would read)."""
+    out = np.zeros((M, K), np.float32)
+    for g in range(len(b["occurrence"]) - 1):
+        cols = b["compact_column"][b["column_stride"][g]:b["column_stride"][g + 1]]
+        for p in range(b["occurrence"][g], b["occurrence"][g + 1]):
+            w = b["weights"][b["row_offset"][p]:b["row_offset"][p + 1]]
+            assert len(w) == len(cols)
+            out[b["reorder"][p], cols] = w
+    return out
+
+
+def index_bytes_bcrc(b) -> int:
+    """Bytes of everything in BCRC that is not a weight (32-bit entries, as CSR is counted below)."""
+    return 4 * (len(b["reorder"]) + len(b["row_offset"]) + len(b["occurrence"]) + len(b["column_stride"]) + len(b["compact_column"]))
+
+
+def index_bytes_csr(mask) -> int:
+    """Bytes of CSR's row pointers and column ids for the same matrix (32-bit entries)."""
+    keep = np.asarray(mask) != 0
+    return 4 * (keep.shape[0] + 1 + int(keep.sum()))

@@ -33,7 +33,7 @@ EXPORTED = [
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
-    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve",
+    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve", "grim_bcr_export_bcrc",
 ]
 
 
@@ -55,6 +55,10 @@ class grim_bcr_info_t(C.Structure):
                 ("export_bytes", C.c_int64), ("index_bytes_tc", C.c_int64)]
 
 
+class grim_bcrc_sizes_t(C.Structure):
+    _fields_ = [("M", C.c_int64), ("K", C.c_int64), ("nnz", C.c_int64), ("groups", C.c_int64), ("compact_columns", C.c_int64)]
+
+
 class grim_tune_t(C.Structure):
     _fields_ = [("tile_n", C.c_int32), ("path", C.c_int32), ("reserved", C.c_int32 * 6)]
 
@@ -74,6 +78,7 @@ lib.grim_bcr_reserve.argtypes = [_vp, C.c_int64]
 lib.grim_bcr_info.argtypes = [_vp, C.POINTER(grim_bcr_info_t)]
 lib.grim_bcr_export.argtypes = [_vp, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.grim_bcr_unpack_dense.argtypes = [_vp, _vp, C.c_int64]
+lib.grim_bcr_export_bcrc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(grim_bcrc_sizes_t)]
 lib.grim_bcr_spmm.argtypes = [_vp, C.POINTER(grim_mat_t), C.POINTER(grim_mat_t), _vp]
 lib.grim_bcr_spmm_ex.argtypes = [_vp, C.POINTER(grim_mat_t), C.POINTER(grim_mat_t), C.POINTER(grim_tune_t), _vp]
 lib.grim_bcr_tune.argtypes = [_vp, C.POINTER(grim_mat_t), C.POINTER(grim_mat_t), C.c_int, C.POINTER(grim_tune_t),
@@ -165,6 +170,18 @@ def grim_bcr_export(h: int) -> bytes:
     written = C.c_int64(0)
     _check(lib.grim_bcr_export(h, buf.ctypes.data, n, C.byref(written)), "grim_bcr_export")
     return buf[:written.value].tobytes()
+
+
+def grim_bcr_export_bcrc(h: int) -> dict:
+    sz = grim_bcrc_sizes_t()
+    _check(lib.grim_bcr_export_bcrc(h, None, None, None, None, None, None, C.byref(sz)), "grim_bcr_export_bcrc")
+    out = dict(reorder=np.empty(sz.M, np.int32), row_offset=np.empty(sz.M + 1, np.int64),
+               occurrence=np.empty(sz.groups + 1, np.int32), column_stride=np.empty(sz.groups + 1, np.int64),
+               compact_column=np.empty(sz.compact_columns, np.int32), weights=np.empty(sz.nnz, np.float32))
+    _check(lib.grim_bcr_export_bcrc(h, out["reorder"].ctypes.data, out["row_offset"].ctypes.data, out["occurrence"].ctypes.data,
+                                    out["column_stride"].ctypes.data, out["compact_column"].ctypes.data,
+                                    out["weights"].ctypes.data, C.byref(sz)), "grim_bcr_export_bcrc")
+    return out
 
 
 def grim_bcr_unpack_dense(h: int) -> np.ndarray:

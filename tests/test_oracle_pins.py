@@ -429,3 +429,77 @@ def test_gru_two_steps_by_hand_uses_previous_state_and_mask():
             new.append((1 - z) * n + z * h[u])
         h = new
         np.testing.assert_allclose(y[t], h, atol=1e-13)
+
+
+# ---------------------------------------------------------------------------- BCRC (Section 4.3)
+
+
+def test_bcrc_reproduces_the_fragments_quoted_in_the_text():
+    """Section 4.3 quotes the first entries of the arrays of its (unavailable) figure: reorder 0, 3; row offset 0, 3;
+    column stride 0, 3; the first column list 0, 3, 6; occurrence 0, 2 (rows 0 and 1 of the reordered matrix share
+    that list).  A matrix with that property: original rows 0 and 3 keep columns 0, 3, 6; the other rows keep fewer."""
+    mask = np.zeros((4, 8), np.uint8)
+    mask[0, [0, 3, 6]] = 1
+    mask[3, [0, 3, 6]] = 1
+    mask[1, [1, 4]] = 1
+    mask[2, [2]] = 1
+    W = np.arange(1, 33, dtype=np.float32).reshape(4, 8)
+    b = orc.bcrc_export(W, mask)
+    assert list(b["reorder"][:2]) == [0, 3]
+    assert list(b["row_offset"][:2]) == [0, 3]
+    assert list(b["column_stride"][:2]) == [0, 3]
+    assert list(b["compact_column"][:3]) == [0, 3, 6]
+    assert list(b["occurrence"][:2]) == [0, 2]
+    # the shared list is stored once: 3 + 2 + 1 column ids for 3 + 3 + 2 + 1 weights
+    assert len(b["compact_column"]) == 6 and len(b["weights"]) == 9
+    assert list(b["weights"][:6]) == [1, 4, 7, 25, 28, 31]
+
+
+@pytest.mark.parametrize("shape", [(32, 64, 8, 16, 4.0), (19, 45, 4, 16, 3.0), (48, 96, 16, 32, 6.0)])
+def test_bcrc_invariants(shape):
+    M, K, bh, bw, c = shape
+    W = gen.dense_weight(M, K, seed=24)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=c, seed=25, empty_frac=0.2)
+    b = orc.bcrc_export(W, mask)
+    want = np.where(mask != 0, W, np.float32(0))
+    assert np.array_equal(orc.bcrc_to_dense(b, M, K).view(np.uint32), want.view(np.uint32))   # rebuilds the masked weight
+    assert sorted(b["reorder"]) == list(range(M))                                               # a permutation
+    nnz_sorted = np.diff(b["row_offset"])
+    assert np.all(nnz_sorted[:-1] >= nnz_sorted[1:]) and b["row_offset"][-1] == int(mask.sum())
+    for g in range(len(b["occurrence"]) - 1):                                                   # groups are maximal runs
+        cols = b["compact_column"][b["column_stride"][g]:b["column_stride"][g + 1]]
+        assert np.all(np.diff(cols) > 0)
+        for p in range(b["occurrence"][g], b["occurrence"][g + 1]):
+            assert np.array_equal(np.flatnonzero(mask[b["reorder"][p]]), cols)
+        if g > 0:
+            prev = b["compact_column"][b["column_stride"][g - 1]:b["column_stride"][g]]
+            assert not np.array_equal(prev, cols)
+    assert orc.index_bytes_bcrc(b) <= orc.index_bytes_csr(mask) + 4 * (2 * M + 3)   # never worse than CSR + its fixed arrays
+
+
+def test_bcrc_reduces_to_csr_when_no_two_rows_share_a_list():
+    """With all column lists distinct every row is its own group, and (compact_column, column_stride) are the column ids
+    and row pointers of CSR for the reordered matrix (library routine: scipy.sparse.csr_matrix)."""
+    import scipy.sparse as sp
+    rng = np.random.default_rng(26)
+    M, K = 12, 40
+    mask = np.zeros((M, K), np.uint8)
+    for r in range(M):
+        mask[r, rng.choice(K, size=3 + r, replace=False)] = 1   # different lengths: all lists differ
+    W = gen.dense_weight(M, K, seed=27)
+    b = orc.bcrc_export(W, mask)
+    assert len(b["occurrence"]) == M + 1
+    csr = sp.csr_matrix(np.where(mask != 0, W, 0)[b["reorder"]])
+    csr.sort_indices()
+    assert np.array_equal(csr.indices, b["compact_column"]) and np.array_equal(csr.indptr, b["column_stride"])
+    assert np.array_equal(csr.data.astype(np.float32), b["weights"])
+
+
+def test_bcrc_saves_column_ids_when_rows_share_lists():
+    """One block per row band (block = whole row width): every kept row of a band shares the band's column list, so BCRC
+    stores one list per band where CSR stores one per row (Section 4.3's argument for the format)."""
+    M, K, bh = 64, 128, 8
+    mask = gen.bcr_mask(M, K, bh, 64, compression=4, seed=28)   # two blocks per band
+    b = orc.bcrc_export(gen.dense_weight(M, K, seed=29), mask)
+    assert len(b["compact_column"]) < int(mask.sum())
+    assert orc.index_bytes_bcrc(b) < orc.index_bytes_csr(mask)

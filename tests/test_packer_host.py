@@ -102,3 +102,21 @@ def test_host_only_handle_refuses_compute(B):
     import ctypes as C
     assert B.lib.grim_bcr_spmm(h, C.byref(mx), C.byref(my), None) == B.GRIM_ERR_INVALID_ARG
     B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("dtype", [0, 1])
+@pytest.mark.parametrize("case", CASES)
+def test_bcrc_export_matches_oracle(B, case, dtype):
+    """The library's BCRC export (Section 4.3) against the oracle's, array by array."""
+    M, K, bh, bw, kw = case
+    W = gen.dense_weight(M, K, seed=56)
+    mask = gen.bcr_mask(M, K, bh, bw, seed=57, **kw)
+    h = B.grim_bcr_pack(W, mask, bh, bw, dtype, B.GRIM_PACK_HOST_ONLY)
+    try:
+        got = B.grim_bcr_export_bcrc(h)
+        want = orc.bcrc_export(W, mask, dtype)
+        for k in ("reorder", "row_offset", "occurrence", "column_stride", "compact_column"):
+            assert np.array_equal(got[k], want[k]), k
+        assert np.array_equal(got["weights"].view(np.uint32), want["weights"].view(np.uint32))
+    finally:
+        B.grim_bcr_destroy(h)
