@@ -162,6 +162,17 @@ grim_status_t grim_bcr_export_bcrc(grim_bcr_t h, int32_t* reorder, int64_t* row_
                                    int64_t* column_stride, int32_t* compact_column, float* weights,
                                    grim_bcrc_sizes_t* sizes);
 
+/* Projection onto the BCR-sparse set (Section 5.2, Eq. (4): the step of the ADMM pruning that produces the masks this
+ * library packs).  V_host [M x K] (row stride ldv) is read, mask_host [M x K] (row stride ldm) receives 1 for kept and
+ * 0 for pruned entries; the projected matrix is V with the pruned entries set to zero.  The mask is BCR on the bh x bw
+ * grid and keeps at most (1 - sparsity) * M * K entries.  The exact nearest member of the set is a combinatorial
+ * problem and the paper gives no algorithm; this is a deterministic greedy one: a line (one row or one column of one
+ * block) costs the mean square of its entries that are still kept, and the cheapest line (ties: smallest
+ * block * (bh + bw) + row, or + bh + column) goes until the budget is met.  With 1 x 1 blocks it is magnitude pruning,
+ * i.e. the exact projection.  HOST only; *kept (may be NULL) receives the number of kept entries. */
+grim_status_t grim_bcr_project(const float* V_host, int64_t ldv, int64_t M, int64_t K, int bh, int bw, double sparsity,
+                               uint8_t* mask_host, int64_t ldm, int64_t* kept);
+
 /* Writes the masked weight (zeros at pruned positions; bf16 handles: the rounded values) as
  * fp32 into HOST memory W_host[M x K], row stride ldw. */
 grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);

@@ -320,3 +320,107 @@ def index_bytes_csr(mask) -> int:
     """Bytes of CSR's row pointers and column ids for the same matrix (32-bit entries)."""
     keep = np.asarray(mask) != 0
     return 4 * (keep.shape[0] + 1 + int(keep.sum()))
+
+
+# ----------------------------------------------------------------------------------------------
+# Projection onto the BCR-sparse set (Section 5.2, Eq. (4)).  The paper names the Euclidean projection but gives no
+# algorithm for it.  Two functions: the exact projection by exhaustive search (tiny inputs only; this is the
+# definition), and the greedy line-removal steps the library takes, written out naively (every cost recomputed from
+# scratch at every step).
+# ----------------------------------------------------------------------------------------------
+
+
+def bcr_project_exact(V, bh: int, bw: int, sparsity: float):
+    """The nearest BCR-sparse matrix by brute force: every choice of kept rows and kept columns per block, subject to
+    kept entries <= (1 - sparsity) * M * K, minimising the sum of squares of the removed entries.  Returns (mask, loss).
+    Exponential: a few blocks of at most 3 x 3."""
+    V = np.asarray(V, dtype=np.float64)
+    M, K = V.shape
+    nbr, nbc = -(-M // bh), -(-K // bw)
+    budget = int(np.floor((1.0 - sparsity) * M * K + 1e-9))
+    total = float((V ** 2).sum())
+    per_block = []
+    for i in range(nbr):
+        for j in range(nbc):
+            sub = V[i * bh:(i + 1) * bh, j * bw:(j + 1) * bw]
+            r, c = sub.shape
+            opts = {}
+            for rm in range(1 << r):
+                for cm in range(1 << c):
+                    rk = np.array([(rm >> t) & 1 for t in range(r)], bool)
+                    ck = np.array([(cm >> t) & 1 for t in range(c)], bool)
+                    n = int(rk.sum() * ck.sum())
+                    e = float((sub[np.ix_(rk, ck)] ** 2).sum())
+                    if n not in opts or e > opts[n][0]:      # per block only the best energy for each count matters
+                        opts[n] = (e, np.outer(rk, ck))
+            per_block.append(opts)
+    best = {0: (0.0, [])}                                       # kept count -> (kept energy, chosen masks)
+    for opts in per_block:
+        nxt = {}
+        for n0, (e0, ch) in best.items():
+            for n1, (e1, m1) in opts.items():
+                if n0 + n1 <= budget and (n0 + n1 not in nxt or e0 + e1 > nxt[n0 + n1][0]):
+                    nxt[n0 + n1] = (e0 + e1, ch + [m1])
+        best = nxt
+    e, ch = max(best.values(), key=lambda t: t[0])
+    mask = np.zeros((M, K), np.uint8)
+    for b, m in enumerate(ch):
+        i, j = divmod(b, nbc)
+        mask[i * bh:i * bh + m.shape[0], j * bw:j * bw + m.shape[1]] = m
+    return mask, total - e
+
+
+def bcr_project(V, bh: int, bw: int, sparsity: float) -> np.ndarray:
+    """Greedy projection: all rows and columns of all blocks start kept; a line is one row or one column of one block
+    and costs the mean square of its entries still kept (summed in index order, in double precision); the cheapest
+    line (ties: smallest id = block * (bh + bw) + row, or + bh + column) is removed until at most
+    (1 - sparsity) * M * K entries are kept.  Returns the keep mask."""
+    V = np.asarray(V, dtype=np.float32)
+    M, K = V.shape
+    nbr, nbc = -(-M // bh), -(-K // bw)
+    budget = int(np.floor((1.0 - sparsity) * M * K + 1e-9))
+    rowkeep = [[[True] * min(bh, M - i * bh) for j in range(nbc)] for i in range(nbr)]
+    colkeep = [[[True] * min(bw, K - j * bw) for j in range(nbc)] for i in range(nbr)]
+    kept = M * K
+
+    def cost(i, j, l):
+        rk, ck = rowkeep[i][j], colkeep[i][j]
+        if l < bh:
+            if l >= len(rk) or not rk[l]:
+                return None
+            vals = [float(V[i * bh + l, j * bw + c]) for c in range(len(ck)) if ck[c]]
+        else:
+            c = l - bh
+            if c >= len(ck) or not ck[c]:
+                return None
+            vals = [float(V[i * bh + r, j * bw + c]) for r in range(len(rk)) if rk[r]]
+        if not vals:
+            return None
+        s = 0.0
+        for v in vals:
+            s += v * v
+        return s / len(vals)
+
+    while kept > budget:
+        best = None
+        for i in range(nbr):
+            for j in range(nbc):
+                for l in range(bh + bw):
+                    c = cost(i, j, l)
+                    if c is not None and (best is None or c < best[0]):     # strict: the first (smallest id) wins ties
+                        best = (c, i, j, l)
+        if best is None:
+            break
+        _, i, j, l = best
+        if l < bh:
+            kept -= sum(colkeep[i][j])
+            rowkeep[i][j][l] = False
+        else:
+            kept -= sum(rowkeep[i][j])
+            colkeep[i][j][l - bh] = False
+    mask = np.zeros((M, K), np.uint8)
+    for i in range(nbr):
+        for j in range(nbc):
+            m = np.outer(rowkeep[i][j], colkeep[i][j])
+            mask[i * bh:i * bh + m.shape[0], j * bw:j * bw + m.shape[1]] = m
+    return mask

@@ -33,7 +33,7 @@ EXPORTED = [
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
-    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve", "grim_bcr_export_bcrc",
+    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve", "grim_bcr_export_bcrc", "grim_bcr_project",
 ]
 
 
@@ -78,6 +78,7 @@ lib.grim_bcr_reserve.argtypes = [_vp, C.c_int64]
 lib.grim_bcr_info.argtypes = [_vp, C.POINTER(grim_bcr_info_t)]
 lib.grim_bcr_export.argtypes = [_vp, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.grim_bcr_unpack_dense.argtypes = [_vp, _vp, C.c_int64]
+lib.grim_bcr_project.argtypes = [_vp, C.c_int64, C.c_int64, C.c_int64, C.c_int, C.c_int, C.c_double, _vp, C.c_int64, C.POINTER(C.c_int64)]
 lib.grim_bcr_export_bcrc.argtypes = [_vp, _vp, _vp, _vp, _vp, _vp, _vp, C.POINTER(grim_bcrc_sizes_t)]
 lib.grim_bcr_spmm.argtypes = [_vp, C.POINTER(grim_mat_t), C.POINTER(grim_mat_t), _vp]
 lib.grim_bcr_spmm_ex.argtypes = [_vp, C.POINTER(grim_mat_t), C.POINTER(grim_mat_t), C.POINTER(grim_tune_t), _vp]
@@ -182,6 +183,17 @@ def grim_bcr_export_bcrc(h: int) -> dict:
                                     out["column_stride"].ctypes.data, out["compact_column"].ctypes.data,
                                     out["weights"].ctypes.data, C.byref(sz)), "grim_bcr_export_bcrc")
     return out
+
+
+def grim_bcr_project(V: np.ndarray, bh: int, bw: int, sparsity: float) -> np.ndarray:
+    V = np.ascontiguousarray(V, dtype=np.float32)
+    M, K = V.shape
+    mask = np.empty((M, K), np.uint8)
+    kept = C.c_int64(0)
+    _check(lib.grim_bcr_project(V.ctypes.data, K, M, K, bh, bw, float(sparsity), mask.ctypes.data, K, C.byref(kept)),
+           "grim_bcr_project")
+    assert int(mask.sum()) == kept.value
+    return mask
 
 
 def grim_bcr_unpack_dense(h: int) -> np.ndarray:

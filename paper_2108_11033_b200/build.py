@@ -11,7 +11,7 @@ ROOT = os.path.dirname(PKG)
 CSRC = os.path.join(PKG, "csrc")
 OBJ = os.path.join(PKG, "_build")
 LIB = os.path.join(PKG, "libgrim.so")
-SOURCES = ["grim_pack.cu", "grim_spmm.cu", "grim_stream.cu", "grim_ffma.cu", "grim_tc.cu", "grim_tc2.cu", "grim_api.cu", "grim_gru.cu", "grim_bcrc.cu"]
+SOURCES = ["grim_pack.cu", "grim_spmm.cu", "grim_stream.cu", "grim_ffma.cu", "grim_tc.cu", "grim_tc2.cu", "grim_api.cu", "grim_gru.cu", "grim_bcrc.cu", "grim_project.cu"]
 ARCH = ["-gencode", "arch=compute_100a,code=sm_100a"]
 
 

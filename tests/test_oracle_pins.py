@@ -503,3 +503,45 @@ def test_bcrc_saves_column_ids_when_rows_share_lists():
     b = orc.bcrc_export(gen.dense_weight(M, K, seed=29), mask)
     assert len(b["compact_column"]) < int(mask.sum())
     assert orc.index_bytes_bcrc(b) < orc.index_bytes_csr(mask)
+
+
+# ---------------------------------------------------------------------------- projection onto the BCR set (Section 5.2)
+
+
+def test_projection_with_unit_blocks_is_magnitude_pruning():
+    """1 x 1 blocks: the BCR set is plain sparsity and the Euclidean projection is textbook - keep the largest
+    magnitudes.  The greedy steps must give exactly that."""
+    V = gen.normal_f32((12, 17), 1.0, 30, 0)
+    for sparsity in (0.0, 0.5, 0.9, 1.0):
+        mask = orc.bcr_project(V, 1, 1, sparsity)
+        k = int(np.floor((1 - sparsity) * V.size + 1e-9))
+        order = np.argsort(-np.abs(V).ravel(), kind="stable")
+        want = np.zeros(V.size, np.uint8)
+        want[order[:k]] = 1
+        assert int(mask.sum()) == k and np.array_equal(mask.ravel(), want)
+
+
+@pytest.mark.parametrize("seed", [31, 32, 33, 34])
+def test_projection_is_feasible_and_never_beats_the_exact_one(seed):
+    """Tiny blocks, exhaustive search: the greedy result lies in the set (BCR structure, enough zeros), so its distance
+    can only be >= the exact projection's; and the exact search itself is checked on the case where it is obvious."""
+    V = gen.normal_f32((4, 6), 1.0, seed, 0)
+    for sparsity in (0.3, 0.5, 0.75):
+        mask = orc.bcr_project(V, 2, 3, sparsity)
+        _, ok = orc.extract_blocks(mask, 2, 3)
+        assert ok and mask.sum() <= np.floor((1 - sparsity) * V.size + 1e-9)
+        exact_mask, exact_loss = orc.bcr_project_exact(V, 2, 3, sparsity)
+        _, ok2 = orc.extract_blocks(exact_mask, 2, 3)
+        assert ok2 and exact_mask.sum() <= np.floor((1 - sparsity) * V.size + 1e-9)
+        loss = float((V.astype(np.float64)[mask == 0] ** 2).sum())
+        assert abs(float((V.astype(np.float64)[exact_mask == 0] ** 2).sum()) - exact_loss) < 1e-9
+        assert loss >= exact_loss - 1e-12
+        assert loss <= 2.5 * exact_loss + 1e-12      # and it is not far off on these inputs
+
+
+def test_exact_projection_on_an_obvious_case():
+    """One 2 x 2 block, half the entries must go: a dominant column is what stays."""
+    V = np.array([[5.0, 0.1], [4.0, 0.2]], np.float32)
+    mask, loss = orc.bcr_project_exact(V, 2, 2, 0.5)
+    assert np.array_equal(mask, [[1, 0], [1, 0]]) and abs(loss - (0.01 + 0.04)) < 1e-6
+    assert np.array_equal(orc.bcr_project(V, 2, 2, 0.5), mask)

@@ -120,3 +120,17 @@ def test_bcrc_export_matches_oracle(B, case, dtype):
         assert np.array_equal(got["weights"].view(np.uint32), want["weights"].view(np.uint32))
     finally:
         B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("case", [(24, 40, 4, 8, 0.6), (19, 45, 4, 16, 0.75), (32, 64, 8, 32, 0.875), (7, 5, 1, 1, 0.5),
+                                  (16, 70, 16, 64, 0.5)])
+def test_projection_matches_oracle(B, case):
+    """The library's projection onto the BCR set (Section 5.2) takes the same decisions as the oracle's naive loop:
+    masks equal bit for bit; and what it returns can be packed."""
+    M, K, bh, bw, sparsity = case
+    V = gen.normal_f32((M, K), 1.0, 58, 0)
+    got = B.grim_bcr_project(V, bh, bw, sparsity)
+    assert np.array_equal(got, orc.bcr_project(V, bh, bw, sparsity))
+    h = B.grim_bcr_pack(V, got, bh, bw, 0, B.GRIM_PACK_HOST_ONLY)
+    assert B.grim_bcr_info(h).nnz == int(got.sum()) <= np.floor((1 - sparsity) * M * K + 1e-9)
+    B.grim_bcr_destroy(h)
