@@ -1005,6 +1005,26 @@ def run_bcrc_study(args):
                               total_saving=1.0 - (bcrc + 4 * nnz) / (csr + 4 * nnz))))
 
 
+def run_block_sweep(args):
+    """Time against number of blocks for one 1024 x 1024 matrix at 10x (the experiment of Section 5.1, left panel of its
+    figure) with the block shapes the packer takes, and the block size the search of that section then picks."""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2108_11033_b200.build import build_library
+    build_library()
+    from paper_2108_11033_b200 import blocksize as bs
+    sizes = [(1, 1), (1, 4), (2, 8), (4, 16), (8, 32), (16, 64)]
+    for N in (1, 64, 1024):
+        rows = []
+        for size in sizes:
+            layer = bs.synthesize(1024, 1024, 10.0, size)
+            rows.append(dict(block=f"{size[0]}x{size[1]}", blocks=(1024 // size[0]) * (1024 // size[1]),
+                             nnz=int(layer["mask"].sum()), ms=bs.run_layer(layer, N)))
+        pick, ms, trace = bs.find_opt_blk((1024, 1024), 10.0, sizes[1:], N=N, threshold=1.05)
+        print(json.dumps(dict(experiment="time vs number of blocks, 1024 x 1024, 10x, fp32", N=N, points=rows,
+                              find_opt_blk=dict(threshold=1.05, picked=pick, ms=ms, timed=[[list(t[0]), t[1]] for t in trace]))))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -1029,7 +1049,11 @@ def main():
     ap.add_argument("--sweep-blocks", default="4x16,8x32,16x64")
     ap.add_argument("--out", default="sweep.jsonl")
     ap.add_argument("--bcrc-study", action="store_true", help="host only: index bytes of the BCRC export against CSR")
+    ap.add_argument("--block-sweep", action="store_true", help="time vs number of blocks at 1024 x 1024, 10x, and the block-size search")
     args = ap.parse_args()
+    if args.block_sweep:
+        run_block_sweep(args)
+        return
     if args.bcrc_study:
         run_bcrc_study(args)
         return
