@@ -277,6 +277,13 @@ grim_status_t grim_gru_seq(grim_gru_t g, const float* x_dev, int64_t T, const fl
 grim_status_t grim_gru_status(grim_gru_t g);
 grim_status_t grim_gru_destroy(grim_gru_t g);
 
+/* One time step for a batch of B independent sequences (Section 6.3 times the GRU at sequence length 1, batch 32): the
+ * same equations with the batch as the right-hand side of the two sparse multiplies of every layer.  x_dev [B x in_0],
+ * h_dev [layers x B x H] holds every layer's state and is updated in place, y_dev [B x H] or NULL receives the last
+ * layer's new state; all fp32 DEVICE, batch-major.  Needs 2 * B <= max_T of grim_gru_create (GRIM_ERR_SHAPE
+ * otherwise).  Asynchronous; allocates nothing. */
+grim_status_t grim_gru_step(grim_gru_t g, const float* x_dev, int64_t B, float* h_dev, float* y_dev, grim_stream_t stream);
+
 /* Layer pipelining of grim_gru_seq (execution detail, Section 4.2's concern with keeping all units busy; the paper
  * has no multi-layer schedule).  With more than one layer the sequence is cut into `chunks` pieces in time and layer
  * l works on piece k while layer l - 1 works on piece k + 1, each layer on an internal stream ordered by events; the

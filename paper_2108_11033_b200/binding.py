@@ -33,7 +33,7 @@ EXPORTED = [
     "grim_bcr_spmm", "grim_bcr_spmm_ex", "grim_bcr_status", "grim_bcr_tune", "grim_bcr_conv2d", "grim_maxpool2x2",
     "grim_gru_create", "grim_gru_seq", "grim_gru_status", "grim_gru_destroy", "grim_gru_debug_barrier",
     "grim_gru_profile", "grim_gru_profile_read", "grim_gru_seq_static", "grim_gru_set_pipeline",
-    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve", "grim_bcr_export_bcrc", "grim_bcr_project",
+    "grim_launch_count", "grim_launch_count_reset", "grim_status_string", "grim_version", "grim_measure_ffma_peak", "grim_bcr_reserve", "grim_bcr_export_bcrc", "grim_bcr_project", "grim_gru_step",
 ]
 
 
@@ -91,6 +91,7 @@ lib.grim_gru_create.argtypes = [C.c_int, C.POINTER(_vp), C.POINTER(_vp), C.POINT
 lib.grim_gru_seq.argtypes = [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp]
 lib.grim_gru_seq_static.argtypes = [_vp, _vp, C.c_int64, _vp, _vp, _vp, _vp]
 lib.grim_gru_status.argtypes = [_vp]
+lib.grim_gru_step.argtypes = [_vp, _vp, C.c_int64, _vp, _vp, _vp]
 lib.grim_gru_destroy.argtypes = [_vp]
 lib.grim_gru_debug_barrier.argtypes = [_vp, C.c_int, C.c_uint]
 lib.grim_gru_profile.argtypes = [_vp, C.c_int]
@@ -277,6 +278,12 @@ def grim_gru_seq_static(g: int, x, y, h0=None, hT=None, stream=None):
     _check(lib.grim_gru_seq_static(g, x.data_ptr(), x.shape[0], h0.data_ptr() if h0 is not None else None,
                                    y.data_ptr(), hT.data_ptr() if hT is not None else None, _stream_ptr(stream)),
            "grim_gru_seq_static")
+
+
+def grim_gru_step(g: int, x, h, y=None, stream=None):
+    assert x.is_cuda and h.is_cuda and x.is_contiguous() and h.is_contiguous() and x.dim() == 2 and h.dim() == 3
+    _check(lib.grim_gru_step(g, x.data_ptr(), x.shape[0], h.data_ptr(), y.data_ptr() if y is not None else None,
+                             _stream_ptr(stream)), "grim_gru_step")
 
 
 def grim_gru_status(g: int) -> int:

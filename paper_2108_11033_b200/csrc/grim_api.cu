@@ -201,6 +201,29 @@ extern "C" grim_status_t grim_bcr_conv2d(grim_bcr_t h, const grim_conv_desc_t* d
   a.bias = d->bias_dev; a.relu = (d->flags & GRIM_CONV_RELU) ? 1 : 0;
   a.conv = 1; a.C = (int)d->C; a.H = (int)d->H; a.W = (int)d->W; a.KH = d->KH; a.KW = d->KW;
   a.stride = d->stride; a.pad = d->pad; a.OH = (int)OH; a.OW = (int)OW;
+  if (d->KH == 1 && d->KW == 1 && d->stride == 1 && d->pad == 0 && !(d->flags & (GRIM_CONV_PAIRED | GRIM_CONV_SINGLE))) {
+    // 1 x 1 kernels: the expanded input IS the input - per image a plain Cout x C times C x (H*W) product on the
+    // tensors as they lie in memory (row stride H*W), no gather at all; one launch per image
+    const int64_t hw = d->H * d->W;
+    const size_t in_esz = d->in_dtype == GRIM_BF16 ? 2 : 4, out_esz = d->out_dtype == GRIM_BF16 ? 2 : 4;
+    for (int64_t n = 0; n < d->N; ++n) {
+      SpmmArgs m;
+      m.X = static_cast<const uint8_t*>(in) + (size_t)(n * d->C * hw) * in_esz;
+      m.Y = static_cast<uint8_t*>(out) + (size_t)(n * h->M * hw) * out_esz;
+      m.ncols = hw; m.x_sk = hw; m.x_sq = 1; m.y_sr = hw; m.y_sq = 1;
+      m.x_dtype = d->in_dtype; m.y_dtype = d->out_dtype;
+      m.bias = d->bias_dev; m.relu = a.relu;
+      grim_status_t st;
+      if (tc2_path_supported(h, m) && hw >= 256 && h->tc_mtiles >= 2 &&
+          2 * ((h->tc_mtiles + 1) / 2) * ((hw + 511) / 512) * 3 >= 2 * (int64_t)sm_count(h->device))
+        st = launch_spmm_tc2(h, m, (cudaStream_t)stream);
+      else if (tc_path_supported(h, m) && hw >= 128) st = launch_spmm_tc(h, m, (cudaStream_t)stream);
+      else if (ffma_path_supported(h, m)) st = launch_ffma(h, m, (cudaStream_t)stream);
+      else st = launch_spmm(h, m, (cudaStream_t)stream);
+      if (st != GRIM_OK) return st;
+    }
+    return GRIM_OK;
+  }
   if (d->flags & GRIM_CONV_PAIRED) {
     if (!tc2_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
     return launch_spmm_tc2(h, a, (cudaStream_t)stream);

@@ -1135,3 +1135,63 @@ extern "C" grim_status_t grim_gru_seq_static(grim_gru_t g, const float* x, int64
   g->transposed_inputs = saved_tin;
   return st;
 }
+
+// -------------------------------------------------------------------------------------------------------------
+// One time step for a batch of sequences (Section 6.3 times the GRU at sequence length 1 and batch 32): per layer two
+// sparse multiplies with the batch as right-hand side (W_ih x and W_hh h, each with its bias in the epilogue) and one
+// fused gate kernel.
+// -------------------------------------------------------------------------------------------------------------
+namespace {
+// h'[b, u] = (1 - z) * n + z * h[b, u] with r, z, n from the two pre-activation buffers (batch-major, 3H per row);
+// the state is updated in place and copied to y when given.
+__global__ void gru_gate_kernel(const float* __restrict__ gi, const float* __restrict__ gh, float* __restrict__ h,
+                                float* __restrict__ y, int64_t B, int64_t H) {
+  const int64_t total = B * H;
+  for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+    const int64_t b = i / H, u = i - b * H;
+    const float* a = gi + b * 3 * H;
+    const float* q = gh + b * 3 * H;
+    const float r = sigmoidf_(a[u] + q[u]);
+    const float z = sigmoidf_(a[H + u] + q[H + u]);
+    const float n = tanhf(a[2 * H + u] + r * q[2 * H + u]);
+    const float hn = (1.f - z) * n + z * h[i];
+    h[i] = hn;
+    if (y) y[i] = hn;
+  }
+}
+}  // namespace
+
+extern "C" grim_status_t grim_gru_step(grim_gru_t g, const float* x, int64_t B, float* h, float* y, grim_stream_t stream) {
+  if (!g || !x || !h || B <= 0) return GRIM_ERR_INVALID_ARG;
+  if (2 * B > g->max_T) return GRIM_ERR_SHAPE;  // both pre-activation buffers of a layer live in its T x 3H scratch
+  cudaStream_t s = (cudaStream_t)stream;
+  const int64_t H = g->H;
+  const float* in = x;
+  for (int l = 0; l < g->L; ++l) {
+    float* hl = h + (int64_t)l * B * H;
+    float* gi = g->d_gi[(size_t)l];
+    float* gh = gi + B * 3 * H;
+    const grim_bcr* mats[2] = {g->Wih[(size_t)l], g->Whh[(size_t)l]};
+    const float* rhs[2] = {in, hl};
+    float* outs[2] = {gi, gh};
+    const float* bias[2] = {g->d_bih[(size_t)l], g->d_bhh[(size_t)l]};
+    for (int t = 0; t < 2; ++t) {
+      // batch-major operands: X(k, b) at b * K + k, Y(r, b) at b * 3H + r
+      SpmmArgs a;
+      a.X = rhs[t]; a.Y = outs[t]; a.ncols = B;
+      a.x_sk = 1; a.x_sq = mats[t]->K; a.y_sr = 1; a.y_sq = 3 * H;
+      a.x_dtype = GRIM_F32; a.y_dtype = GRIM_F32;
+      a.bias = bias[t];
+      const grim_status_t st = ffma_path_supported(mats[t], a) ? launch_ffma(mats[t], a, s) : launch_spmm(mats[t], a, s);
+      if (st != GRIM_OK) return st;
+    }
+    const int64_t total = B * H;
+    gru_gate_kernel<<<(unsigned)std::min<int64_t>((total + 255) / 256, (int64_t)sm_count(g->device) * 8), 256, 0, s>>>(
+        gi, gh, hl, l == g->L - 1 ? y : nullptr, B, H);
+    count_launch();
+    if (cudaGetLastError() != cudaSuccess) return GRIM_ERR_CUDA;
+    in = hl;
+  }
+  g->last_stream = s;
+  return GRIM_OK;
+}

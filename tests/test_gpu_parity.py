@@ -367,6 +367,21 @@ def test_conv_small(B, geom, bf16):
 
 
 @pytest.mark.parametrize("bf16", [False, True])
+def test_conv_11x11_and_1x1(B, bf16):
+    """The large kernels of the paper's 3 x 3 against 11 x 11 comparison (Section 6.3), at stride 1 and at the stride 4
+    of the classic first layer that uses them, and 1 x 1 kernels, which run as plain products per image (wide enough
+    pixel counts to reach the tensor-core kernels with bf16)."""
+    L = gen.conv_layer(2, 6, 48, 23, ksize=11, bh=8, bw=32, compression=5, seed=110)
+    check_conv(B, L, L["x"], ksize=11, stride=1, pad=5, bf16=bf16)
+    check_conv(B, L, L["x"], ksize=11, stride=4, pad=2, bf16=bf16, relu=False, out_bf16=bf16)
+    L1 = gen.conv_layer(3, 96, 264, 24, ksize=1, bh=8, bw=32, compression=4, seed=111)
+    check_conv(B, L1, L1["x"], ksize=1, stride=1, pad=0, bf16=bf16)
+    check_conv(B, L1, L1["x"], ksize=1, stride=1, pad=0, bf16=bf16, relu=False, out_bf16=bf16)
+    L2 = gen.conv_layer(2, 40, 72, 7, ksize=1, bh=4, bw=16, compression=3, seed=112)   # odd pixel count: unaligned rows
+    check_conv(B, L2, L2["x"], ksize=1, stride=1, pad=0, bf16=bf16)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
 def test_config3_conv_batch1(B, bf16):
     L = gen.conv_layer(1, 512, 512, 28, bf16=bf16)
     check_conv(B, L, L["x"], ksize=3, stride=1, pad=1, bf16=bf16)
@@ -582,6 +597,36 @@ def test_gru_layer_pipelining_gives_the_same_result(B, chunks):
         B.grim_gru_destroy(g)
         for h in handles:
             B.grim_bcr_destroy(h)
+
+
+@pytest.mark.parametrize("cfg", [(153, 1024, 2, 32), (37, 128, 3, 5), (20, 64, 1, 1)])
+def test_gru_batched_step(B, cfg):
+    """One time step for a batch of sequences (the paper's timed GRU shape is sequence length 1, batch 32), two steps in a
+    row so that the carried state is used: against the oracle run per batch element."""
+    in_f, H, L, batch = cfg
+    m = gen.gru_model(in_f, H, L, 2, compression=10 if H == 1024 else 4, seed=99)
+    g, handles = build_gru(B, m, 2 * batch + 2)
+    try:
+        xs = [gen.normal_f32((batch, in_f), 1.0, 100, t) for t in range(2)]
+        h = to_dev(gen.normal_f32((L, batch, H), 0.5, 101, 0))
+        h_np = h.cpu().numpy().astype(np.float64)
+        y = torch.full((batch, H), float("nan"), device="cuda")
+        for t in range(2):
+            B.grim_gru_step(g, to_dev(xs[t]), h, y)
+            torch.cuda.synchronize()
+            want_y = np.empty((batch, H))
+            for b in range(batch):
+                yb, hb = orc.gru_seq(m["layers"], xs[t][b:b + 1], h0=h_np[:, b])
+                want_y[b], h_np[:, b] = yb[0], hb
+            assert rel_fro(y.cpu().numpy(), want_y) <= F32_TOL
+            assert rel_fro(h.cpu().numpy(), h_np) <= F32_TOL
+        with pytest.raises(B.GrimError) as e:
+            B.grim_gru_step(g, torch.zeros(2 * batch + 2, in_f, device="cuda"), torch.zeros(L, 2 * batch + 2, H, device="cuda"))
+        assert e.value.status == B.GRIM_ERR_SHAPE
+    finally:
+        B.grim_gru_destroy(g)
+        for hd in handles:
+            B.grim_bcr_destroy(hd)
 
 
 def test_gru_bounded_wait_reports_timeout(B):
