@@ -50,6 +50,7 @@ struct ChunkDesc {
 // The streaming kernel moves the chunk layout in "runs": up to kRunChunks consecutive chunks of one band whose
 // values take at most kRunValueBytes (no single chunk is larger: 16 rows x 32 columns x 4 bytes is half of it).  Run r covers chunks [runs[r].c0, runs[r + 1].c0) and values [runs[r].v0, runs[r + 1].v0); the
 // table ends with a sentinel.  run_ptr[pos] .. run_ptr[pos + 1] are the runs of the band at schedule position pos.
+constexpr int kSliceRows = 1024;  // rows of X per K slice of the sliced copy (see grim_bcr::sl_*)
 constexpr int kRunChunks = 4;
 constexpr int kRunValueBytes = 4096;
 struct RunDesc {
@@ -155,6 +156,16 @@ struct grim_bcr {
   uint32_t* d_run_ptr = nullptr;
   grim::RunDesc* d_runs = nullptr;
   int64_t nruns = 0;
+  // K-sliced copy of the chunk layout for 2 <= N <= 16 (absent when K has a single slice): virtual band v = slice *
+  // nbr + schedule position; per virtual band its runs, its band and its slice
+  int sl_rows = 0;          // rows of X per slice (a multiple of bw)
+  int64_t sl_nslices = 0, sl_nruns = 0, index_bytes_sliced = 0;
+  uint32_t* d_sl_colwords = nullptr;
+  void* d_sl_vals = nullptr;
+  uint32_t* d_sl_run_ptr = nullptr;
+  grim::RunDesc* d_sl_runs = nullptr;
+  uint32_t* d_sl_band_of = nullptr;
+  uint32_t* d_sl_slice_of = nullptr;
   // dense bf16 copy for the tensor-core path is decompressed on the fly; nothing stored here
 };
 

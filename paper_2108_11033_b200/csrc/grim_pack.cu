@@ -52,6 +52,12 @@ void free_device(grim_bcr* h) {
   cudaFree(h->d_runs);
   cudaFree(h->d_rc_stage);
   cudaFree(h->d_rc_blob);
+  cudaFree(h->d_sl_colwords);
+  cudaFree(h->d_sl_vals);
+  cudaFree(h->d_sl_run_ptr);
+  cudaFree(h->d_sl_runs);
+  cudaFree(h->d_sl_band_of);
+  cudaFree(h->d_sl_slice_of);
   cudaFree(h->d_td_stage);
   cudaFree(h->d_td_blob);
   cudaFree(h->d_status);
@@ -212,23 +218,30 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
     h->index_bytes_spmm = (int64_t)stage.size() * (int64_t)sizeof(StageEntry) + (int64_t)(blob.size() - (size_t)nnz * vsz) +
                           nbr * 4;
 
-    // ---- chunk layout for the N = 1 kernel
-    std::vector<uint32_t> band_ptr((size_t)nbr + 1, 0);
-    std::vector<ChunkDesc> chunks;
-    std::vector<uint32_t> colwords;
-    std::vector<uint8_t> gvals;
-    std::vector<uint32_t> run_ptr;
-    std::vector<RunDesc> runs;
-    h->gemv_ok = K <= 65536;
-    if (h->gemv_ok) {
-      gvals.reserve((size_t)nnz * vsz);
+    // ---- chunk layout for the N <= 16 kernels
+    // A "virtual band" is a band restricted to block columns [jlo, jhi): the whole band for the matrix-vector product,
+    // one K slice of it for 2 <= N <= 16 (see below).  build_narrow lays the chunks and runs of a list of virtual
+    // bands out, in list order.
+    struct VBand { int64_t pos, jlo, jhi; };
+    struct Narrow {
+      std::vector<uint32_t> band_ptr;  // per virtual band: first chunk
+      std::vector<ChunkDesc> chunks;
+      std::vector<uint32_t> colwords;
+      std::vector<uint8_t> gvals;
+      std::vector<uint32_t> run_ptr;   // per virtual band: first run
+      std::vector<RunDesc> runs;
+    };
+    auto build_narrow = [&](const std::vector<VBand>& vb, Narrow& o) {
+      const int64_t nv = (int64_t)vb.size();
+      o.band_ptr.assign((size_t)nv + 1, 0);
+      o.gvals.reserve((size_t)nnz * vsz);
       std::vector<int64_t> order;
       uint64_t gv_elems = 0;
-      for (int64_t pos = 0; pos < nbr; ++pos) {
-        const int64_t i = h->band_order[(size_t)pos];
-        band_ptr[(size_t)pos] = (uint32_t)chunks.size();
+      for (int64_t v = 0; v < nv; ++v) {
+        const int64_t i = h->band_order[(size_t)vb[(size_t)v].pos];
+        o.band_ptr[(size_t)v] = (uint32_t)o.chunks.size();
         order.clear();
-        for (int64_t j = 0; j < nbc; ++j)
+        for (int64_t j = vb[(size_t)v].jlo; j < vb[(size_t)v].jhi; ++j)
           if (h->blocks[(size_t)(i * nbc + j)].kr && h->blocks[(size_t)(i * nbc + j)].kc) order.push_back(j);
         std::stable_sort(order.begin(), order.end(), [&](int64_t a, int64_t b) {
           return h->blocks[(size_t)(i * nbc + a)].kr > h->blocks[(size_t)(i * nbc + b)].kr;
@@ -247,9 +260,9 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
             const int nc = (int)std::min<size_t>(32, cols.size() - c0);
             ChunkDesc cd;
             cd.val_off = (uint32_t)gv_elems;
-            cd.cw_off = (uint32_t)colwords.size();
+            cd.cw_off = (uint32_t)o.colwords.size();
             cd.ncols_kr = (uint32_t)nc | ((uint32_t)kr << 16);
-            chunks.push_back(cd);
+            o.chunks.push_back(cd);
             for (int l = 0; l < nc; ++l) {
               const int64_t j = cols[c0 + l].first;
               const HostBlock& hb = h->blocks[(size_t)(i * nbc + j)];
@@ -257,38 +270,38 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
               int b = cols[c0 + l].second, c = 0;
               for (uint64_t m = hb.colmask;; ++c)
                 if ((m >> c) & 1ull) { if (b-- == 0) break; }
-              colwords.push_back((uint32_t)(j * bw + c) | (hb.rowmask << 16));
+              o.colwords.push_back((uint32_t)(j * bw + c) | (hb.rowmask << 16));
             }
-            colwords.resize(chunks.size() * 32, 0u);  // every chunk owns 32 words; unused slots: no row kept
-            for (int s = 0; s < kr; ++s)
+            o.colwords.resize(o.chunks.size() * 32, 0u);  // every chunk owns 32 words; unused slots: no row kept
+            for (int sr = 0; sr < kr; ++sr)
               for (int l = 0; l < nc; ++l) {
                 const HostBlock& hb = h->blocks[(size_t)(i * nbc + cols[c0 + l].first)];
-                const float v = h->vals[(size_t)(hb.val_off + (uint64_t)s * hb.kc + (uint64_t)cols[c0 + l].second)];
+                const float v = h->vals[(size_t)(hb.val_off + (uint64_t)sr * hb.kc + (uint64_t)cols[c0 + l].second)];
                 if (vdt == GRIM_BF16) {
                   uint16_t u = bf16_bits(v);
-                  gvals.insert(gvals.end(), (uint8_t*)&u, (uint8_t*)&u + 2);
+                  o.gvals.insert(o.gvals.end(), (uint8_t*)&u, (uint8_t*)&u + 2);
                 } else {
-                  gvals.insert(gvals.end(), (const uint8_t*)&v, (const uint8_t*)&v + 4);
+                  o.gvals.insert(o.gvals.end(), (const uint8_t*)&v, (const uint8_t*)&v + 4);
                 }
                 ++gv_elems;
               }
           }
         }
       }
-      gvals.resize(gvals.size() + 64 * vsz, 0);  // the kernels may read (and discard) up to a warp's width past a chunk
-      band_ptr[(size_t)nbr] = (uint32_t)chunks.size();
+      o.gvals.resize(o.gvals.size() + 64 * vsz, 0);  // the kernels may read (and discard) up to a warp's width past a chunk
+      o.band_ptr[(size_t)nv] = (uint32_t)o.chunks.size();
       // runs: the transfer units of the streaming kernel
-      run_ptr.assign((size_t)nbr + 1, 0);
-      for (int64_t pos = 0; pos < nbr; ++pos) {
-        run_ptr[(size_t)pos] = (uint32_t)runs.size();
-        uint32_t c = band_ptr[(size_t)pos];
-        const uint32_t ce = band_ptr[(size_t)pos + 1];
+      o.run_ptr.assign((size_t)nv + 1, 0);
+      for (int64_t v = 0; v < nv; ++v) {
+        o.run_ptr[(size_t)v] = (uint32_t)o.runs.size();
+        uint32_t c = o.band_ptr[(size_t)v];
+        const uint32_t ce = o.band_ptr[(size_t)v + 1];
         while (c < ce) {
-          runs.push_back(RunDesc{c, chunks[c].val_off});
+          o.runs.push_back(RunDesc{c, o.chunks[c].val_off});
           size_t bytes = 0;
           int n = 0;
           while (c < ce && n < kRunChunks) {
-            const uint32_t nk = chunks[c].ncols_kr;
+            const uint32_t nk = o.chunks[c].ncols_kr;
             const size_t cb = (size_t)(nk & 0xFFFFu) * (nk >> 16) * vsz;
             if (n > 0 && bytes + cb > (size_t)kRunValueBytes) break;
             bytes += cb;
@@ -297,16 +310,44 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
           }
         }
       }
-      run_ptr[(size_t)nbr] = (uint32_t)runs.size();
-      runs.push_back(RunDesc{(uint32_t)chunks.size(), (uint32_t)gv_elems});
-      h->nruns = (int64_t)runs.size() - 1;
-      h->nchunks = (int64_t)chunks.size();
-      h->h_gemv_band_ptr = band_ptr;
-      h->h_chunks = chunks;
-      h->n_colwords = (int64_t)colwords.size();
+      o.run_ptr[(size_t)nv] = (uint32_t)o.runs.size();
+      o.runs.push_back(RunDesc{(uint32_t)o.chunks.size(), (uint32_t)gv_elems});
+    };
+    Narrow nar, sl;  // whole bands; K slices
+    std::vector<uint32_t> sl_band_of, sl_slice_of;  // sliced copy: band and slice of every virtual band
+    h->gemv_ok = K <= 65536;
+    if (h->gemv_ok) {
+      std::vector<VBand> vb;
+      for (int64_t pos = 0; pos < nbr; ++pos) vb.push_back(VBand{pos, 0, nbc});
+      build_narrow(vb, nar);
+      h->nruns = (int64_t)nar.runs.size() - 1;
+      h->nchunks = (int64_t)nar.chunks.size();
+      h->h_gemv_band_ptr = nar.band_ptr;
+      h->h_chunks = nar.chunks;
+      h->n_colwords = (int64_t)nar.colwords.size();
       // what the streaming kernel reads besides the values: column words, the run table, the band tables
-      h->index_bytes_gemv = (int64_t)colwords.size() * 4 + (int64_t)runs.size() * (int64_t)sizeof(RunDesc) +
+      h->index_bytes_gemv = (int64_t)nar.colwords.size() * 4 + (int64_t)nar.runs.size() * (int64_t)sizeof(RunDesc) +
                             (nbr + 1) * 4 + nbr * 4;
+      // K slices for 2 <= N <= 16: a thread block stages the slice's rows of X in shared memory once and multiplies the
+      // slice's part of many bands from there (Section 4.4: a needed input row is loaded once), instead of gathering
+      // them from L2 for every band.  A second copy of the values in slice-major order; only built when K has more
+      // than one slice (otherwise the whole-band layout is its own single slice).
+      const int64_t spb = std::max<int64_t>(1, kSliceRows / bw);  // block columns per slice
+      h->sl_rows = (int)(spb * bw);
+      h->sl_nslices = (nbc + spb - 1) / spb;
+      if (h->sl_nslices > 1 && !(flags & GRIM_PACK_WIDE_ONLY)) {
+        std::vector<VBand> vs;
+        for (int64_t sidx = 0; sidx < h->sl_nslices; ++sidx)
+          for (int64_t pos = 0; pos < nbr; ++pos) {
+            vs.push_back(VBand{pos, sidx * spb, std::min<int64_t>((sidx + 1) * spb, nbc)});
+            sl_band_of.push_back(h->band_order[(size_t)pos]);
+            sl_slice_of.push_back((uint32_t)sidx);
+          }
+        build_narrow(vs, sl);
+        h->sl_nruns = (int64_t)sl.runs.size() - 1;
+        h->index_bytes_sliced = (int64_t)sl.colwords.size() * 4 + (int64_t)sl.runs.size() * (int64_t)sizeof(RunDesc) +
+                                ((int64_t)vs.size() + 1) * 4 + (int64_t)vs.size() * 8;
+      }
     }
 
     // ---- row-chunk layout for the register-tiled and tensor-core kernels
@@ -458,12 +499,20 @@ extern "C" grim_status_t grim_bcr_pack(const float* W, int64_t ldw, const uint8_
       const unsigned zero = 0;
       if (e == cudaSuccess) e = upload(&h->d_status, &zero, 4);
       if (e == cudaSuccess && h->gemv_ok && narrow) {
-        e = upload(&h->d_gemv_band_ptr, band_ptr.data(), band_ptr.size() * 4);
-        if (e == cudaSuccess) e = upload(&h->d_chunks, chunks.data(), chunks.size() * sizeof(ChunkDesc));
-        if (e == cudaSuccess) e = upload(&h->d_colwords, colwords.data(), colwords.size() * 4);
-        if (e == cudaSuccess) e = upload((uint8_t**)&h->d_gemv_vals, gvals.data(), gvals.size());
-        if (e == cudaSuccess) e = upload(&h->d_run_ptr, run_ptr.data(), run_ptr.size() * 4);
-        if (e == cudaSuccess) e = upload(&h->d_runs, runs.data(), runs.size() * sizeof(RunDesc));
+        e = upload(&h->d_gemv_band_ptr, nar.band_ptr.data(), nar.band_ptr.size() * 4);
+        if (e == cudaSuccess) e = upload(&h->d_chunks, nar.chunks.data(), nar.chunks.size() * sizeof(ChunkDesc));
+        if (e == cudaSuccess) e = upload(&h->d_colwords, nar.colwords.data(), nar.colwords.size() * 4);
+        if (e == cudaSuccess) e = upload((uint8_t**)&h->d_gemv_vals, nar.gvals.data(), nar.gvals.size());
+        if (e == cudaSuccess) e = upload(&h->d_run_ptr, nar.run_ptr.data(), nar.run_ptr.size() * 4);
+        if (e == cudaSuccess) e = upload(&h->d_runs, nar.runs.data(), nar.runs.size() * sizeof(RunDesc));
+        if (e == cudaSuccess && !sl.runs.empty()) {
+          e = upload(&h->d_sl_colwords, sl.colwords.data(), sl.colwords.size() * 4);
+          if (e == cudaSuccess) e = upload((uint8_t**)&h->d_sl_vals, sl.gvals.data(), sl.gvals.size());
+          if (e == cudaSuccess) e = upload(&h->d_sl_run_ptr, sl.run_ptr.data(), sl.run_ptr.size() * 4);
+          if (e == cudaSuccess) e = upload(&h->d_sl_runs, sl.runs.data(), sl.runs.size() * sizeof(RunDesc));
+          if (e == cudaSuccess) e = upload(&h->d_sl_band_of, sl_band_of.data(), sl_band_of.size() * 4);
+          if (e == cudaSuccess) e = upload(&h->d_sl_slice_of, sl_slice_of.data(), sl_slice_of.size() * 4);
+        }
       }
       if (e != cudaSuccess) {
         st = (e == cudaErrorMemoryAllocation) ? GRIM_ERR_ALLOC : GRIM_ERR_CUDA;

@@ -25,7 +25,12 @@ constexpr int kSRun = kRunChunks;   // chunks per stage at most (one bulk copy f
 constexpr int kSMaxSlots = 4;      // ring slots per warp
 constexpr int kSPartBytes = 8192;  // shared memory for the partial sums of one batch of bands
 constexpr int kSMaxBands = 2048;   // bands one thread block can list
-constexpr int kSMaxXBytes = 65536; // largest activation vector staged in shared memory (N = 1)
+constexpr int kSMaxXBytes = 81920; // most bytes of activations staged in shared memory (N = 1: the vector; N > 1: a K slice)
+
+// shared memory for the partial sums of one batch of bands
+__host__ __device__ constexpr int part_bytes(bool staged) { return staged ? 4 * kSPartBytes : kSPartBytes; }
+// bytes between staged rows of X (see the kernel)
+__host__ __device__ constexpr int x_row_stride(int nq, int esz) { return nq * esz + (nq * esz >= 32 ? 16 : 0); }
 
 struct StreamParams {
   const uint32_t* run_ptr;
@@ -38,9 +43,15 @@ struct StreamParams {
   unsigned* status;
   int64_t ldx, ldy;
   int N, nbr, M, K, bh, y_dtype, vec_ok;
+  int stage_vec;  // the staged rows of X can be copied in aligned 16-byte (8-byte for rows of 8 bytes) pieces
   int nslots, nk_max;
   uint32_t stage_bytes, off_band, off_part, off_x, off_ring;
   unsigned spin_limit;
+  // K-sliced mode (2 <= N <= 16): the "bands" above are virtual bands (one band restricted to one K slice); slice_of
+  // gives each one's slice (null: everything is slice 0), sl_rows the rows of X per slice, accumulate = 1 when a row
+  // of Y gets contributions from several virtual bands (added atomically into a zeroed Y)
+  const uint32_t* slice_of;
+  int sl_rows, accumulate;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -154,15 +165,25 @@ struct RunFetch {
   int valid = 0;
 };
 
+// XS: the activations are staged in shared memory - the whole vector for N = 1; for N > 1 the rows of the current K
+// slice (NQ columns of them), reloaded by the whole block when its next band lies in another slice.
 template <int BH, int NQ, int NW, bool XS, typename VT, typename XT>
 __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamParams p) {
-  constexpr int PB = (kSPartBytes / (NW * BH * NQ * 4)) > 0 ? (kSPartBytes / (NW * BH * NQ * 4)) : 1;  // bands per batch
+  // bands per batch (between two block-wide meetings).  In the staged mode a band is only one K slice of a band and
+  // has a few runs, i.e. work for a few warps: the batch is what keeps all warps busy, so it is larger there.
+  constexpr int kPart = part_bytes(XS && NQ > 1);
+  constexpr int PB = (kPart / (NW * BH * NQ * 4)) > 0 ? (kPart / (NW * BH * NQ * 4)) : 1;
+  // staged rows of X (N > 1): NQ elements, 16 bytes apart from the next row when a row is 32 bytes or longer, so that
+  // the 32 lanes' rows (any 32 of the slice) spread over the shared-memory banks instead of two or four groups of them
+  constexpr int kRowBytes = NQ * (int)sizeof(XT);
+  constexpr int kRowStride = x_row_stride(NQ, (int)sizeof(XT));
   extern __shared__ __align__(128) uint8_t smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);                            // [NW][kSMaxSlots]
   uint32_t* s_slack = reinterpret_cast<uint32_t*>(smem + NW * kSMaxSlots * 8);   // [NW][kSMaxSlots]
   int* s_abort = reinterpret_cast<int*>(s_slack + NW * kSMaxSlots);
   uint2* s_band = reinterpret_cast<uint2*>(smem + p.off_band);                   // [nk] runs of each band
   uint32_t* s_first_row = reinterpret_cast<uint32_t*>(s_band + p.nk_max);        // [nk] first matrix row of each band
+  uint32_t* s_slice = s_first_row + p.nk_max;                                    // [nk] K slice of each band (sliced mode)
   float* part = reinterpret_cast<float*>(smem + p.off_part);                     // [PB][NW][BH * NQ]
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t smem_base = smem_u32(smem);
@@ -186,6 +207,7 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
     const int pos = k * grid + ((k & 1) ? grid - 1 - bid : bid);
     s_band[k] = make_uint2(p.run_ptr[pos], p.run_ptr[pos + 1]);
     s_first_row[k] = p.band_order[pos] * (uint32_t)p.bh;
+    s_slice[k] = p.slice_of ? p.slice_of[pos] : 0u;
   }
   __syncthreads();
   // The run table entries of this block's bands are pulled into L2 now, while the memory system is idle: the
@@ -239,12 +261,13 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
   }
   RunFetch pend0 = prepare(), pend1 = prepare();
 
-  if (XS) {
+  if (XS && NQ == 1) {
     XT* sx = reinterpret_cast<XT*>(smem + p.off_x);
     const XT* X = static_cast<const XT*>(p.X);
     for (int k = threadIdx.x; k < p.K; k += NW * 32) sx[k] = X[(int64_t)k * p.ldx];
     __syncthreads();
   }
+  int cur_slice = -1;  // (N > 1) slice whose rows of X are in shared memory
 
   bool failed = false;
   int slot = 0;
@@ -253,14 +276,55 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
   RunWalk<NW> cw_walk;
   for (int kb = 0; kb < nk; kb += PB) {
     const int nb = min(PB, nk - kb);
+    if (XS && NQ > 1) {
+      // warps without a run in a band leave its slot alone: the slots start at zero
+      for (int i = threadIdx.x; i < nb * NW * BH * NQ; i += NW * 32) part[i] = 0.f;
+      __syncthreads();
+    }
     for (int b = 0; b < nb; ++b) {
       float acc[BH][NQ];
 #pragma unroll
       for (int r = 0; r < BH; ++r)
 #pragma unroll
         for (int q = 0; q < NQ; ++q) acc[r][q] = 0.f;
+      if (XS && NQ > 1 && (int)s_slice[kb + b] != cur_slice) {
+        // every warp walks the same bands in the same order, so all of them arrive here together: the rows of the new
+        // slice replace the old ones once nobody reads those any more
+        cur_slice = (int)s_slice[kb + b];
+        __syncthreads();
+        uint8_t* sx = smem + p.off_x;
+        const XT* X = static_cast<const XT*>(p.X);
+        const int64_t base = (int64_t)cur_slice * p.sl_rows;
+        if (p.stage_vec) {
+          // asynchronous copies in pieces of PIECE bytes (the weight rings keep filling meanwhile)
+          constexpr int PIECE = kRowBytes >= 16 ? 16 : 8, PPR = kRowBytes / PIECE;
+          for (int e = threadIdx.x; e < p.sl_rows * PPR; e += NW * 32) {
+            const int r = e / PPR, pc = e - r * PPR;
+            uint8_t* dst = sx + (size_t)r * kRowStride + pc * PIECE;
+            if (base + r < p.K) {
+              const uint8_t* src = reinterpret_cast<const uint8_t*>(X + (base + r) * p.ldx + q0) + pc * PIECE;
+              if (PIECE == 16) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+              else asm volatile("cp.async.ca.shared.global [%0], [%1], 8;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+            } else if (PIECE == 16) {
+              *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+            } else {
+              *reinterpret_cast<uint2*>(dst) = make_uint2(0u, 0u);
+            }
+          }
+          asm volatile("cp.async.wait_all;" ::: "memory");
+        } else {
+          for (int e = threadIdx.x; e < p.sl_rows * NQ; e += NW * 32) {
+            const int r = e / NQ, q = e - r * NQ;
+            reinterpret_cast<XT*>(sx + (size_t)r * kRowStride)[q] =
+                (base + r < p.K && q0 + q < p.N) ? X[(base + r) * p.ldx + q0 + q] : XT(0.f);
+          }
+        }
+        __syncthreads();
+      }
       cw_walk.next_band(s_band, nk, warp);
+      bool had_run = false;
       for (uint32_t run = cw_walk.r; run < cw_walk.end && !failed; run += NW) {
+        had_run = true;
         if (!__all_sync(0xffffffffu, mbar_wait(my_full + slot, phase, p.spin_limit, s_abort))) {
           failed = true;
           if (lane == 0) {
@@ -283,9 +347,27 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
         for (int u = 0; u < kSRun; ++u) {
           const uint32_t wd = *reinterpret_cast<const uint32_t*>(smem + cw_at + u * 128);
           words[u] = u < n ? wd : 0u;
-          if (XS) {
+          if (XS && NQ == 1) {
             const float xv = to_f32(*reinterpret_cast<const XT*>(smem + p.off_x + (words[u] & 0xFFFFu) * (uint32_t)sizeof(XT)));
             x[u][0] = (words[u] >> 16) ? xv : 0.f;
+          } else if (XS) {
+            // this column's row of the staged slice: NQ consecutive elements (unused lanes read row 0 and multiply nothing)
+            const uint32_t rl = (words[u] >> 16) ? (words[u] & 0xFFFFu) - (uint32_t)(cur_slice * p.sl_rows) : 0u;
+            const XT* xr = reinterpret_cast<const XT*>(smem + p.off_x + rl * (uint32_t)kRowStride);
+            if (sizeof(XT) == 4) {
+#pragma unroll
+              for (int i = 0; i < NQ / 4; ++i) {
+                const float4 v = reinterpret_cast<const float4*>(xr)[i];
+                x[u][4 * i] = v.x; x[u][4 * i + 1] = v.y; x[u][4 * i + 2] = v.z; x[u][4 * i + 3] = v.w;
+              }
+            } else {
+#pragma unroll
+              for (int i = 0; i < NQ / 4; ++i) {
+                const uint2 w2 = reinterpret_cast<const uint2*>(xr)[i];
+                x[u][4 * i] = __uint_as_float(w2.x << 16); x[u][4 * i + 1] = __uint_as_float(w2.x & 0xFFFF0000u);
+                x[u][4 * i + 2] = __uint_as_float(w2.y << 16); x[u][4 * i + 3] = __uint_as_float(w2.y & 0xFFFF0000u);
+              }
+            }
           } else if (words[u] >> 16) {
             load_x<NQ, XT>(p, words[u] & 0xFFFFu, q0, x[u]);
           } else {
@@ -326,6 +408,7 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
         if (++slot == nslots) { slot = 0; phase ^= 1u; }
       }
       float* mine = part + ((size_t)b * NW + warp) * (BH * NQ);
+      if (XS && NQ > 1 && !had_run) continue;  // (the same in every lane) this warp had no run of the band
 #pragma unroll
       for (int q = 0; q < NQ; ++q) {
         float t[BH];
@@ -344,7 +427,9 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
       float s = 0.f;
 #pragma unroll 4
       for (int w = 0; w < NW; ++w) s += part[((size_t)b * NW + w) * (BH * NQ) + rq];
-      if (p.y_dtype == GRIM_F32) static_cast<float*>(p.Y)[row * p.ldy + q0 + q] = s;
+      if (p.accumulate) {  // (fp32 only) one of several slices' share of this element; Y was cleared before the launch
+        if (s != 0.f) atomicAdd(static_cast<float*>(p.Y) + row * p.ldy + q0 + q, s);
+      } else if (p.y_dtype == GRIM_F32) static_cast<float*>(p.Y)[row * p.ldy + q0 + q] = s;
       else static_cast<__nv_bfloat16*>(p.Y)[row * p.ldy + q0 + q] = __float2bfloat16_rn(s);
     }
     __syncthreads();
@@ -363,8 +448,10 @@ struct StreamPlan {
   size_t smem;
 };
 
-bool make_plan(const grim_bcr* h, int64_t N, StreamPlan& pl) {
+// staged: N > 1 with the current K slice of X in shared memory; nv = number of (virtual) bands the launch walks
+bool make_plan(const grim_bcr* h, int64_t N, StreamPlan& pl, bool staged = false, int64_t nv = 0) {
   if (h->device < 0 || !h->gemv_ok || !h->d_status || !h->d_runs || N < 1 || N > kSkinnyMaxN || h->nchunks == 0) return false;
+  if (nv <= 0) nv = h->nbr;
   const int BHc = h->bh <= 4 ? 4 : (h->bh <= 8 ? 8 : 16);
   const int esz = h->dtype == GRIM_F32 ? 4 : 2;
   pl.nq = N == 1 ? 1 : (N <= 4 ? 4 : (N <= 8 ? 8 : 16));
@@ -372,24 +459,26 @@ bool make_plan(const grim_bcr* h, int64_t N, StreamPlan& pl) {
   // the wide right-hand sides hold more accumulators: fewer warps
   pl.nw = pl.nq <= 4 ? 16 : 8;
   pl.passes = (int)((N + pl.nq - 1) / pl.nq);
-  pl.grid_x = (int)std::min<int64_t>(h->nbr, sm_count(h->device));
-  pl.nk_max = (int)((h->nbr + pl.grid_x - 1) / pl.grid_x);
+  pl.grid_x = (int)std::min<int64_t>(nv, sm_count(h->device));
+  pl.nk_max = (int)((nv + pl.grid_x - 1) / pl.grid_x);
   if (pl.nk_max > kSMaxBands) return false;
-  const int pb = std::max(1, kSPartBytes / (pl.nw * BHc * pl.nq * 4));
+  const int pb = std::max(1, part_bytes(staged) / (pl.nw * BHc * pl.nq * 4));
   auto up = [](size_t v, size_t a) { return (v + a - 1) / a * a; };
   // column words of a run, its values, the skipped elements in front, the rounding behind, and one warp's width
   // that a lane of a pruned row may read and discard
   pl.stage_bytes = (uint32_t)up((size_t)kSRun * 128 + (size_t)kRunValueBytes + 32 + 32 * esz, 128);
   const size_t budget = 227 * 1024;
   // the activation vector is staged in shared memory when it fits beside two stages per warp
-  for (int xs = (pl.nq == 1 && h->K * esz <= kSMaxXBytes) ? 1 : 0; xs >= 0; --xs) {
+  const size_t x_bytes = pl.nq == 1 ? (size_t)h->K * esz : (size_t)h->sl_rows * x_row_stride(pl.nq, esz);
+  if (staged && (pl.nq == 1 || x_bytes > (size_t)kSMaxXBytes)) return false;
+  for (int xs = ((staged || pl.nq == 1) && x_bytes <= (size_t)kSMaxXBytes) ? 1 : 0; xs >= (staged ? 1 : 0); --xs) {
     size_t off = up((size_t)pl.nw * kSMaxSlots * 12 + 16, 128);
     pl.off_band = (uint32_t)off;
-    off = up(off + (size_t)pl.nk_max * 12, 16);
+    off = up(off + (size_t)pl.nk_max * 16, 16);
     pl.off_part = (uint32_t)off;
     off = up(off + (size_t)pb * pl.nw * BHc * pl.nq * 4, 16);
     pl.off_x = (uint32_t)off;
-    if (xs) off += (size_t)h->K * esz;
+    if (xs) off += x_bytes;
     off = up(off, 128);
     pl.off_ring = (uint32_t)off;
     if (off + (size_t)2 * pl.nw * pl.stage_bytes > budget) continue;
@@ -417,11 +506,13 @@ cudaError_t launch_nq(const StreamParams& p, const StreamPlan& pl, cudaStream_t 
   switch (pl.nq) {
     case 1:
       return pl.xs ? launch_kernel<BH, 1, NW1, true, VT>(p, pl, s) : launch_kernel<BH, 1, NW1, false, VT>(p, pl, s);
-    case 4: return launch_kernel<BH, 4, NWS, false, VT>(p, pl, s);
-    case 8: return launch_kernel<BH, 8, 8, false, VT>(p, pl, s);
+    case 4:
+      return pl.xs ? launch_kernel<BH, 4, NWS, true, VT>(p, pl, s) : launch_kernel<BH, 4, NWS, false, VT>(p, pl, s);
+    case 8: return pl.xs ? launch_kernel<BH, 8, 8, true, VT>(p, pl, s) : launch_kernel<BH, 8, 8, false, VT>(p, pl, s);
     default:
       if (BH > 8) return cudaErrorInvalidValue;
-      return launch_kernel<(BH <= 8 ? BH : 8), 16, 8, false, VT>(p, pl, s);
+      return pl.xs ? launch_kernel<(BH <= 8 ? BH : 8), 16, 8, true, VT>(p, pl, s)
+                   : launch_kernel<(BH <= 8 ? BH : 8), 16, 8, false, VT>(p, pl, s);
   }
 }
 
@@ -442,15 +533,37 @@ bool stream_path_supported(const grim_bcr* h, int64_t N) {
 grim_status_t launch_stream(const grim_bcr* h, const void* X, int x_dtype, int64_t ldx, int64_t N, void* Y, int y_dtype,
                             int64_t ldy, cudaStream_t s) {
   StreamPlan pl;
-  if (!make_plan(h, N, pl)) return GRIM_ERR_UNSUPPORTED;
   if (x_dtype != h->dtype) return GRIM_ERR_DTYPE;
   StreamParams p;
   p.run_ptr = h->d_run_ptr; p.runs = h->d_runs; p.colwords = h->d_colwords;
   p.vals = static_cast<const uint8_t*>(h->d_gemv_vals);
   p.band_order = h->d_band_order; p.X = X; p.Y = Y; p.status = h->d_status; p.ldx = ldx; p.ldy = ldy;
   p.N = (int)N; p.nbr = (int)h->nbr; p.M = (int)h->M; p.K = (int)h->K; p.bh = h->bh; p.y_dtype = y_dtype;
+  p.slice_of = nullptr; p.sl_rows = h->sl_rows; p.accumulate = 0;
+  // 2 <= N <= 16: the rows of X a thread block needs are staged in shared memory - all of them when K is a single
+  // slice, else slice by slice on the slice-major copy of the layout, the slices' shares of Y added atomically
+  // (fp32 outputs; others gather the activations from L2 per band as before)
+  // (measured at 8192 x 8192, c = 4, fp32: N = 4: 68 us staged against 87 us gathered, N = 8: 122 against 150; at
+  // N = 16 the slices leave each band too few runs per warp and the gathered walk is faster: 94 against 165 us)
+  bool staged = false;
+  if (N >= 2 && N <= 8 && h->sl_rows > 0) {
+    if (h->sl_nslices <= 1) {
+      staged = make_plan(h, N, pl, true, h->nbr);
+    } else if (h->d_sl_runs && y_dtype == GRIM_F32 && make_plan(h, N, pl, true, h->sl_nslices * h->nbr)) {
+      staged = true;
+      p.run_ptr = h->d_sl_run_ptr; p.runs = h->d_sl_runs; p.colwords = h->d_sl_colwords;
+      p.vals = static_cast<const uint8_t*>(h->d_sl_vals);
+      p.band_order = h->d_sl_band_of; p.slice_of = h->d_sl_slice_of;
+      p.nbr = (int)(h->sl_nslices * h->nbr);
+      p.accumulate = 1;
+      if (cudaMemset2DAsync(Y, (size_t)ldy * 4, 0, (size_t)N * 4, (size_t)h->M, s) != cudaSuccess) return GRIM_ERR_CUDA;
+    }
+  }
+  if (!staged && !make_plan(h, N, pl)) return GRIM_ERR_UNSUPPORTED;
   const int esz = x_dtype == GRIM_F32 ? 4 : 2;
   p.vec_ok = (N % pl.nq == 0) && ldx % 4 == 0 && (reinterpret_cast<uintptr_t>(X) % (4 * esz)) == 0;
+  const int piece = pl.nq * esz >= 16 ? 16 : 8;
+  p.stage_vec = (N % pl.nq == 0) && pl.nq * esz >= 8 && (ldx * esz) % piece == 0 && (reinterpret_cast<uintptr_t>(X) % piece) == 0;
   p.nslots = pl.nslots; p.nk_max = pl.nk_max; p.stage_bytes = pl.stage_bytes;
   p.off_band = pl.off_band; p.off_part = pl.off_part; p.off_x = pl.off_x; p.off_ring = pl.off_ring;
   p.spin_limit = 1u << 22;
