@@ -304,6 +304,20 @@ class SpmmWorkload:
         self.rotating = len(self.sets) > 1
         self.per_step_events = True
         self._i = 0
+        # tile-shape search (Section 4.5): every handle times the candidate kernels / tiles for this request once and
+        # keeps the answer; the plain multiply below then uses it
+        self.tuned = None
+        for h, x, y in self.sets:
+            if self.bf16 and self.N > 16:
+                B.grim_bcr_reserve(h, self.N)  # workspace of the split tensor-core multiply (used when the grid is small)
+            self.tuned = B.grim_bcr_tune(h, x, y, reps=5)
+        torch.cuda.synchronize()
+        names = {1: "bcr_ffma_kernel", 2: "bcr_tc_kernel", 4: "bcr_spmm_kernel", 5: "bcr_tc2_kernel",
+                 3: "bcr_skinny_kernel" if self.tuned["tile_n"] == 1 else "bcr_stream_kernel"}
+        self.kernel = names.get(self.tuned["path"], self.kernel)
+        self.peak_kind = "tensor" if self.tuned["path"] in (2, 5) else "alu"
+        if self.peak_kind == "tensor":
+            self.kernel_bytes = float(i.value_bytes + i.index_bytes_tc + i.k_used * self.N * esz + self.M * self.N * 4)
 
     def step(self):
         h, x, y = self.sets[self._i % len(self.sets)]
@@ -860,6 +874,8 @@ def record_of(bench, wl, label, ms, parity):
                t_hbm_us=roof["t_hbm_us"], t_flop_us=roof["t_flop_us"], parity=parity)
     if "layers" in roof:
         rec["layers"] = roof["layers"]
+    if getattr(wl, "tuned", None):
+        rec["tuned"] = dict(path=wl.tuned["path"], tile_n=wl.tuned["tile_n"])
     if isinstance(wl, GruWorkload):
         rec["bound"] = "latency (hbm figure: bytes moved once)"
         rec["us_per_time_step"] = ms * 1e3 / wl.T
