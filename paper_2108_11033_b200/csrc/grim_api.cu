@@ -137,14 +137,16 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   float best_t = -1.f;
   grim_tune_t cand_best{};
   // candidates: (path, tile_n); a candidate that cannot take the request is skipped
-  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {2, 0}, {5, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
+  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {1, 8}, {1, 9}, {2, 0}, {5, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
   for (const auto& cd : cand) {
     grim_tune_t c{};
     c.path = cd[0];
     c.tile_n = cd[1];
     if (c.path == 3 && X->cols > kSkinnyMaxN) continue;
     if (c.path == 4 && c.tile_n > 16 && c.tile_n / 2 >= X->cols) continue;  // idle lanes only
-    if (c.path == 1 && c.tile_n > (h->bh <= 4 ? 4 : (h->bh <= 8 ? 2 : 1))) continue;
+    // CUDA-core kernel: 1, 2, 4 = bands per warp; 8, 9 = two 128-column pieces per lane with one or two bands per warp
+    if (c.path == 1 && c.tile_n <= 4 && c.tile_n > (h->bh <= 4 ? 4 : (h->bh <= 8 ? 2 : 1))) continue;
+    if (c.path == 1 && c.tile_n >= 8 && (h->bh > (c.tile_n == 8 ? 8 : 4) || X->cols <= 128)) continue;
     st = run_spmm(h, X, Y, &c, s);  // warm-up
     if (st == GRIM_ERR_UNSUPPORTED) { st = GRIM_OK; continue; }
     if (st != GRIM_OK) break;
