@@ -94,7 +94,8 @@ typedef struct {
   int32_t tile_n;  /* path 4: output columns per thread block (16, 32, 64 or 128);
                       path 1: groups of 16 row bands per thread block (1, 2 or 4) with 128 output columns per
                       thread block, or 8 / 9 = 256 output columns per thread block (a lane owns two 4-column
-                      pieces) with 1 / 2 groups (block height <= 8 / <= 4); plus 256 x the number of
+                      pieces) with 1 / 2 groups (block height <= 8 / <= 4), or 17 / 18 / 20 = the 16-column tile
+                      for N <= 16 (a lane owns one column) with 1 / 2 / 4 groups; plus 256 x the number of
                       thread blocks that share a tile's block columns (split multiply, 1 - 8);
                       path 3: 1 = values staged in registers, 2 = values streamed through shared memory by bulk
                       asynchronous copies (persistent thread blocks), 0 = the streaming variant when it fits */

@@ -56,6 +56,14 @@ grim_status_t run_spmm(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, const g
     if (!tc2_path_supported(h, a)) return GRIM_ERR_UNSUPPORTED;
     return launch_spmm_tc2(h, a, s);
   }
+  // 8 <= N <= 16, measured at 8192 x 8192 and 4096 x 4096: bf16 handles are fastest on the tensor-core tile (56 us
+  // split over K against 102 us on the lane-per-column kernel), fp32 handles with blocks of 8 rows or more on the
+  // CUDA-core kernel's 16-column tile (93 against 98 - 124 us); narrower right-hand sides stay on the lane-per-column
+  // kernel
+  if (path == 0 && X->cols >= 8 && X->cols <= kSkinnyMaxN) {
+    if (tc_path_supported(h, a) && h->tc_mtiles >= 8) return launch_spmm_tc(h, a, s);
+    if (h->dtype == GRIM_F32 && h->bh >= 8 && ffma_path_supported(h, a)) return launch_ffma(h, a, s);
+  }
   if (path == 3 || (path == 0 && X->cols <= kSkinnyMaxN && h->gemv_ok)) {
     // tile_n = 1 under path 3 asks for the register-staged variant; otherwise the streaming one runs when it can
     if (!(path == 3 && a.tile_n == 1) && stream_path_supported(h, X->cols))
@@ -137,7 +145,7 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   float best_t = -1.f;
   grim_tune_t cand_best{};
   // candidates: (path, tile_n); a candidate that cannot take the request is skipped
-  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {1, 8}, {1, 9}, {2, 0}, {5, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
+  const int cand[][2] = {{1, 1}, {1, 2}, {1, 4}, {1, 8}, {1, 9}, {1, 17}, {1, 18}, {1, 20}, {2, 0}, {5, 0}, {3, 1}, {3, 2}, {4, 16}, {4, 32}, {4, 64}, {4, 128}};
   for (const auto& cd : cand) {
     grim_tune_t c{};
     c.path = cd[0];
@@ -146,7 +154,10 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
     if (c.path == 4 && c.tile_n > 16 && c.tile_n / 2 >= X->cols) continue;  // idle lanes only
     // CUDA-core kernel: 1, 2, 4 = bands per warp; 8, 9 = two 128-column pieces per lane with one or two bands per warp
     if (c.path == 1 && c.tile_n <= 4 && c.tile_n > (h->bh <= 4 ? 4 : (h->bh <= 8 ? 2 : 1))) continue;
-    if (c.path == 1 && c.tile_n >= 8 && (h->bh > (c.tile_n == 8 ? 8 : 4) || X->cols <= 128)) continue;
+    if (c.path == 1 && (c.tile_n == 8 || c.tile_n == 9) && (h->bh > (c.tile_n == 8 ? 8 : 4) || X->cols <= 128)) continue;
+    // ... 17, 18, 20 = the narrow tile (at most 16 columns) with 1, 2, 4 bands per warp
+    if (c.path == 1 && c.tile_n >= 17 && (X->cols > 16 || c.tile_n - 16 > (h->bh <= 8 ? 4 : 2))) continue;
+    if (c.path == 1 && c.tile_n < 17 && X->cols <= 16) continue;
     st = run_spmm(h, X, Y, &c, s);  // warm-up
     if (st == GRIM_ERR_UNSUPPORTED) { st = GRIM_OK; continue; }
     if (st != GRIM_OK) break;

@@ -26,11 +26,17 @@ namespace {
 
 constexpr int kFThreads = 512;
 constexpr int kFWarps = 16;
-constexpr int kTN = 128;          // output columns per thread block
+constexpr int kTN = 128;          // output columns per thread block and piece
+constexpr int kNarrowTN = 16;     // ... of the narrow variant
 constexpr int kStages = 4;        // ring slots
 constexpr int kAhead = 2;         // stages requested ahead of the one being multiplied
+// The narrow variant's stages are small (a 2 KiB slab and a few KiB of records): with two in flight a thread block
+// moves about 7 KiB per memory latency, far below its share of the bandwidth; its ring is deeper.
+constexpr int kNarrowStages = 8;
+constexpr int kNarrowAhead = 6;
+constexpr int kMaxRing = 8;
 constexpr int kJlistCap = 2048;   // block columns per matrix the stage list can hold
-constexpr int kHdrBytes = (128 + kStages * 16 + kJlistCap * 2 + 127) / 128 * 128;  // barriers, flags, per-slot blob sizes, stage list
+constexpr int kHdrBytes = (192 + kMaxRing * 16 + kJlistCap * 2 + 127) / 128 * 128;  // barriers, flags, per-slot blob sizes, stage list
 
 enum { kModeTma = 0, kModeGather = 1 };
 
@@ -138,17 +144,29 @@ __device__ __forceinline__ float2 unpack2(unsigned long long v) {
   return f;
 }
 
+// One slab element (narrow tiles).
+__device__ __forceinline__ float ld_x1(const float* slab, unsigned col, int q, int sld) { return slab[col * sld + q]; }
+__device__ __forceinline__ float ld_x1(const __nv_bfloat16* slab, unsigned col, int q, int sld) {
+  return __uint_as_float((unsigned)reinterpret_cast<const unsigned short*>(slab)[col * sld + q] << 16);
+}
+
 // CW: 128-column pieces of the output tile per lane (a lane owns four columns of each piece).
+// CW = 0 is the narrow tile for right-hand sides of at most 16 columns: a lane owns ONE output column, and the two
+// halves of a warp split the kept columns of a chunk between them (lanes 0-15 the first four, lanes 16-31 the
+// other four; their sums meet in one shuffle at the end).  The kept values then stream through shared memory once
+// and each costs a quarter of a broadcast load and one FMA per lane - no per-lane gathers from global memory.
 template <int BH, int BPW, int CW, typename XT, int MODE>
-__global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_constant__ CUtensorMap tmX, const FParams p) {
-  constexpr int TN = kTN * CW;  // output columns per thread block
+__global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(const __grid_constant__ CUtensorMap tmX, const FParams p) {
+  constexpr bool NARROW = CW == 0;
+  constexpr int NS = NARROW ? kNarrowStages : kStages, AH = NARROW ? kNarrowAhead : kAhead;  // ring slots, stages in flight
+  constexpr int TN = NARROW ? kNarrowTN : kTN * CW;  // output columns per thread block
   extern __shared__ __align__(128) uint8_t smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
-  uint64_t* empty = full + kStages;
-  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 64);
-  int* s_nst = reinterpret_cast<int*>(smem + 68);
-  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 128);               // [kStages][4] blob bytes per band group
-  const uint16_t* jlist = reinterpret_cast<const uint16_t*>(smem + 128 + kStages * 16);  // non-empty block columns, ascending
+  uint64_t* empty = full + kMaxRing;
+  volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 128);
+  int* s_nst = reinterpret_cast<int*>(smem + 132);
+  uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 192);               // [ring slot][4] blob bytes per band group
+  const uint16_t* jlist = reinterpret_cast<const uint16_t*>(smem + 192 + kMaxRing * 16);  // non-empty block columns, ascending
   uint8_t* slots = smem + kHdrBytes;
   const uint32_t slot_bytes = p.slab_bytes + BPW * p.blob_stride;
   const int sld = MODE == kModeTma ? TN : p.slab_ld;
@@ -176,7 +194,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
     if (lane == 0) {
       *s_nst = n;
       *s_abort = 0;
-      for (int s = 0; s < kStages; ++s) {
+      for (int s = 0; s < NS; ++s) {
         mbar_init(full + s, MODE == kModeTma ? 1u : (unsigned)kFThreads);
         mbar_init(empty + s, kFWarps);
       }
@@ -215,7 +233,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
 
   // Requests stage n (the n-th non-empty block column) into its ring slot.
   auto request = [&](int n) {
-    const int slot = n % kStages;
+    const int slot = n % NS;
     const int j = jlist[n];
     uint8_t* base = slots + (size_t)slot * slot_bytes;
     if (MODE == kModeTma) {
@@ -287,36 +305,40 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
   };
 
   // accumulators as packed pairs of neighbouring columns: [band][row][pair]; pairs 2c, 2c + 1 belong to piece c
-  unsigned long long acc[BPW][BH][2 * CW];
+  unsigned long long acc[BPW][BH][NARROW ? 1 : 2 * CW];
+  float nacc[BPW][NARROW ? BH : 1];  // narrow tiles: one column per lane
 #pragma unroll
   for (int b = 0; b < BPW; ++b)
 #pragma unroll
-    for (int r = 0; r < BH; ++r)
+    for (int r = 0; r < BH; ++r) {
 #pragma unroll
-      for (int c = 0; c < 2 * CW; ++c) acc[b][r][c] = 0ull;
+      for (int c = 0; c < (NARROW ? 1 : 2 * CW); ++c) acc[b][r][c] = 0ull;
+      if (NARROW) nacc[b][NARROW ? r : 0] = 0.f;
+    }
   const int lane4 = lane * 4;
+  const int nhalf = lane >> 4, nq = lane & 15;  // narrow tiles: which four columns of a chunk, which output column
 
-  // prologue: the first kAhead stages go into fresh slots
-  for (int n = 0; n < kAhead && n < nst; ++n)
+  // prologue: the first AH stages go into fresh slots
+  for (int n = 0; n < AH && n < nst; ++n)
     if (MODE != kModeTma || tid == 0) request(n);
 
   bool failed = false;
   for (int n = 0; n < nst; ++n) {
-    // ---- producer duty: request stage n + kAhead; its slot was last used by stage n + kAhead - kStages
-    const int m = n + kAhead;
+    // ---- producer duty: request stage n + AH; its slot was last used by stage n + AH - NS
+    const int m = n + AH;
     if (m < nst) {
       const bool mine = MODE != kModeTma || (warp == (n % kFWarps) && lane == 0);
       if (mine) {
         bool ok = true;
-        if (m >= kStages) ok = mbar_wait(empty + m % kStages, (unsigned)((m / kStages - 1) & 1), p.spin_limit, s_abort);
+        if (m >= NS) ok = mbar_wait(empty + m % NS, (unsigned)((m / NS - 1) & 1), p.spin_limit, s_abort);
         if (ok) request(m);
         else failed = true;
       }
     }
     if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     // ---- wait for stage n
-    const int slot = n % kStages;
-    if (!mbar_wait(full + slot, (unsigned)((n / kStages) & 1), p.spin_limit, s_abort)) failed = true;
+    const int slot = n % NS;
+    if (!mbar_wait(full + slot, (unsigned)((n / NS) & 1), p.spin_limit, s_abort)) failed = true;
     if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     const uint8_t* base = slots + (size_t)slot * slot_bytes;
     const XT* slab = reinterpret_cast<const XT*>(base);
@@ -333,12 +355,36 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
       const float4* wp = reinterpret_cast<const float4*>(rec + ((8 + nch * kRcChunk + 15) & ~15));
       // The slab rows of KS kept columns are held in registers at a time: all eight of a chunk for one piece per
       // lane, four when a lane owns two pieces (the registers go to the accumulators instead).
-      constexpr int KS = kRcChunk / CW;
+      if constexpr (NARROW) {
+        const float4* wq0 = wp + nhalf;
+        for (int ch = 0; ch < nch; ++ch) {
+          const uint2 cc = *reinterpret_cast<const uint2*>(cols + ch * kRcChunk);
+          const unsigned c4 = nhalf ? cc.y : cc.x;
+          float x[4];
+#pragma unroll
+          for (int e = 0; e < 4; ++e) x[e] = ld_x1(slab, (c4 >> (8 * e)) & 0xFFu, nq, sld);
+          const float4* wq = wq0;
+#pragma unroll
+          for (int r = 0; r < BH; ++r) {
+            if ((rm >> r) & 1u) {
+              const float4 w = *wq;
+              wq += 2;
+              // two chains of two instead of one of four: rows cannot overlap (each sits behind its own branch)
+              const float t = fmaf(w.y, x[1], w.x * x[0]);
+              const float u = fmaf(w.w, x[3], w.z * x[2]);
+              nacc[b][NARROW ? r : 0] += t + u;
+            }
+          }
+          wq0 += 2 * kr;
+        }
+        continue;
+      }
+      constexpr int KS = kRcChunk / (NARROW ? 1 : CW);
       for (int ch = 0; ch < nch; ++ch) {
         const uint2 cc = *reinterpret_cast<const uint2*>(cols + ch * kRcChunk);
 #pragma unroll
         for (int hs = 0; hs < kRcChunk / KS; ++hs) {
-          ulonglong2 x[KS][CW];
+          ulonglong2 x[KS][NARROW ? 1 : CW];
 #pragma unroll
           for (int e = 0; e < KS; ++e) {
             const int idx = hs * KS + e;
@@ -384,13 +430,48 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
   __syncthreads();
   if (*s_abort) {
     if (tid == 0)
-      for (int s = 0; s < kStages; ++s)
+      for (int s = 0; s < NS; ++s)
         for (unsigned i = 0; i < 4096u && !mbar_try_wait(full + s, 0) && !mbar_try_wait(full + s, 1); ++i) {}
     return;
   }
 
   // ---- epilogue: bias, activation, store every row of the band (rows kept by no block are +0)
   const int64_t ohw = (int64_t)a.OH * a.OW;
+  if constexpr (NARROW) {
+    const int64_t q = q0 + nq;
+    int64_t qbase = 0;  // offset of column q in row 0 of the output
+    if (q < a.ncols) {
+      if (a.conv) {
+        const int64_t img = q / ohw;
+        qbase = img * p.M * ohw + (q - img * ohw);
+      } else {
+        qbase = q * a.y_sq;
+      }
+    }
+    const int64_t rstride = a.conv ? ohw : a.y_sr;
+#pragma unroll
+    for (int b = 0; b < BPW; ++b) {
+      const int pos = (g0 + b) * kRcBands + warp;
+      if (pos >= p.nbr) continue;  // (uniform over the warp: the shuffles below are taken by all lanes or none)
+      const int band = p.band_order[pos];
+#pragma unroll
+      for (int r = 0; r < BH; ++r) {
+        float t = nacc[b][NARROW ? r : 0];
+        t += __shfl_xor_sync(0xffffffffu, t, 16);
+        const int64_t row = (int64_t)band * p.bh + r;
+        if (r >= p.bh || row >= p.M || nhalf != 0 || q >= a.ncols) continue;
+        const int64_t off = row * rstride + qbase;
+        if (p.ksplit > 1) {
+          if (t != 0.f) atomicAdd(static_cast<float*>(a.Y) + off, t);
+          continue;
+        }
+        t += a.bias ? __ldg(a.bias + row) : 0.f;
+        if (a.relu) t = fmaxf(t, 0.f);
+        if (a.y_dtype == GRIM_F32) static_cast<float*>(a.Y)[off] = t;
+        else static_cast<__nv_bfloat16*>(a.Y)[off] = __float2bfloat16_rn(t);
+      }
+    }
+  } else {
 #pragma unroll
   for (int cp = 0; cp < CW; ++cp) {
   const int64_t q = q0 + cp * kTN + lane4;
@@ -476,6 +557,7 @@ __global__ void __launch_bounds__(kFThreads, 1) bcr_ffma_kernel(const __grid_con
     }
   }
   }  // pieces
+  }
 }
 
 // The driver's tensor-map encoder, looked up through the runtime so that the library does not link
@@ -548,6 +630,11 @@ cudaError_t launch_variant(const CUtensorMap& tm, const FParams& p, size_t smem,
 // The accumulators of a lane take BH * BPW * CW * 4 registers: at most 64.
 template <int BH, typename XT, int MODE>
 cudaError_t launch_bpw(int bpw, int cw, const CUtensorMap& tm, const FParams& p, size_t smem, dim3 grid, cudaStream_t s) {
+  if (cw == 0) {
+    if (BH <= 8 && bpw == 4) return launch_variant<BH, (BH <= 8 ? 4 : 1), 0, XT, MODE>(tm, p, smem, grid, s);
+    if (bpw == 2) return launch_variant<BH, 2, 0, XT, MODE>(tm, p, smem, grid, s);
+    return launch_variant<BH, 1, 0, XT, MODE>(tm, p, smem, grid, s);
+  }
   if (cw == 2) {
     if (BH <= 4 && bpw == 2) return launch_variant<BH, (BH <= 4 ? 2 : 1), (BH <= 4 ? 2 : 1), XT, MODE>(tm, p, smem, grid, s);
     if (BH <= 8) return launch_variant<BH, 1, (BH <= 8 ? 2 : 1), XT, MODE>(tm, p, smem, grid, s);
@@ -567,11 +654,12 @@ cudaError_t launch_bh(int BHc, int bpw, int cw, const CUtensorMap& tm, const FPa
 
 constexpr size_t kSmemBudget = 220 * 1024;
 
-int slab_ld_for(const SpmmArgs& a, bool tma, int cw) { return (!tma && !a.conv && a.x_sq != 1) ? kTN * cw + 4 : kTN * cw; }
+int tile_cols(int cw) { return cw ? kTN * cw : kNarrowTN; }
+int slab_ld_for(const SpmmArgs& a, bool tma, int cw) { return (!tma && !a.conv && a.x_sq != 1) ? tile_cols(cw) + 4 : tile_cols(cw); }
 size_t slab_bytes_for(const grim_bcr* h, int sld, int esz) { return ((size_t)h->bw * sld * esz + 127) & ~size_t(127); }
-size_t smem_need(const grim_bcr* h, int bpw, int esz, int sld = kTN + 4) {
+size_t smem_need(const grim_bcr* h, int bpw, int esz, int sld = kTN + 4, int stages = kStages) {
   const size_t blob_stride = ((size_t)h->rc_max_blob + 127) & ~size_t(127);
-  return kHdrBytes + (size_t)kStages * (slab_bytes_for(h, sld, esz) + bpw * blob_stride);
+  return kHdrBytes + (size_t)stages * (slab_bytes_for(h, sld, esz) + bpw * blob_stride);
 }
 
 }  // namespace
@@ -595,15 +683,18 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   // warp: the slab addresses, the weight loads and the row tests of a block are then shared by twice the FMAs.
   int bpw = BHc == 4 ? 4 : (BHc == 8 ? 2 : 1), cw = 1;
   const int tn = a.tile_n % 256;
-  auto tiles_of = [&](int bpw_, int cw_) { return ((a.ncols + kTN * cw_ - 1) / (kTN * cw_)) * ((h->rc_groups + bpw_ - 1) / bpw_); };
-  auto fits = [&](int bpw_, int cw_) { return smem_need(h, bpw_, esz, kTN * cw_ + 4) <= kSmemBudget; };
+  auto tiles_of = [&](int bpw_, int cw_) { return ((a.ncols + tile_cols(cw_) - 1) / tile_cols(cw_)) * ((h->rc_groups + bpw_ - 1) / bpw_); };
+  auto fits = [&](int bpw_, int cw_) { return smem_need(h, bpw_, esz, tile_cols(cw_) + 4, cw_ ? kStages : kNarrowStages) <= kSmemBudget; };
   if (tn == 1 || tn == 2 || tn == 4) {
     bpw = std::min(tn, bpw);
   } else if (tn == 8 && BHc <= 8) {
     cw = 2; bpw = 1;
   } else if (tn == 9 && BHc <= 4) {
     cw = 2; bpw = 2;
-
+  } else if (tn == 17 || tn == 18 || tn == 20) {
+    cw = 0; bpw = std::min(tn - 16, BHc <= 8 ? 4 : 2);
+  } else if (a.ncols <= kNarrowTN) {
+    cw = 0; bpw = 1;
   } else {
     // (measured at 8192 x 8192 and 4096 x 4096, N = 256 and 1024: two pieces per lane are 10 - 20 % faster than
     // any one-piece variant, also where they leave the grid smaller than the GPU - the split below then applies)
@@ -615,7 +706,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
     }
   }
   if (!fits(bpw, cw)) return GRIM_ERR_UNSUPPORTED;
-  const int64_t qtiles = (a.ncols + kTN * cw - 1) / (kTN * cw);
+  const int64_t qtiles = (a.ncols + tile_cols(cw) - 1) / tile_cols(cw);
   const int64_t gy = (h->rc_groups + bpw - 1) / bpw;
   if (gy > 65535) return GRIM_ERR_UNSUPPORTED;
   // too few tiles for the GPU: split the block columns over several thread blocks (fp32 output only)
@@ -625,6 +716,9 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
     ksplit = (int)std::min<int64_t>(std::min<int64_t>(8, sms / (qtiles * gy)), std::max<int64_t>(1, h->nbc / 4));
     if (ksplit < 1) ksplit = 1;
   }
+  // narrow tiles are light (two thread blocks share an SM): as many parts as still run in one wave
+  if (cw == 0 && split_ok && qtiles * gy < 2 * sms)
+    ksplit = (int)std::max<int64_t>(1, std::min<int64_t>(std::min<int64_t>(8, 2 * sms / (qtiles * gy)), h->nbc / 4));
   if (a.tile_n >= 256) ksplit = split_ok ? std::max(1, std::min(8, a.tile_n / 256)) : 1;  // test / tuning override
 
   FParams p;
@@ -643,7 +737,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
   if (tma) {
     const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
     const cuuint64_t strides[1] = {(cuuint64_t)(a.x_sk * esz)};
-    const cuuint32_t box[2] = {(cuuint32_t)(kTN * cw), (cuuint32_t)h->bw};
+    const cuuint32_t box[2] = {(cuuint32_t)tile_cols(cw), (cuuint32_t)h->bw};
     const cuuint32_t estr[2] = {1, 1};
     EncodeTiledFn encode = encode_tiled_fn();
     if (!encode) return GRIM_ERR_CUDA;
@@ -653,7 +747,7 @@ grim_status_t launch_ffma(const grim_bcr* h, const SpmmArgs& a, cudaStream_t s) 
                                               CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) return GRIM_ERR_CUDA;
   }
-  const size_t smem = smem_need(h, bpw, esz, p.slab_ld);
+  const size_t smem = smem_need(h, bpw, esz, p.slab_ld, cw ? kStages : kNarrowStages);
   dim3 grid((unsigned)qtiles, (unsigned)gy, (unsigned)ksplit);
   cudaError_t e = cudaSuccess;
   if (ksplit > 1 && !(a.y_prefilled && !a.relu)) {

@@ -171,18 +171,6 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
 
-  // Requests the packed record of K tile k into record slot rs; one thread.
-  auto request_record = [&](int k, int rs) {
-    uint32_t bytes = 0, off = 0;
-    if (has_tile) {
-      const RcStage se = p.stage[(int64_t)tile * p.nkt + k];
-      bytes = se.bytes; off = se.off16;
-    }
-    s_meta[rs] = bytes;
-    mbar_arrive_expect_tx(rec_full + rs, bytes);
-    if (bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)off * 16, bytes, rec_full + rs);
-  };
-
   bool failed = false;
   int fail_site = 0;
   Im2colCtx im;
@@ -266,11 +254,22 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
     // ------------------------------------------------------------------ packed records, a ring of nr slots
     // (their own thread: the table entry is a global load and the request a handful of dependent shared-memory
     // accesses, which would otherwise sit in the expansion warps' critical path)
-    if (lane == 0) {
-      for (int kt = 0; kt < nkt; ++kt) {
-        const int rs = kt % nr;
-        if (kt >= nr && !mbar_wait<true>(rec_free + rs, (unsigned)((kt / nr - 1) & 1), p.spin_limit, s_abort, 20)) { failed = true, fail_site = 7; break; }
-        request_record(kt, rs);
+    // The table entries are read 32 K tiles at a time, one per lane, so that no request waits for a global load.
+    for (int kt0 = 0; kt0 < nkt && !failed; kt0 += 32) {
+      RcStage mine;
+      mine.off16 = 0; mine.bytes = 0;
+      if (has_tile && kt0 + lane < nkt) mine = p.stage[(int64_t)tile * p.nkt + kt0 + lane];
+      const int n = nkt - kt0 < 32 ? nkt - kt0 : 32;
+      for (int i = 0; i < n; ++i) {
+        const int kt = kt0 + i, rs = kt % nr;
+        const uint32_t bytes = __shfl_sync(0xffffffffu, mine.bytes, i), off = __shfl_sync(0xffffffffu, mine.off16, i);
+        if (kt >= nr && !__all_sync(0xffffffffu, mbar_wait<true>(rec_free + rs, (unsigned)((kt / nr - 1) & 1), p.spin_limit, s_abort, 20))) { failed = true, fail_site = 7; break; }
+        if (lane == 0) {
+          s_meta[rs] = bytes;
+          mbar_arrive_expect_tx(rec_full + rs, bytes);
+          if (bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)off * 16, bytes, rec_full + rs);
+        }
+        __syncwarp();
       }
     }
   } else if (CONV && warp > kRecWarp) {

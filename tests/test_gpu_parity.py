@@ -125,6 +125,35 @@ def test_register_tiled_kernel_explicit(B, case, bf16):
     check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=groups, path=1, flags=1)
 
 
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("case", [(512, 768, 8, 32, 8, 328), (512, 768, 8, 32, 8, 600), (300, 520, 4, 16, 8, 328),
+                                  (300, 520, 4, 16, 9, 515), (96, 153, 8, 32, 8, 257), (64, 27, 8, 32, 8, 1024)])
+def test_register_tiled_kernel_two_pieces_per_lane(B, case, bf16):
+    """The same kernel with 256-column tiles (a lane owns two 4-column pieces; tile_n 8 and 9), on column counts that
+    leave the second piece partly or wholly empty in the last tile."""
+    M, K, bh, bw, tile_n, N = case
+    W = gen.dense_weight(M, K, seed=173)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=174, empty_frac=0.1)
+    mask[: 2 * bh] = 0
+    X = gen.normal_f32((K, N), 1.0, 175, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=tile_n, path=1, flags=1)
+
+
+@pytest.mark.parametrize("bf16", [False, True])
+@pytest.mark.parametrize("case", [(512, 768, 8, 32, 17, 16), (512, 768, 8, 32, 18, 12), (512, 768, 8, 32, 20, 9),
+                                  (300, 520, 4, 16, 20, 16), (260, 700, 16, 64, 17, 16), (96, 153, 8, 32, 17, 5),
+                                  (64, 27, 8, 32, 17, 1), (2048, 1024, 8, 32, 17 + 256 * 3, 16)])
+def test_register_tiled_kernel_narrow_tile(B, case, bf16):
+    """The 16-column tile for N <= 16 (a lane owns one column, the halves of a warp split each chunk's kept columns;
+    tile_n 17, 18, 20 = 1, 2, 4 band groups per thread block), unsplit and split over the block columns."""
+    M, K, bh, bw, tile_n, N = case
+    W = gen.dense_weight(M, K, seed=183)
+    mask = gen.bcr_mask(M, K, bh, bw, compression=6, dist="zipf", seed=184, empty_frac=0.1)
+    mask[: 2 * bh] = 0
+    X = gen.normal_f32((K, N), 1.0, 185, 0)
+    check_spmm(B, W, mask, X, bh, bw, bf16=bf16, tile_n=tile_n, path=1, flags=1)
+
+
 @pytest.mark.parametrize("row_tiles", [1, 2])
 def test_tensor_core_row_tiles_per_block(B, row_tiles):
     """One or two 128-row tiles per thread block (two share every X tile), on a row count that leaves the last
