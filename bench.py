@@ -276,7 +276,10 @@ class SpmmWorkload:
         self.B, self.torch = B, torch
         s = self.s
         dt = B.GRIM_BF16 if self.bf16 else B.GRIM_F32
-        self.pack_flags = B.GRIM_PACK_REORDER | (B.GRIM_PACK_NARROW_ONLY if self.N <= 16 else B.GRIM_PACK_WIDE_ONLY)
+        # one regime's device layouts where only that regime's kernels can take the request; 8 <= N <= 16 is served by
+        # kernels of both regimes (the tile search decides), so those handles keep every layout
+        self.pack_flags = B.GRIM_PACK_REORDER | (B.GRIM_PACK_NARROW_ONLY if self.N < 8 else
+                                                 (B.GRIM_PACK_WIDE_ONLY if self.N > 16 else 0))
         self.h = B.grim_bcr_pack(s["W"], s["mask"], self.bh, self.bw, dt, self.pack_flags)
         tdt = torch.bfloat16 if self.bf16 else torch.float32
         self.x_host = torch.from_numpy(s["X"]).to(tdt).pin_memory()
@@ -308,9 +311,10 @@ class SpmmWorkload:
         # keeps the answer; the plain multiply below then uses it
         self.tuned = None
         for h, x, y in self.sets:
-            if self.bf16 and self.N > 16:
+            if self.bf16 and self.N >= 8:
                 B.grim_bcr_reserve(h, self.N)  # workspace of the split tensor-core multiply (used when the grid is small)
-            self.tuned = B.grim_bcr_tune(h, x, y, reps=5)
+            # operands that are streamed from HBM every step (the rotating sets) are tuned with a cold L2 as well
+            self.tuned = B.grim_bcr_tune(h, x, y, reps=-5 if self.rotating else 5)
         torch.cuda.synchronize()
         names = {1: "bcr_ffma_kernel", 2: "bcr_tc_kernel", 4: "bcr_spmm_kernel", 5: "bcr_tc2_kernel",
                  3: "bcr_skinny_kernel" if self.tuned["tile_n"] == 1 else "bcr_stream_kernel"}

@@ -216,7 +216,11 @@ grim_status_t grim_bcr_spmm_ex(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y,
  * and returns the fastest in *best (Section 4.5: per-kernel tuning of tile shape; the paper's
  * genetic search is replaced by a small fixed candidate set).  Y is overwritten.  The answer is also
  * stored in the handle: later grim_bcr_spmm calls with N in the same power-of-two bucket and the same
- * dtypes use it. */
+ * dtypes use it.  reps > 0: every candidate is launched reps times back to back (operands that fit the L2 cache are
+ * read from it - right for small matrices called in a loop); reps < 0: -reps launches, each after the L2 cache has
+ * been flushed by clearing a 256 MiB scratch (right for operands that are streamed from HBM every time; the
+ * scratch is allocated and freed inside the call; GRIM_ERR_ALLOC when it cannot be had); 0 = 5.  A set-up call:
+ * it synchronises and, with reps < 0, allocates. */
 grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_mat_t* Y, int reps, grim_tune_t* best,
                             float* best_ms, grim_stream_t stream);
 

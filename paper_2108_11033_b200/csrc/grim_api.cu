@@ -138,10 +138,15 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
   if (!best) return GRIM_ERR_INVALID_ARG;
   grim_status_t st = check_mats(h, X, Y);
   if (st != GRIM_OK) return st;
-  if (reps <= 0) reps = 5;
+  const bool cold = reps < 0;  // flush the L2 cache before every timed launch
+  if (reps < 0) reps = -reps;
+  if (reps == 0) reps = 5;
   cudaStream_t s = (cudaStream_t)stream;
+  constexpr size_t kFlushBytes = size_t(256) << 20;
+  void* flush = nullptr;
+  if (cold && cudaMalloc(&flush, kFlushBytes) != cudaSuccess) { cudaGetLastError(); return GRIM_ERR_ALLOC; }
   cudaEvent_t e0, e1;
-  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return GRIM_ERR_CUDA;
+  if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) { cudaFree(flush); return GRIM_ERR_CUDA; }
   float best_t = -1.f;
   grim_tune_t cand_best{};
   // candidates: (path, tile_n); a candidate that cannot take the request is skipped
@@ -161,18 +166,36 @@ extern "C" grim_status_t grim_bcr_tune(grim_bcr_t h, const grim_mat_t* X, grim_m
     st = run_spmm(h, X, Y, &c, s);  // warm-up
     if (st == GRIM_ERR_UNSUPPORTED) { st = GRIM_OK; continue; }
     if (st != GRIM_OK) break;
-    cudaEventRecord(e0, s);
-    for (int r = 0; r < reps && st == GRIM_OK; ++r) st = run_spmm(h, X, Y, &c, s);
-    cudaEventRecord(e1, s);
-    if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
     float ms = 0.f;
-    cudaEventElapsedTime(&ms, e0, e1);
+    if (!cold) {
+      cudaEventRecord(e0, s);
+      for (int r = 0; r < reps && st == GRIM_OK; ++r) st = run_spmm(h, X, Y, &c, s);
+      cudaEventRecord(e1, s);
+      if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
+      cudaEventElapsedTime(&ms, e0, e1);
+    } else {
+      for (int r = 0; r < reps && st == GRIM_OK; ++r) {
+        cudaMemsetAsync(flush, r & 1, kFlushBytes, s);
+        cudaEventRecord(e0, s);
+        st = run_spmm(h, X, Y, &c, s);
+        cudaEventRecord(e1, s);
+        if (st != GRIM_OK || cudaEventSynchronize(e1) != cudaSuccess) { st = st == GRIM_OK ? GRIM_ERR_CUDA : st; break; }
+        float t = 0.f;
+        cudaEventElapsedTime(&t, e0, e1);
+        ms += t;
+      }
+      if (st != GRIM_OK) break;
+    }
     ms /= reps;
     if (best_t < 0.f || ms < best_t) { best_t = ms; cand_best = c; }
   }
   if (st == GRIM_OK && best_t < 0.f) st = GRIM_ERR_UNSUPPORTED;
   cudaEventDestroy(e0);
   cudaEventDestroy(e1);
+  if (flush) {
+    cudaStreamSynchronize(s);
+    cudaFree(flush);
+  }
   if (st != GRIM_OK) return st;
   *best = cand_best;
   if (best_ms) *best_ms = best_t;

@@ -1,18 +1,25 @@
-// Register-tiled CUDA-core kernel for Y = W * X with N > 16 (Sections 3.1, 4.2 - 4.5).
+// Register-tiled CUDA-core kernel for Y = W * X (Sections 3.1, 4.2 - 4.5): N > 16 and, with its narrow tile, N <= 16.
 //
-// One thread block (16 warps) owns BPW groups of 16 row bands and a tile of 128 output columns and walks
-// the block columns.  Per block column a slab of X (bw rows x 128 columns) is brought into shared memory
+// One thread block (16 warps) owns BPW groups of 16 row bands and a tile of 128 or 256 output columns and walks
+// the block columns.  Per block column a slab of X (bw rows x the tile's columns) is brought into shared memory
 // once - by TMA when X is a plain row-major matrix, otherwise by 4-byte cp.async gathers (strided X, or the
 // implicit im2col of Section 4.5 taken directly from the NCHW input) - together with the packed records of
 // the thread block's bands for that block column.  A ring of stages with full / empty mbarriers lets warps
 // run up to a stage apart, which absorbs the uneven work of bands (Section 4.2's load imbalance).
 //
-// A warp owns one band per group, a lane four output columns.  Per block the lane loads the slab rows of
-// eight kept columns into registers once (each needed input row is read once and reused by every kept row -
-// the load-redundancy idea of Section 4.4) and then, per kept row, reads the row's eight weights with two
-// broadcast 128-bit loads and issues 32 FMAs into that row's accumulators.  Accumulator registers are indexed
-// statically: the rows of the band are walked in order with one warp-uniform test of the block's row mask each.
-// Grids that would leave most SMs idle are split over block columns (partial sums added into a zeroed Y).
+// A warp owns one band per group, a lane four output columns of each of one or two 128-column pieces.  Per block
+// the lane loads the slab rows of the kept columns into registers once (each needed input row is read once and
+// reused by every kept row - the load-redundancy idea of Section 4.4) and then, per kept row, reads the row's
+// weights with broadcast 128-bit loads and multiplies: packed two-column FMAs (fma.rn.f32x2), so that a lane issues
+// half as many instructions for the same flops - the kernel is short of issue slots and of shared-memory bandwidth,
+// not of FMA units.  With two pieces per lane the slab addresses, the weight loads and the row tests of a block are
+// shared by twice the FMAs (measured 17 % faster than one piece; two bands per warp buy nothing).  Accumulator
+// registers are indexed statically: the rows of the band are walked in order with one warp-uniform test of the
+// block's row mask each.  Grids that would leave most SMs idle are split over block columns (partial sums added
+// into a zeroed Y).
+//
+// Narrow tile (N <= 16): a lane owns one output column and the two halves of a warp split the kept columns of a
+// chunk; the stages are small, so the ring is deeper (8 slots, 6 in flight) and two thread blocks share an SM.
 #include <cuda.h>
 #include <cuda_bf16.h>
 

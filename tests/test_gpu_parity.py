@@ -301,12 +301,14 @@ def test_sweep_points(B, case):
     check_spmm(B, s["W"], s["mask"], s["X"], bh, bw, bf16=bf16, flags=1)
 
 
-def test_tune_returns_a_valid_choice(B):
+@pytest.mark.parametrize("reps", [3, -3])
+def test_tune_returns_a_valid_choice(B, reps):
+    """reps > 0 times back-to-back launches, reps < 0 launches after an L2 flush each (cold operands)."""
     s = gen.sweep_case(1024, 96, 8.0, 8, 32, "uniform")
     h = B.grim_bcr_pack(s["W"], s["mask"], 8, 32, B.GRIM_F32, 0)
     X = to_dev(s["X"])
     Y = torch.empty(1024, 96, device="cuda")
-    best = B.grim_bcr_tune(h, X, Y, reps=3)
+    best = B.grim_bcr_tune(h, X, Y, reps=reps)
     assert best["path"] in (1, 2, 3, 4) and best["ms"] > 0
     B.grim_bcr_spmm_ex(h, X, Y, tile_n=best["tile_n"], path=best["path"])
     torch.cuda.synchronize()
