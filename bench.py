@@ -959,6 +959,8 @@ def run_sweep(args):
         Xf = gen.normal_f32((M, max(ncols)), 1.0, 5, 33)
         for bf16, reorder in itertools.product([False, True], [1, 0]):
             h = B.grim_bcr_pack(W, mask, bh, bw, B.GRIM_BF16 if bf16 else B.GRIM_F32, reorder)
+            if bf16:
+                B.grim_bcr_reserve(h, min(max(ncols), 256))  # workspace of the split tensor-core multiply (small grids)
             info = B.grim_bcr_info(h)
             esz = 2 if bf16 else 4
             for N in ncols:
@@ -966,8 +968,11 @@ def run_sweep(args):
                 if bf16:
                     X = X.to(torch.bfloat16)
                 Y = torch.empty(M, N, device="cuda")
-                tc = bf16 and N >= 128
-                idx = info.index_bytes_gemv if N <= 16 else (info.index_bytes_tc if tc else info.index_bytes_spmm)
+                # the library's default routing: bf16 handles take the tensor-core tiles from N = 8, fp32 handles with
+                # blocks of 8 rows or more the CUDA-core kernel from N = 8, everything narrower the lane-per-column kernel
+                tc = bf16 and N >= 8
+                cuda_core = not tc and (N > 16 or (N >= 8 and bh >= 8 and not bf16))
+                idx = info.index_bytes_tc if tc else (info.index_bytes_spmm if cuda_core else info.index_bytes_gemv)
                 nbytes = float(info.value_bytes + idx + info.k_used * N * esz + M * N * 4)
                 flops = 2.0 * nnz * N
                 for _ in range(3):
@@ -982,12 +987,13 @@ def run_sweep(args):
                     e1.record()
                     e1.synchronize()
                     ms.append(e0.elapsed_time(e1))
+                status = B.grim_bcr_status(h)  # a bounded device-side wait that gave up leaves Y invalid: flag the record
                 t = statistics.median(ms) * 1e-3
                 t_hbm = nbytes / (peaks["hbm_gbs"] * 1e9)
                 t_flop = flops / (peaks["bf16_tflops_burst"] * 1e12 if tc else alu_peak)
                 rec = dict(M=M, N=N, c=c, block=f"{bh}x{bw}", dist=dist_name, dtype="bf16" if bf16 else "f32", reorder=reorder,
                            nnz=nnz, ms=t * 1e3, gflops=flops / t / 1e9, bound="hbm" if t_hbm >= t_flop else ("tensor" if tc else "alu"),
-                           frac=max(t_hbm, t_flop) / t, kernel="skinny" if N <= 16 else ("tc" if tc else "ffma"))
+                           frac=max(t_hbm, t_flop) / t, kernel="tc" if tc else ("ffma" if cuda_core else "stream"), status=int(status))
                 out.write(json.dumps(rec) + "\n")
                 fracs.append(rec["frac"])
                 n_runs += 1

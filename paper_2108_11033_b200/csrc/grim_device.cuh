@@ -157,33 +157,5 @@ __device__ __forceinline__ void expand_scatter(uint32_t rec_s, uint32_t bytes, u
   }
 }
 
-// The same expansion for a caller that has already read the first PRE 16-byte pieces of its share of the record
-// into registers (piece wt + i * NT in pre[i]; zeros past the end) - the reads then overlap the wait for the tile,
-// and only the clear, one barrier and the stores follow it.  Pieces beyond those are read here.
-template <int NT, int PRE>
-__device__ __forceinline__ void expand_scatter_pre(uint32_t rec_s, uint32_t n16, const uint4 (&pre)[PRE], uint32_t a_s,
-                                                   int wt, int bar_id) {
-#pragma unroll
-  for (int i = 0; i < 16384 / 16 / NT; ++i) sts128(a_s + (uint32_t)(wt + i * NT) * 16u, 0u, 0u, 0u, 0u);
-  named_barrier(bar_id, NT);
-#pragma unroll
-  for (int i = 0; i < PRE; ++i) {
-    if ((uint32_t)wt + (uint32_t)i * NT < n16) {
-      const uint4 e = pre[i];
-      sts16(a_s + (e.x >> 16), e.x);
-      sts16(a_s + (e.y >> 16), e.y);
-      sts16(a_s + (e.z >> 16), e.z);
-      sts16(a_s + (e.w >> 16), e.w);
-    }
-  }
-  for (uint32_t v = (uint32_t)wt + (uint32_t)PRE * NT; v < n16; v += NT) {
-    const uint4 e = lds128(rec_s + v * 16u);
-    sts16(a_s + (e.x >> 16), e.x);
-    sts16(a_s + (e.y >> 16), e.y);
-    sts16(a_s + (e.z >> 16), e.z);
-    sts16(a_s + (e.w >> 16), e.w);
-  }
-}
-
 }  // namespace ptx
 }  // namespace grim

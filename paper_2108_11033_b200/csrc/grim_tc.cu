@@ -32,8 +32,7 @@ constexpr int kTcWorkers = 12;     // warps that expand the packed weights; the 
 constexpr int kTcGroups = 3;       // the workers form groups that take K tiles in turn, so that expansions overlap
 constexpr int kTcGroupWarps = kTcWorkers / kTcGroups;
 constexpr int kTcGroupThreads = 32 * kTcGroupWarps;
-constexpr int kTcRecWarp = 2 + kTcWorkers;  // requests the packed records
-constexpr int kTcThreads = 64 + 32 * kTcWorkers + 32;  // warp 0: copies, warp 1: tensor core, the workers, the record warp
+constexpr int kTcThreads = 64 + 32 * kTcWorkers;  // warp 0: copies, warp 1: tensor core, then the workers
 constexpr int kTcBuilders = 12;    // convolution only: warps that build the X tile from the NCHW input
 constexpr int kTcBuildGroups = 3;  // they form groups that take K tiles in turn, like the expansion warps
 constexpr int kTcBuildGroupWarps = kTcBuilders / kTcBuildGroups;
@@ -45,7 +44,6 @@ constexpr int kTcStages = 4;        // ring slots at most; fewer when the packed
 constexpr int kATileBytes = kTM * kTK * 2;   // 16 KiB
 constexpr int kBTileBytes = kTQ * kTK * 2;   // 32 KiB
 constexpr int kTcHdrBytes = 1024;
-constexpr int kTcScatterPre = 4;   // 16-byte pieces of a record that a thread reads ahead of the tile slot
 constexpr int kTcRecSlots = 8;      // ring of packed records (small), deeper than the ring of tiles so that records
                                     // are on chip well before the weight tile they expand into becomes free
 constexpr unsigned kTmemCols = 256;
@@ -118,7 +116,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   uint64_t* built = empty + kTcStages;                         // convolution: the X tile of a stage is written
   uint64_t* acc_done = built + kTcStages;                      // all multiplies of the tile are complete
   uint64_t* rec_full = acc_done + 1;                           // a packed record has landed
-  uint64_t* rec_free = rec_full + kTcRecSlots;                 // ... and every warp of the group that expanded it has read it
+  unsigned* s_done = reinterpret_cast<unsigned*>(smem + 640);    // [record slot] warps that have finished expanding it
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
   uint64_t* seg_free = reinterpret_cast<uint64_t*>(smem + 704);  // staged convolution: the builders are done with a slot of planes
@@ -158,7 +156,7 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     }
     for (int s = 0; s < kTcRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
-      mbar_init(rec_free + s, kTcGroupWarps);
+      s_done[s] = 0;
     }
     mbar_init(acc_done, 1);
     *s_abort = 0;
@@ -173,11 +171,31 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
 
+  // Requests the packed records of K tile k (one per row tile) into record slot rs; one thread.
+  auto request_records = [&](int k, int rs) {
+    uint32_t bytes[2] = {0u, 0u}, off[2] = {0u, 0u}, total = 0;
+    for (int m = 0; m < p.mt; ++m) {
+      const int t = (int)blockIdx.y * p.mt + m;
+      if (t < p.mtiles) {
+        const RcStage se = p.stage[(int64_t)t * p.nkt + kbase + k];
+        bytes[m] = se.bytes; off[m] = se.off16;
+      }
+      s_meta[rs * 2 + m] = bytes[m];
+      total += bytes[m];
+    }
+    mbar_arrive_expect_tx(rec_full + rs, total);
+    for (int m = 0; m < p.mt; ++m)
+      if (bytes[m]) bulk_load(recs + (size_t)(rs * p.mt + m) * p.rec_stride, p.blob + (size_t)off[m] * 16, bytes[m], rec_full + rs);
+  };
+
   bool failed = false;
   int fail_site = 0;
   if (warp == 0) {
     // ------------------------------------------------------------------ copies
     if (lane == 0) {
+      // the first records (the ring of records is deeper than the ring of tiles); later ones are requested by the
+      // expansion warps as they free a record slot
+      for (int rk = 0; rk < nr && rk < nkt; ++rk) request_records(rk, rk);
       for (int kt = 0; kt < nkt && !CONV; ++kt) {  // the convolution builds its X tiles itself
         const int slot = kt % ns;
         if (kt >= ns && !mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort)) { failed = true, fail_site = 1; break; }
@@ -220,43 +238,9 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
       }
       if (!failed) umma_commit(acc_done);
     }
-  } else if (warp == kTcRecWarp) {
-    // ------------------------------------------------------------------ packed records, a ring of nr slots
-    // (a thread of their own: the table entry is a global load and the request a handful of dependent shared-memory
-    // accesses, which would otherwise sit in the expansion warps' critical path)
-    // The table entries are read 32 K tiles at a time, one per lane, so that no request waits for a global load.
-    for (int kt0 = 0; kt0 < nkt && !failed; kt0 += 32) {
-      RcStage mine[2];
-#pragma unroll
-      for (int m = 0; m < 2; ++m) {
-        mine[m].off16 = 0; mine[m].bytes = 0;
-        const int t = (int)blockIdx.y * p.mt + m;
-        if (m < p.mt && t < p.mtiles && kt0 + lane < nkt) mine[m] = p.stage[(int64_t)t * p.nkt + kbase + kt0 + lane];
-      }
-      const int n = nkt - kt0 < 32 ? nkt - kt0 : 32;
-      for (int i = 0; i < n; ++i) {
-        const int kt = kt0 + i, rs = kt % nr;
-        uint32_t bytes[2], off[2];
-#pragma unroll
-        for (int m = 0; m < 2; ++m) {
-          bytes[m] = __shfl_sync(0xffffffffu, mine[m].bytes, i);
-          off[m] = __shfl_sync(0xffffffffu, mine[m].off16, i);
-        }
-        if (kt >= nr && !__all_sync(0xffffffffu, mbar_wait(rec_free + rs, (unsigned)((kt / nr - 1) & 1), p.spin_limit, s_abort, 20))) { failed = true, fail_site = 7; break; }
-        if (lane == 0) {
-          s_meta[rs * 2] = bytes[0];
-          s_meta[rs * 2 + 1] = bytes[1];
-          mbar_arrive_expect_tx(rec_full + rs, bytes[0] + bytes[1]);
-#pragma unroll
-          for (int m = 0; m < 2; ++m)
-            if (bytes[m]) bulk_load(recs + (size_t)(rs * p.mt + m) * p.rec_stride, p.blob + (size_t)off[m] * 16, bytes[m], rec_full + rs);
-        }
-        __syncwarp();
-      }
-    }
-  } else if (CONV && warp > kTcRecWarp) {
+  } else if (CONV && warp >= 2 + kTcWorkers) {
     // ------------------------------------------------------------------ implicit im2col (3x3, stride 1, pad 1)
-    const int bgrp = (warp - kTcRecWarp - 1) / kTcBuildGroupWarps;
+    const int bgrp = (warp - 2 - kTcWorkers) / kTcBuildGroupWarps;
     const int bt = tid - kTcThreads - bgrp * (32 * kTcBuildGroupWarps);  // 0 .. 127 inside the group
     if (!conv_build_tiles<CONV>(im, bgrp, kTcBuildGroups, bt, lane, fail_site)) failed = true;
   } else {
@@ -265,42 +249,26 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
     const int wt = tid - 64 - grp * kTcGroupThreads;           // 0 .. kTcGroupThreads - 1 inside the group
     for (int kt = grp; kt < nkt; kt += kTcGroups) {
       const int slot = kt % ns, rs = kt % nr;
-      // The record(s) first: the entries are read into registers while the tile slot may still be in use, so that
-      // between the slot coming free and the tile being ready lie only the clear, one barrier and the stores.
-      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
-      uint4 pre[2][kTcScatterPre];
-      uint32_t n16[2] = {0u, 0u};
-      bool all_read = true;  // (uniform over the group)
-#pragma unroll
-      for (int m = 0; m < 2; ++m) {
-        if (m < p.mt) {
-          const uint32_t rec_s = smem_u32(recs + (size_t)(rs * p.mt + m) * p.rec_stride);
-          n16[m] = s_meta[rs * 2 + m] >> 4;
-#pragma unroll
-          for (int i = 0; i < kTcScatterPre; ++i) {
-            const uint32_t v = (uint32_t)wt + (uint32_t)i * kTcGroupThreads;
-            pre[m][i] = v < n16[m] ? ptx::lds128(rec_s + v * 16u) : make_uint4(0u, 0u, 0u, 0u);
-          }
-          all_read = all_read && n16[m] <= (uint32_t)(kTcScatterPre * kTcGroupThreads);
-        }
-      }
-      __syncwarp();
-      if (all_read && lane == 0) mbar_arrive(rec_free + rs);
+      // the weight tile of the slot is free once the multiplies of its previous use are done; the record is
+      // normally long there
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 4; break; }
+      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
       uint8_t* st = stages + (size_t)slot * stage_bytes;
       // clear the tile, meet, then one 2-byte store per kept value at the offset stored beside it
-#pragma unroll
-      for (int m = 0; m < 2; ++m)
-        if (m < p.mt)
-          ptx::expand_scatter_pre<kTcGroupThreads, kTcScatterPre>(smem_u32(recs + (size_t)(rs * p.mt + m) * p.rec_stride), n16[m], pre[m],
-                                                                  smem_u32(st + m * kATileBytes), wt, 1 + grp);
-      if (!all_read) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(rec_free + rs);
-      }
+      for (int m = 0; m < p.mt; ++m)
+        ptx::expand_scatter<kTcGroupThreads>(smem_u32(recs + (size_t)(rs * p.mt + m) * p.rec_stride), s_meta[rs * 2 + m],
+                                             smem_u32(st + m * kATileBytes), wt, 1 + grp);
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // generic-proxy writes -> visible to the tensor core
       __syncwarp();
-      if (lane == 0) mbar_arrive(ready + slot);
+      if (lane == 0) {
+        mbar_arrive(ready + slot);
+        // the last warp of the group to finish with the record frees its slot: it requests the record that uses
+        // the slot next (every read of the old record precedes that warp's count)
+        if (atomicAdd(s_done + rs, 1u) == (unsigned)kTcGroupWarps - 1u) {
+          s_done[rs] = 0;
+          if (kt + nr < nkt) request_records(kt + nr, rs);
+        }
+      }
       if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     }
     // ------------------------------------------------------------------ epilogue

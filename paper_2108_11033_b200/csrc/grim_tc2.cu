@@ -32,9 +32,8 @@ namespace {
 using namespace ptx;
 
 constexpr int kWorkers = 12, kGroups = 3, kGroupWarps = kWorkers / kGroups, kGroupThreads = 32 * kGroupWarps;
-constexpr int kIssueWarp2 = 2 + kWorkers;  // second issuing warp
-constexpr int kRecWarp = kIssueWarp2 + 1;  // requests the packed records
-constexpr int kThreads = 64 + 32 * kWorkers + 64;
+constexpr int kIssueWarp2 = 2 + kWorkers;  // second issuing warp (the last warp of the block)
+constexpr int kThreads = 64 + 32 * kWorkers + 32;
 constexpr int kBuilders = 12, kBuildGroups = 3;  // convolution only: warps that build the X tile from the NCHW input
 constexpr int kConvThreads = kThreads + 32 * kBuilders;
 constexpr int kRows = 128;              // rows of W per block
@@ -42,7 +41,6 @@ constexpr int kColsPerBlock = 256;      // X columns staged per block per K tile
 constexpr int kPairCols = 512;          // output columns per pair
 constexpr int kK = 64;                  // K per stage
 constexpr int kMaxStages = 4, kRecSlots = 8;
-constexpr int kScatterPre = 4;  // 16-byte pieces of a record that a thread reads ahead of the tile slot
 constexpr int kABytes = kRows * kK * 2;            // 16 KiB
 constexpr int kBBytes = kColsPerBlock * kK * 2;    // 32 KiB
 constexpr int kStageBytes = kABytes + kBBytes;
@@ -125,10 +123,10 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
   uint64_t* empty = ready + kMaxStages;                   // the pair's multiplies on a stage are done (set in both blocks)
   uint64_t* acc_done = empty + kMaxStages;                // all multiplies are complete (set in both blocks)
   uint64_t* rec_full = acc_done + 1;                      // a packed record has landed
-  uint64_t* rec_free = rec_full + kRecSlots;              // ... and every warp of the group that expanded it has read it
   uint32_t* s_tmem = reinterpret_cast<uint32_t*>(smem + 384);
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 388);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 512);  // [record slot] bytes of the record (0: the tile is empty)
+  unsigned* s_done = reinterpret_cast<unsigned*>(smem + 640);  // [record slot] warps that have finished with it
   uint64_t* seg_full = reinterpret_cast<uint64_t*>(smem + 704);  // staged convolution: the planes of a K tile have landed
   uint64_t* seg_free = reinterpret_cast<uint64_t*>(smem + 768);  // ... and the builders are done with them
   uint8_t* stages = smem + kHdrBytes;
@@ -155,7 +153,7 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
     }
     for (int s = 0; s < kRecSlots; ++s) {
       mbar_init(rec_full + s, 1);
-      mbar_init(rec_free + s, kGroupWarps);
+      s_done[s] = 0;
     }
     mbar_init(acc_done, 2);
     *s_abort = 0;
@@ -171,6 +169,18 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
 
+  // Requests the packed record of K tile k into record slot rs; one thread.
+  auto request_record = [&](int k, int rs) {
+    uint32_t bytes = 0, off = 0;
+    if (has_tile) {
+      const RcStage se = p.stage[(int64_t)tile * p.nkt + k];
+      bytes = se.bytes; off = se.off16;
+    }
+    s_meta[rs] = bytes;
+    mbar_arrive_expect_tx(rec_full + rs, bytes);
+    if (bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)off * 16, bytes, rec_full + rs);
+  };
+
   bool failed = false;
   int fail_site = 0;
   Im2colCtx im;
@@ -184,8 +194,12 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
   if (warp == 0) {
     // ------------------------------------------------------------------ copies
     if (CONV) {
+      if (lane == 0)
+        for (int rk = 0; rk < nr && rk < nkt; ++rk) request_record(rk, rk);
+      __syncwarp();
       if (CONV >= 2 && !conv_copy_planes<CONV>(im, lane)) failed = true, fail_site = 1;
     } else if (lane == 0) {
+      for (int rk = 0; rk < nr && rk < nkt; ++rk) request_record(rk, rk);
       // 64-column boxes wholly past the last column are not requested (their part of the tile keeps whatever it
       // held; the accumulator columns computed from it are never stored)
       auto boxes_from = [&](int64_t first) {
@@ -250,31 +264,9 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
       if (!failed) umma2_commit_both(acc_done);
       if (!failed && (p.flags & 1)) umma2_commit_both(acc_done);
     }
-  } else if (warp == kRecWarp) {
-    // ------------------------------------------------------------------ packed records, a ring of nr slots
-    // (their own thread: the table entry is a global load and the request a handful of dependent shared-memory
-    // accesses, which would otherwise sit in the expansion warps' critical path)
-    // The table entries are read 32 K tiles at a time, one per lane, so that no request waits for a global load.
-    for (int kt0 = 0; kt0 < nkt && !failed; kt0 += 32) {
-      RcStage mine;
-      mine.off16 = 0; mine.bytes = 0;
-      if (has_tile && kt0 + lane < nkt) mine = p.stage[(int64_t)tile * p.nkt + kt0 + lane];
-      const int n = nkt - kt0 < 32 ? nkt - kt0 : 32;
-      for (int i = 0; i < n; ++i) {
-        const int kt = kt0 + i, rs = kt % nr;
-        const uint32_t bytes = __shfl_sync(0xffffffffu, mine.bytes, i), off = __shfl_sync(0xffffffffu, mine.off16, i);
-        if (kt >= nr && !__all_sync(0xffffffffu, mbar_wait<true>(rec_free + rs, (unsigned)((kt / nr - 1) & 1), p.spin_limit, s_abort, 20))) { failed = true, fail_site = 7; break; }
-        if (lane == 0) {
-          s_meta[rs] = bytes;
-          mbar_arrive_expect_tx(rec_full + rs, bytes);
-          if (bytes) bulk_load(recs + (size_t)rs * p.rec_stride, p.blob + (size_t)off * 16, bytes, rec_full + rs);
-        }
-        __syncwarp();
-      }
-    }
-  } else if (CONV && warp > kRecWarp) {
+  } else if (CONV && warp > kIssueWarp2) {
     // ------------------------------------------------------------------ implicit im2col: this block's 256 pixels
-    const int bgrp = (warp - kRecWarp - 1) / kImBuildWarps;
+    const int bgrp = (warp - kIssueWarp2 - 1) / kImBuildWarps;
     const int bt = tid - kThreads - bgrp * (32 * kImBuildWarps);
     if (!conv_build_tiles<CONV>(im, bgrp, kBuildGroups, bt, lane, fail_site)) failed = true;
   } else {
@@ -283,31 +275,21 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
     const int wt = tid - 64 - grp * kGroupThreads;
     for (int kt = grp; kt < nkt; kt += kGroups) {
       const int slot = kt % ns, rs = kt % nr;
-      // The record first: its entries are read into registers while the tile slot may still be in use, so that
-      // between the slot coming free and the tile being ready lie only the clear, one barrier and the stores.
-      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
-      const uint32_t rec_s = smem_u32(recs + (size_t)rs * p.rec_stride);
-      const uint32_t n16 = s_meta[rs] >> 4;
-      uint4 pre[kScatterPre];
-#pragma unroll
-      for (int i = 0; i < kScatterPre; ++i) {
-        const uint32_t v = (uint32_t)wt + (uint32_t)i * kGroupThreads;
-        pre[i] = v < n16 ? lds128(rec_s + v * 16u) : make_uint4(0u, 0u, 0u, 0u);
-      }
-      const bool all_read = n16 <= (uint32_t)(kScatterPre * kGroupThreads);  // (uniform over the group)
-      __syncwarp();
-      if (all_read && lane == 0) mbar_arrive(rec_free + rs);
       if (kt >= ns && !__all_sync(0xffffffffu, mbar_wait<true>(empty + slot, (unsigned)((kt / ns - 1) & 1), p.spin_limit, s_abort, 32))) { failed = true, fail_site = 4; break; }
-      expand_scatter_pre<kGroupThreads, kScatterPre>(rec_s, n16, pre, smem_u32(stages + (size_t)slot * kStageBytes), wt, 1 + grp);
-      if (!all_read) {
-        __syncwarp();
-        if (lane == 0) mbar_arrive(rec_free + rs);
-      }
+      if (!__all_sync(0xffffffffu, mbar_wait(rec_full + rs, (unsigned)((kt / nr) & 1), p.spin_limit, s_abort))) { failed = true, fail_site = 5; break; }
+      expand_scatter<kGroupThreads>(smem_u32(recs + (size_t)rs * p.rec_stride), s_meta[rs],
+                                    smem_u32(stages + (size_t)slot * kStageBytes), wt, 1 + grp);
       fence_proxy_async();  // generic-proxy writes -> visible to the tensor core
       __syncwarp();
       if (lane == 0) {
         if (rank == 0) mbar_arrive(ready + slot);
         else mbar_arrive_remote(ready + slot, 0);
+        // the last warp of the group to finish with the record frees its slot: it requests the record that uses
+        // the slot next (every read of the old record precedes that warp's count)
+        if (atomicAdd(s_done + rs, 1u) == (unsigned)kGroupWarps - 1u) {
+          s_done[rs] = 0;
+          if (kt + nr < nkt) request_record(kt + nr, rs);
+        }
       }
     }
     // ------------------------------------------------------------------ epilogue
