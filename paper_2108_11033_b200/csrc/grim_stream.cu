@@ -198,6 +198,12 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
   const int q0 = blockIdx.y * NQ;
   const int nslots = p.nslots;
 
+  // Programmatic dependent launch: the launch that follows in the stream may start as soon as SMs free up (this
+  // kernel reads nothing an earlier launch wrote until the wait below), and this one, if it was launched that way
+  // itself, has come this far while its predecessor was still running.  Until the wait it touches only the packed
+  // matrix (immutable) and its own shared memory: tables, barriers and the first weight copies are under way when
+  // the predecessor ends, which hides most of a launch's fixed cost in a chain of back-to-back products.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   if (threadIdx.x == 0) *s_abort = 0;
   if (lane == 0) {
     for (int s = 0; s < kSMaxSlots; ++s) mbar_init(my_full + s, 1);
@@ -260,6 +266,9 @@ __global__ void __launch_bounds__(NW * 32, 1) bcr_stream_kernel(const StreamPara
       if (s < nslots) issue(first[s], s);
   }
   RunFetch pend0 = prepare(), pend1 = prepare();
+
+  // everything earlier launches in the stream wrote (X, a cleared Y) is complete and visible from here on
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (XS && NQ == 1) {
     XT* sx = reinterpret_cast<XT*>(smem + p.off_x);
@@ -495,8 +504,17 @@ cudaError_t launch_kernel(const StreamParams& p, const StreamPlan& pl, cudaStrea
   auto kern = bcr_stream_kernel<BH, NQ, NW, XS, VT, VT>;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), pl.smem);
   if (e != cudaSuccess) return e;
-  kern<<<dim3((unsigned)pl.grid_x, (unsigned)pl.passes), NW * 32, pl.smem, s>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((unsigned)pl.grid_x, (unsigned)pl.passes);
+  cfg.blockDim = dim3(NW * 32);
+  cfg.dynamicSmemBytes = pl.smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may overlap the tail of the launch before it
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, p);
 }
 
 template <int BH, typename VT>

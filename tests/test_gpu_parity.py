@@ -301,6 +301,33 @@ def test_sweep_points(B, case):
     check_spmm(B, s["W"], s["mask"], s["X"], bh, bw, bf16=bf16, flags=1)
 
 
+@pytest.mark.parametrize("N", [1, 4])
+def test_streaming_kernel_chained_launches(B, N):
+    """The streaming kernel is launched with programmatic stream serialization: a launch may begin (tables, barriers,
+    first weight copies) while the launch before it still runs, and waits for it before it reads X or writes Y.  A chain
+    of dependent products through two ping-pong buffers, queued without any host synchronisation, must therefore give
+    what the oracle gives step by step - both the read-after-write (X of a step is Y of the step before) and the
+    write-after-read (Y of a step is X of the step before) orders are exercised."""
+    M = 2048
+    s = gen.sweep_case(M, N, 4.0, 8, 32, "uniform")
+    W = (s["W"] * 8.0).astype(np.float32)  # keeps the iterates at the same scale from step to step
+    h = B.grim_bcr_pack(W, s["mask"], 8, 32, B.GRIM_F32, 1)
+    try:
+        bufs = [to_dev(s["X"]), torch.empty(M, N, device="cuda")]
+        steps = 6
+        for i in range(steps):
+            B.grim_bcr_spmm_ex(h, bufs[i & 1], bufs[(i + 1) & 1], path=3, tile_n=2)
+        torch.cuda.synchronize()
+        assert B.grim_bcr_status(h) == B.GRIM_OK
+        want = s["X"].astype(np.float64)
+        for i in range(steps):
+            want = orc.spmm(W, s["mask"], want.astype(np.float32)).astype(np.float64)
+        got = bufs[steps & 1].cpu().numpy()
+        assert rel_fro(got, want) <= 10 * F32_TOL, rel_fro(got, want)
+    finally:
+        B.grim_bcr_destroy(h)
+
+
 @pytest.mark.parametrize("reps", [3, -3])
 def test_tune_returns_a_valid_choice(B, reps):
     """reps > 0 times back-to-back launches, reps < 0 launches after an L2 flush each (cold operands)."""
