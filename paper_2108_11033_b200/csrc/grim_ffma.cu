@@ -170,6 +170,9 @@ __global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(co
   extern __shared__ __align__(128) uint8_t smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);
   uint64_t* empty = full + kMaxRing;
+  // the launch that follows in the stream may start as SMs free up: it waits (griddepcontrol.wait) before it reads or
+  // writes anything this launch touches
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   volatile int* s_abort = reinterpret_cast<volatile int*>(smem + 128);
   int* s_nst = reinterpret_cast<int*>(smem + 132);
   uint32_t* s_meta = reinterpret_cast<uint32_t*>(smem + 192);               // [ring slot][4] blob bytes per band group
@@ -209,6 +212,9 @@ __global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(co
     }
   }
   __syncthreads();
+  // (programmatic dependent launch) whatever earlier launches in the stream wrote - X, a cleared scratch or Y - is
+  // complete and visible from here on; up to here only the packed matrix and this block's own shared memory were touched
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   // with a split over block columns this thread block multiplies only its share of the stage list
   const int nst_all = *s_nst;
   const int n_lo = (int)((int64_t)blockIdx.z * nst_all / p.ksplit), n_hi = (int)((int64_t)(blockIdx.z + 1) * nst_all / p.ksplit);
@@ -630,8 +636,7 @@ cudaError_t launch_variant(const CUtensorMap& tm, const FParams& p, size_t smem,
   auto kern = bcr_ffma_kernel<BH, BPW, CW, XT, MODE>;
   cudaError_t e = ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem);
   if (e != cudaSuccess) return e;
-  kern<<<grid, kFThreads, smem, s>>>(tm, p);
-  return cudaGetLastError();
+  return launch_pdl(kern, grid, dim3(kFThreads), smem, s, tm, p);
 }
 
 // The accumulators of a lane take BH * BPW * CW * 4 registers: at most 64.

@@ -211,4 +211,21 @@ int sm_count(int device);
 // kept by the kernel, so it is set once per kernel and size, not per launch)
 cudaError_t ensure_dynamic_smem(const void* kernel, size_t bytes);
 
+// Launch with programmatic stream serialization: the kernel may begin while the launch before it in the stream still
+// runs; it calls griddepcontrol.wait before it touches anything but the packed matrix and its own shared memory.
+template <typename K, typename... A>
+cudaError_t launch_pdl(K kern, dim3 grid, dim3 block, size_t smem, cudaStream_t s, A... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, args...);
+}
+
 }  // namespace grim

@@ -109,6 +109,9 @@ template <int BH, int CONV>
 __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_kernel(const __grid_constant__ CUtensorMap tmX, const TcParams p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles must start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes)
+  // the launch that follows in the stream may start as SMs free up: it waits (griddepcontrol.wait) before it reads or
+  // writes anything this launch touches
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem);        // the X tile of a stage has landed
   uint64_t* ready = full + kTcStages;                        // the expanded weight tile of a stage is written
@@ -170,6 +173,9 @@ __global__ void __launch_bounds__(CONV ? kTcConvThreads : kTcThreads, 1) bcr_tc_
   __syncthreads();
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
+  // (programmatic dependent launch) whatever earlier launches in the stream wrote - X, a cleared scratch or Y - is
+  // complete and visible from here on; up to here only the packed matrix and this block's own shared memory were touched
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // Requests the packed records of K tile k (one per row tile) into record slot rs; one thread.
   auto request_records = [&](int k, int rs) {
@@ -525,9 +531,9 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
     const size_t smem = tc_smem_need(h, p.mt, p.nstages, p.nrec, extra);
     if (ensure_dynamic_smem(reinterpret_cast<const void*>(kern), smem) != cudaSuccess) return GRIM_ERR_CUDA;
     dim3 grid((unsigned)((a.ncols + kTQ - 1) / kTQ), (unsigned)((h->tc_mtiles + p.mt - 1) / p.mt), (unsigned)p.ksplit);
-    kern<<<grid, kTcConvThreads, smem, s>>>(tm, p);
+    const cudaError_t le = launch_pdl(kern, grid, dim3(kTcConvThreads), smem, s, tm, p);
     count_launch();
-    if (cudaGetLastError() != cudaSuccess) return GRIM_ERR_CUDA;
+    if (le != cudaSuccess) { cudaGetLastError(); return GRIM_ERR_CUDA; }
     return finalize();
   }
   const cuuint64_t dims[2] = {(cuuint64_t)a.ncols, (cuuint64_t)h->K};
@@ -545,9 +551,9 @@ grim_status_t launch_spmm_tc(const grim_bcr* h, const SpmmArgs& a, cudaStream_t 
   const int64_t qtiles = (a.ncols + kTQ - 1) / kTQ;
   const int64_t mtiles = (h->tc_mtiles + p.mt - 1) / p.mt;
   dim3 grid((unsigned)qtiles, (unsigned)mtiles, (unsigned)p.ksplit);
-  kern<<<grid, kTcThreads, smem, s>>>(tm, p);
+  const cudaError_t le = launch_pdl(kern, grid, dim3(kTcThreads), smem, s, tm, p);
   count_launch();
-  if (cudaGetLastError() != cudaSuccess) return GRIM_ERR_CUDA;
+  if (le != cudaSuccess) { cudaGetLastError(); return GRIM_ERR_CUDA; }
   return finalize();
 }
 

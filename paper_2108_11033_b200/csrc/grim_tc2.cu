@@ -112,6 +112,9 @@ template <int CONV>
 __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_kernel(const __grid_constant__ CUtensorMap tmX, const Tc2Params p) {
   extern __shared__ uint8_t smem_raw[];
   // tiles start on a 1 KiB boundary (the swizzle pattern repeats every 8 rows of 128 bytes); the offset from the
+  // the launch that follows in the stream may start as SMs free up: it waits (griddepcontrol.wait) before it reads or
+  // writes anything this launch touches
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
   // start of the block's shared memory is the same in both blocks, which the paired multiply relies on
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   // One barrier per stage IN THE EVEN BLOCK collects everything the multiplies of that stage need from both blocks:
@@ -168,6 +171,9 @@ __global__ void __launch_bounds__(CONV ? kConvThreads : kThreads, 1) bcr_tc2_ker
   cluster_sync_all();  // both blocks' barriers exist before either signals the other
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem_base = *s_tmem;
+  // (programmatic dependent launch) whatever earlier launches in the stream wrote - X, a cleared scratch or Y - is
+  // complete and visible from here on; up to here only the packed matrix and this block's own shared memory were touched
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   // Requests the packed record of K tile k into record slot rs; one thread.
   auto request_record = [&](int k, int rs) {
@@ -485,13 +491,15 @@ grim_status_t launch_spmm_tc2(const grim_bcr* h, const SpmmArgs& a, cudaStream_t
   cfg.blockDim = dim3(a.conv ? kConvThreads : kThreads);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = 2;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // may begin while the launch before it still runs
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   const cudaError_t e = cudaLaunchKernelEx(&cfg, kern, tm, p);
   count_launch();
   return e == cudaSuccess ? GRIM_OK : GRIM_ERR_CUDA;
