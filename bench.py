@@ -1031,6 +1031,53 @@ def run_bcrc_study(args):
                               total_saving=1.0 - (bcrc + 4 * nnz) / (csr + 4 * nnz))))
 
 
+def run_reorder_study(args):
+    """What the band schedule (Section 4.2, GRIM_PACK_REORDER) buys when the work per band is skewed: matrices whose
+    bands get Zipf-distributed shares of the kept columns (generators.bcr_keep_lists, band_zipf), timed with the
+    schedule off and on through the library's default routing.  One JSON line per point."""
+    import torch
+    torch.cuda.set_device(0)
+    from paper_2108_11033_b200.build import build_library
+    build_library()
+    from paper_2108_11033_b200 import binding as B
+    from workloads import generators as gen
+    flush = torch.empty(1 << 30, dtype=torch.uint8, device="cuda")
+    for M, skew, bf16 in [(4096, 1.0, False), (8192, 1.0, False), (8192, 0.5, False), (8192, 1.0, True)]:
+        W = gen.dense_weight(M, M, 7, 41)
+        mask = gen.bcr_mask(M, M, 8, 32, compression=8.0, dist="uniform", seed=7, stream=42, band_zipf=skew)
+        band = mask.reshape(M // 8, 8, M).sum(axis=(1, 2))
+        Xf = gen.normal_f32((M, 1024), 1.0, 7, 43)
+        times = {}
+        for reorder in (0, 1):
+            h = B.grim_bcr_pack(W, mask, 8, 32, B.GRIM_BF16 if bf16 else B.GRIM_F32, reorder)
+            if bf16:
+                B.grim_bcr_reserve(h, 256)
+            for N in (1, 16, 128, 1024):
+                X = torch.from_numpy(np.ascontiguousarray(Xf[:, :N])).cuda()
+                X = X.to(torch.bfloat16) if bf16 else X
+                Y = torch.empty(M, N, device="cuda")
+                for _ in range(3):
+                    B.grim_bcr_spmm(h, X, Y)
+                ms = []
+                for _ in range(args.steps if args.steps < 50 else 7):
+                    flush.zero_()
+                    flush[: 1 << 29].view(torch.int64).sum()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    B.grim_bcr_spmm(h, X, Y)
+                    e1.record()
+                    e1.synchronize()
+                    ms.append(e0.elapsed_time(e1))
+                assert B.grim_bcr_status(h) == 0
+                times[(reorder, N)] = statistics.median(ms)
+            B.grim_bcr_destroy(h)
+        for N in (1, 16, 128, 1024):
+            print(json.dumps(dict(M=M, N=N, dtype="bf16" if bf16 else "f32", band_zipf=skew, nnz=int(mask.sum()),
+                                  heaviest_band_over_mean=float(band.max() / band.mean()),
+                                  ms_schedule_off=times[(0, N)], ms_schedule_on=times[(1, N)],
+                                  off_over_on=times[(0, N)] / times[(1, N)])), flush=True)
+
+
 def run_block_sweep(args):
     """Time against number of blocks for one 1024 x 1024 matrix at 10x (the experiment of Section 5.1, left panel of its
     figure) with the block shapes the packer takes, and the block size the search of that section then picks."""
@@ -1076,7 +1123,11 @@ def main():
     ap.add_argument("--out", default="sweep.jsonl")
     ap.add_argument("--bcrc-study", action="store_true", help="host only: index bytes of the BCRC export against CSR")
     ap.add_argument("--block-sweep", action="store_true", help="time vs number of blocks at 1024 x 1024, 10x, and the block-size search")
+    ap.add_argument("--reorder-study", action="store_true", help="band schedule off / on for matrices with skewed work per band")
     args = ap.parse_args()
+    if args.reorder_study:
+        run_reorder_study(args)
+        return
     if args.block_sweep:
         run_block_sweep(args)
         return

@@ -68,7 +68,7 @@ def _kr_pmf(h: int, dist: str, zipf_s: float) -> np.ndarray:
 def bcr_keep_lists(M: int, K: int, bh: int, bw: int, *, compression: float | None = None,
                    dist: str = "uniform", seed: int = 0, stream: int = 100,
                    kr_fixed: int | None = None, kc_fixed: int | None = None,
-                   zipf_s: float = 1.2, empty_frac: float = 0.0):
+                   zipf_s: float = 1.2, empty_frac: float = 0.0, band_zipf: float = 0.0):
     """Draw per-block keep flags.
 
     Returns (rowkeep, colkeep): bool arrays of shape (nbr, nbc, bh) and (nbr, nbc, bw).
@@ -78,6 +78,9 @@ def bcr_keep_lists(M: int, K: int, bh: int, bw: int, *, compression: float | Non
     dist = "uniform": kept-row count uniform on 1..bh.  dist = "zipf": P(kr = k) ~ k^-s.
     In the last two the kept-column count is chosen per block so that the expected tile
     size is bh*bw/compression: kc = floor(t) + [u < frac(t)], t = clamp(s / E[kr], 1, bw).
+    band_zipf > 0 makes whole block rows (bands) heavy or light: band i gets the share rank_i^-band_zipf of the
+    kept columns (ranks are a random permutation of the bands, shares scaled to mean 1), so that the work per band
+    is skewed the way the kept-row counts are skewed per block - the case a band schedule has something to balance.
     """
     g = rng(seed, stream)
     nbr = -(-M // bh)
@@ -101,6 +104,9 @@ def bcr_keep_lists(M: int, K: int, bh: int, bw: int, *, compression: float | Non
             kr[sel] = 1 + np.searchsorted(cdf, u_kr[sel], side="right").clip(0, h - 1)
             ekr[sel] = float((pmf * np.arange(1, h + 1)).sum())
         s = HB * WB / float(compression)
+        if band_zipf > 0.0:
+            share = (1.0 + g.permutation(nbr)) ** (-float(band_zipf))
+            s = s * (share / share.mean())[:, None]
         t = np.clip(s / ekr, 1.0, WB)
         u_kc = g.random((nbr, nbc))
         kc = (np.floor(t) + (u_kc < (t - np.floor(t)))).astype(np.int64)
