@@ -26,6 +26,7 @@
 #include <algorithm>
 #include <cstring>
 
+#include "grim_device.cuh"
 #include "grim_internal.h"
 
 namespace grim {
@@ -60,45 +61,9 @@ struct FParams {
   SpmmArgs a;
 };
 
-// ---- mbarrier / async-copy wrappers -----------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
-  unsigned ok;
-  asm volatile(
-      "{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0, 1, 0, p;\n}"
-      : "=r"(ok)
-      : "r"(smem_u32(bar)), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-// Bounded wait: false when the limit ran out (the caller then raises the abort flag and leaves).
-__device__ __forceinline__ bool mbar_wait(uint64_t* bar, unsigned parity, unsigned limit, const volatile int* abort_flag) {
-  for (unsigned i = 0; i < limit; ++i) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((i & 63u) == 63u && *abort_flag) return false;
-  }
-  return false;
-}
-__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* tm, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(smem_u32(dst)), "l"(tm), "r"(x), "r"(y), "r"(smem_u32(bar))
-      : "memory");
-}
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar))
-               : "memory");
-}
+// (mbarrier, bulk-copy and TMA wrappers: grim_device.cuh)
+using namespace ptx;
+
 __device__ __forceinline__ void cp_async4_zfill(void* dst, const void* src, bool valid) {
   const unsigned n = valid ? 4u : 0u;
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(smem_u32(dst)), "l"(src), "r"(n) : "memory");
@@ -116,9 +81,6 @@ __device__ __forceinline__ void gather_elem(float* dst, const void* X, int64_t o
 }
 __device__ __forceinline__ void cp_async16_cg(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_arrive_noinc(uint64_t* bar) {
-  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 
 // Four neighbouring slab elements of one row as two packed pairs (fp32 bit patterns, low word = lower column).
@@ -208,7 +170,7 @@ __global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(co
         mbar_init(full + s, MODE == kModeTma ? 1u : (unsigned)kFThreads);
         mbar_init(empty + s, kFWarps);
       }
-      asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+      fence_mbar_init();
     }
   }
   __syncthreads();
@@ -343,7 +305,7 @@ __global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(co
       const bool mine = MODE != kModeTma || (warp == (n % kFWarps) && lane == 0);
       if (mine) {
         bool ok = true;
-        if (m >= NS) ok = mbar_wait(empty + m % NS, (unsigned)((m / NS - 1) & 1), p.spin_limit, s_abort);
+        if (m >= NS) ok = mbar_wait(empty + m % NS, (unsigned)((m / NS - 1) & 1), p.spin_limit, s_abort, 0);
         if (ok) request(m);
         else failed = true;
       }
@@ -351,7 +313,7 @@ __global__ void __launch_bounds__(kFThreads, CW == 0 ? 2 : 1) bcr_ffma_kernel(co
     if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     // ---- wait for stage n
     const int slot = n % NS;
-    if (!mbar_wait(full + slot, (unsigned)((n / NS) & 1), p.spin_limit, s_abort)) failed = true;
+    if (!mbar_wait(full + slot, (unsigned)((n / NS) & 1), p.spin_limit, s_abort, 0)) failed = true;
     if (__any_sync(0xffffffffu, failed)) { failed = true; break; }
     const uint8_t* base = slots + (size_t)slot * slot_bytes;
     const XT* slab = reinterpret_cast<const XT*>(base);
