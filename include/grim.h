@@ -188,7 +188,9 @@ grim_status_t grim_bcr_unpack_dense(grim_bcr_t h, float* W_host, int64_t ldw);
  * after fp32 accumulation).  Y is fully overwritten (all M rows, beta = 0): rows kept by no
  * block are written as +0.  N = 1 selects the matrix-vector kernel.  X and Y must not overlap.
  * Shape mismatch -> GRIM_ERR_SHAPE, dtype mismatch -> GRIM_ERR_DTYPE, both before any launch.
- * Asynchronous on `stream`; never allocates.  A handle is used on one stream at a time.
+ * Asynchronous on `stream`; never allocates.  A handle is used on one stream at a time.  The kernels are launched
+ * with programmatic stream serialization: their set-up may overlap the end of the launch before them on the stream,
+ * and they wait for that launch to complete before they read X or write Y - stream order is what the caller sees.
  * Without an explicit choice (grim_bcr_spmm_ex) the kernel and tile shape are the ones grim_bcr_tune found for
  * this handle and this kind of request (same power-of-two bucket of N, same dtypes), else a static default.
  */
